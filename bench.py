@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the BPTT training step: sample-timesteps/s per checkpoint strategy.
+
+Default arm: the CUDA library on workload c2 (2 recurrent LIF layers 512-1024-1024-20, T = 1000,
+batch 32, Chunk checkpointing every 32 steps), one process per GPU; with several GPUs every rank
+runs an independent replica (the step does not shard: no collective).  One JSON line on rank 0.
+
+`--impl reference` times the CPU oracle as it stands on the host cores, each step a bounded
+sample (the first T' steps) of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import snn_workloads as wl  # noqa: E402
+
+METRIC = "sample_timesteps_per_s"
+UNIT = "sample-timesteps/s"
+STRATEGY_NAME = {0: "standard", 1: "chunk", 2: "remote", 3: "double"}
+ORACLE_SAMPLE_T = 100   # steps per oracle "step" in --impl reference
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.thread, self.gpu = [], None, None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "200"], stdout=subprocess.PIPE, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        self.proc.wait()
+        self.thread.join(timeout=1)
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_spec(w):
+    from oracle.oracle import NetSpec, leak_from_tau
+    return NetSpec(w.sizes, leak_from_tau(w.tau_mem), w.theta, w.beta, w.scale(), cell=w.cell)
+
+
+def time_oracle(w, d, T_sample):
+    """One oracle train step on the first T_sample steps; returns seconds."""
+    from oracle.oracle import Oracle
+    orc = Oracle("f32")
+    spec = oracle_spec(w.with_T(T_sample))
+    t0 = time.perf_counter()
+    orc.bptt_full(spec, d["input_dense"][:T_sample], d["targets"], d["W_ff"], d["W_rec"], d["W_out"],
+                  keep_states=False)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from oracle.oracle import num_threads
+    w = wl.WORKLOADS[args.workload]
+    Ts = min(ORACLE_SAMPLE_T, w.T)
+    d = wl.make(w.with_T(Ts))
+    for _ in range(args.warmup):
+        time_oracle(w, d, Ts)
+    times = [time_oracle(w, d, Ts) for _ in range(args.steps)]
+    total = sum(times)
+    value = w.B * Ts * args.steps / total
+    sample = f"each step = oracle full-storage BPTT on the first {Ts} of {w.T} steps of {w.name}, full width and batch"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "sizes": list(w.sizes), "T": w.T, "B": w.B, "sample_T": Ts},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def algorithmic_bytes(w, activity, B):
+    """Bytes the method must move per launch of each step kernel (one wavefront launch = one step of
+    every layer), from the per-layer figures: forward gathers the active weight rows and writes V and
+    events; backward streams W_rec and the next layer's W_ff once per step and touches V and delta."""
+    sz = w.sizes
+    fwd = bwd = 0.0
+    for l in range(1, w.L + 1):
+        n_pre, n = sz[l - 1], sz[l]
+        ev = activity[l - 1] * n_pre + activity[l] * n          # events per sample feeding layer l
+        fwd += 4.0 * n * B * ev + 4.0 * ev * B + 8.0 * B * n + B * n / 8.0
+        bwd += 4.0 * n * n + (4.0 * n * sz[l + 1] if l < w.L else 0.0) + 16.0 * B * n
+    return fwd, bwd
+
+
+def run_ours(args, rank, world):
+    import torch
+    from paper_2412_11810_b200 import Session, binding as sb
+
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = wl.WORKLOADS[args.workload]
+    d = wl.make(w, dense_input=(rank == 0 and not args.no_cpu_baseline))
+    s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate_beta=w.beta, cell=w.cell,
+                readout_scale=w.scale(), device=f"cuda:{local_rank}")
+    s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    bits_host = torch.from_numpy(d["input_bits"].view(np.int32)).pin_memory()
+    tg_host = torch.from_numpy(d["targets"]).pin_memory()
+    bits, targets = bits_host.to(s.device), tg_host.to(s.device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=s.device)   # larger than the 126 MB L2
+    kw = dict(strategy=w.strategy, chunk_size=w.chunk_size, remote_chunk_size=w.remote_chunk_size,
+              max_activity=args.max_activity)
+
+    def timed_steps(n, inp, tg, **extra):
+        """n steps, each bracketed by CUDA events on the library's main stream; L2 flushed between."""
+        ms, phases = [], []
+        for _ in range(n):
+            flush.fill_(1)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(s.main):
+                e0.record()
+                s.train_step(inp, tg, **kw, **extra)
+                e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+            if extra.get("time_phases"):
+                phases.append(s.phase_times())
+        return ms, phases
+
+    timed_steps(args.warmup, bits, targets)
+    barrier()
+    clocks = ClockSampler(local_rank)
+    if rank == 0:
+        clocks.start()
+    wall0 = time.perf_counter()
+    ms, phases = timed_steps(args.steps, bits, targets, time_phases=True)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clk = clocks.stop() if rank == 0 else None
+    stats = s.stats()
+    dev_peak, pin_peak = s.peak_memory()
+    total_ms = float(sum(ms))
+    # end to end: inputs start in pinned host memory, the loss comes back to the host
+    timed_steps(1, bits_host, tg_host)
+    e2e_ms, _ = timed_steps(max(3, args.steps // 4), bits_host, tg_host)
+    e2e_total = float(sum(e2e_ms)) / len(e2e_ms) * args.steps
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_total], device=s.device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total = float(t[0]), float(t[1])
+    units = w.B * w.T * args.steps * world
+    value = units / (total_ms / 1e3)
+    e2e_value = units / (e2e_total / 1e3)
+
+    out = None
+    if rank == 0:
+        # measured activity per layer (input, hidden 1..L) from the stored event lists
+        activity = []
+        for layer in range(w.L + 1):
+            off, _ = s.events(layer)
+            activity.append(float(off[w.T + 1].astype(np.int64).sum()) / (w.T * w.B * w.sizes[layer]))
+        fwd_b, bwd_b = algorithmic_bytes(w, activity, w.B)
+        ph = {k: (sum(p[k][0] for p in phases) / len(phases), phases[0][k][1]) for k in phases[0]}
+        peak, peak_kind = read_peaks()
+        dominant = max(("fwd", "refwd1", "refwd2", "bwd", "dw"), key=lambda k: ph[k][0])
+        per_launch_bytes = {"fwd": fwd_b, "refwd1": fwd_b, "refwd2": fwd_b, "bwd": bwd_b}.get(dominant)
+        roof = None
+        if per_launch_bytes and ph[dominant][1] > 0:
+            avg_s = ph[dominant][0] / 1e3 / ph[dominant][1]
+            ach = per_launch_bytes / avg_s / 1e9
+            roof = {"bound": "hbm", "kernel": {"fwd": "fwd_step_kernel<true>", "refwd1": "fwd_step_kernel<false>",
+                                               "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel"}[dominant],
+                    "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak,
+                    "traffic": None, "algorithmic_bytes_per_launch": per_launch_bytes,
+                    "avg_launch_us": avg_s * 1e6, "launches_per_step": ph[dominant][1]}
+        # the other strategies on the same workload (fewer steps), for the per-strategy table
+        per_strategy = {}
+        T = w.T
+        K0 = w.chunk_size if w.strategy in (1, 2) else max(1, int(round(T ** 0.5)))
+        Kd, Rd = (w.chunk_size, w.remote_chunk_size) if w.strategy == 3 else (16, 256)
+        alt = {0: (0, 0), 1: (K0, 0), 2: (K0, 0), 3: (Kd, Rd)}
+        for strat, (K, R) in alt.items():
+            kws = dict(strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=args.max_activity)
+            s.train_step(bits, targets, **kws)
+            tms = []
+            for _ in range(3):
+                flush.fill_(1); torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                with torch.cuda.stream(s.main):
+                    e0.record(); s.train_step(bits, targets, **kws); e1.record()
+                torch.cuda.synchronize()
+                tms.append(e0.elapsed_time(e1))
+            st = s.stats()
+            dp, pp = s.peak_memory()
+            per_strategy[STRATEGY_NAME[strat]] = {
+                "chunk_size": K, "remote_chunk_size": R, "value": w.B * T / (float(np.median(tms)) / 1e3),
+                "ms_per_step": float(np.median(tms)), "device_peak_bytes": dp, "pinned_peak_bytes": pp,
+                "local_state_slots": st.local_state_slots, "state_bytes": st.state_bytes,
+                "kernel_launches": st.kernel_launches}
+        cpu = None
+        if not args.no_cpu_baseline:
+            from oracle.oracle import num_threads
+            sec = time_oracle(w, d, w.T)
+            cpu = {"value": w.B * w.T / sec, "unit": UNIT, "cores": num_threads(), "kind": "oracle",
+                   "sample": f"one oracle train step on the whole workload ({w.T} steps), {sec:.1f} s"}
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "sizes": list(w.sizes), "T": w.T, "B": w.B,
+                       "strategy": STRATEGY_NAME[w.strategy], "chunk_size": w.chunk_size,
+                       "remote_chunk_size": w.remote_chunk_size, "l2": "flushed between timed steps",
+                       "parallelism": "replicas only" if world > 1 else "single gpu",
+                       "measured_activity": activity},
+            "clocks": clk,
+            "e2e": {"value": e2e_value, "unit": UNIT,
+                    "h2d_bytes_per_step": int(bits_host.numel() * 4 + tg_host.numel() * 4), "d2h_bytes_per_step": 8},
+            "gpu_launches": int(stats.kernel_launches) * args.steps,
+            "roofline": roof,
+            "phases_ms": {k: v[0] for k, v in ph.items()}, "phase_launches": {k: v[1] for k, v in ph.items()},
+            "peak_memory": {"device_bytes": dev_peak, "pinned_bytes": pin_peak,
+                            "local_state_slots": stats.local_state_slots, "state_bytes": stats.state_bytes,
+                            "event_bytes": stats.event_bytes},
+            "strategies": per_strategy,
+            "cpu_baseline": cpu,
+            "wall_s_timed_region": wall,
+        }
+    s.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--max-activity", type=float, default=0.25)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,213 @@
+/*
+ * snn.h — C ABI of the BPTT training step for sparse recurrent / spiking networks
+ * under the gradient-checkpointing strategies of "Optimal Gradient Checkpointing
+ * for Sparse and Recurrent Architectures using Off-Chip Memory" (arXiv 2412.11810).
+ *
+ * Strategy names follow the caption of the paper's Fig. 1:
+ *   STANDARD  every membrane state of every step kept ("Base Implementation", Eq. 2)
+ *   CHUNK     local checkpoints every chunk_size steps, one recomputation pass
+ *             (section "Standard Checkpointing", Eqs. 1, 4, 5)
+ *   REMOTE    the same schedule with the checkpoints in remote memory (Eqs. 6, 7)
+ *   DOUBLE    remote checkpoints every remote_chunk_size steps, local ones every
+ *             chunk_size steps recomputed by an extra pass (Eqs. 11-13)
+ * "Local" memory is device memory, "remote" memory is pinned host memory.
+ *
+ * General rules.  Every function returns an snn_status and never throws, aborts
+ * or exits.  The library allocates no device or pinned memory: the caller passes
+ * two workspaces sized by snn_workspace_query and the library carves them up.
+ * Pointers marked "device" must be device pointers on the current CUDA device;
+ * pointers marked "host" are ordinary host pointers; "pinned" means page-locked
+ * host memory.  All floating-point data is fp32, all matrices row-major with the
+ * presynaptic neuron as the row: W_ff^l [N_{l-1}][N_l], W_rec^l [N_l][N_l],
+ * W_out [N_L][N_out].
+ */
+#ifndef SNN_H_
+#define SNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct snn_net snn_net; /* opaque; host-side descriptors only */
+
+typedef enum {
+  SNN_OK = 0,
+  SNN_ERR_INVALID_ARG = 1,
+  SNN_ERR_WORKSPACE_TOO_SMALL = 2,
+  SNN_ERR_EVENT_OVERFLOW = 3, /* more events than max_activity allows; gradients unspecified */
+  SNN_ERR_DEVICE_TIMEOUT = 4,
+  SNN_ERR_CUDA = 5,
+  SNN_ERR_UNSUPPORTED = 6
+} snn_status;
+
+typedef enum { SNN_STANDARD = 0, SNN_CHUNK = 1, SNN_REMOTE = 2, SNN_DOUBLE = 3 } snn_strategy;
+typedef enum { SNN_CELL_LIF = 0, SNN_CELL_GRADED = 1 } snn_cell;
+typedef enum { SNN_SURR_FAST_SIGMOID = 0, SNN_SURR_SIGMOID = 1 } snn_surrogate;
+
+#define SNN_MAX_LAYERS 8      /* hidden layers                                   */
+#define SNN_MAX_NEURONS 65536 /* per layer; hidden sizes must be multiples of 4  */
+
+/* Network description.  The paper trains "by BPTT using the surrogate gradient
+ * approach" (Methods, "BPTT based SNN training") and prints no neuron equations;
+ * this library fixes them as
+ *   I      = S^{l-1}_t W_ff^l + S^l_{t-1} W_rec^l      (one accumulator per neuron,
+ *            feed-forward events first, then recurrent, ascending presynaptic index)
+ *   V^l_t  = fma(alpha, V^l_{t-1}, I) - theta S^l_{t-1}    LIF, alpha = exp(-1/tau_mem)
+ *   S^l_t  = [V^l_t > theta]
+ *   graded cell: no reset, S^l_t = V^l_t [V^l_t > theta]
+ *   loss   = mean soft-max cross-entropy of readout_scale * (sum_t S^L_t) W_out
+ *   backward: delta_t = g_S sigma'(V_t - theta) + alpha delta_{t+1} with
+ *             sigma'(x) = 1/(1+beta|x|)^2 (fast sigmoid) or beta s(beta x)(1-s(beta x)). */
+typedef struct {
+  int32_t n_sizes;      /* L + 2                                               */
+  const int32_t* sizes; /* host: N_0, N_1 .. N_L, N_out (copied)               */
+  float tau_mem;        /* membrane time constant in steps, > 0                */
+  float threshold;      /* theta                                               */
+  int32_t surrogate;    /* snn_surrogate                                       */
+  float surrogate_beta; /* beta > 0                                            */
+  int32_t cell;         /* snn_cell                                            */
+  float readout_scale;  /* multiplies the time-summed readout                  */
+} snn_config;
+
+/* Validates the description and creates the host-side object.  No device work.
+ * Errors: SNN_ERR_INVALID_ARG (null, sizes < 1, tau/beta <= 0),
+ * SNN_ERR_UNSUPPORTED (more than SNN_MAX_LAYERS hidden layers, a hidden size that
+ * is not a multiple of 4 or exceeds SNN_MAX_NEURONS). */
+snn_status snn_create(const snn_config* cfg, snn_net** out);
+void snn_destroy(snn_net* net);
+
+/* The leak alpha = exp(-1/tau_mem), evaluated in double and rounded once to fp32. */
+float snn_alpha(const snn_net* net);
+
+/* Checkpoint hyper-parameters (paper: chunk_size, Eq. 1; remote_chunk_size, Eq. 11).
+ * STANDARD ignores both; CHUNK and REMOTE need chunk_size >= 1; DOUBLE needs
+ * remote_chunk_size >= chunk_size >= 1 and remote_chunk_size % chunk_size == 0.
+ * The sequence length need not be a multiple of either: the last segment is short. */
+typedef struct {
+  int32_t strategy; /* snn_strategy */
+  int32_t chunk_size;
+  int32_t remote_chunk_size;
+} snn_ckpt;
+
+/* Bytes of device and pinned-host workspace a train step of T steps and batch B needs.
+ * max_activity in (0, 1]: upper bound on the mean fraction of active neurons per layer
+ * over the sequence; it sizes the per-sample event pools (the sparse activations of the
+ * whole sequence stay in device memory, as in the paper's Discussion). */
+snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
+                               float max_activity, size_t* device_bytes, size_t* pinned_bytes);
+
+#define SNN_INPUT_BITS 0  /* uint32 [T][B][ceil(N_0/32)], bit i%32 of word i/32 = spike of input i */
+#define SNN_INPUT_DENSE 1 /* fp32 [T][B][N_0], zero = no event (graded cell)                        */
+
+#define SNN_FLAG_INPUT_ON_HOST 1u /* input and targets are pinned host pointers; copied in the call */
+#define SNN_FLAG_FORWARD_ONLY 2u  /* forward pass, readout and loss only                            */
+#define SNN_FLAG_TIME_PHASES 4u   /* bracket every pass with CUDA events (see snn_phase_times_get)  */
+
+typedef struct {
+  int32_t T, B;
+  const void* input;      /* device (or pinned host with SNN_FLAG_INPUT_ON_HOST), read-only       */
+  int32_t input_format;   /* SNN_INPUT_BITS | SNN_INPUT_DENSE                                      */
+  const int32_t* targets; /* [B], same memory space as input                                      */
+  const float* const* W_ff;  /* host array of L device pointers                                   */
+  const float* const* W_rec; /* host array of L device pointers                                   */
+  const float* W_out;        /* device                                                            */
+  float* const* dW_ff;       /* host array of L device pointers; OVERWRITTEN with the gradient    */
+  float* const* dW_rec;      /* of the mean loss                                                  */
+  float* dW_out;
+  void* device_ws;  size_t device_ws_bytes; /* device, 256-byte aligned                           */
+  void* pinned_ws;  size_t pinned_ws_bytes; /* pinned host; may be NULL for STANDARD and CHUNK    */
+  void* main_stream; /* cudaStream_t for the kernels                                              */
+  void* side_stream; /* cudaStream_t for checkpoint copies; must differ from main_stream for
+                        REMOTE and DOUBLE if copies are to overlap recomputation                  */
+  snn_ckpt ckpt;
+  float max_activity;
+  uint32_t flags;
+  float* const* debug_V; /* optional host array of L device pointers [T+1][B][N_l]: the forward
+                            pass also stores every membrane state there (index 0 untouched)       */
+} snn_step_args;
+
+/* One BPTT training step (paper, Fig. 1: forward, recomputation passes, backward) for the
+ * given strategy.  Returns the loss through loss_host_out (host) and the gradients in the
+ * dW buffers; synchronous: all work on both streams has finished on return.  Gradients of
+ * every checkpointing strategy are bit-identical to those of SNN_STANDARD.
+ * Errors: SNN_ERR_INVALID_ARG (nulls, T < 1, B < 1, bad intervals, misaligned workspace),
+ * SNN_ERR_WORKSPACE_TOO_SMALL, SNN_ERR_UNSUPPORTED (input format / cell mismatch) — all
+ * before any kernel is launched; SNN_ERR_EVENT_OVERFLOW, SNN_ERR_CUDA after. */
+snn_status snn_train_step(snn_net* net, const snn_step_args* args, float* loss_host_out);
+
+/* High-water marks of the last train step: bytes of the device workspace and of the pinned
+ * workspace actually used, and the part of the former that scales with the paper's M_s
+ * (number of dense states held locally times bytes per state; Eqs. 2, 4, 6, 11). */
+snn_status snn_peak_memory(const snn_net* net, size_t* device_peak_bytes, size_t* pinned_peak_bytes);
+typedef struct {
+  size_t state_bytes;         /* M_s = 4 B sum_l N_l                              */
+  int32_t local_state_slots;  /* dense states held in device memory               */
+  int32_t remote_state_slots; /* dense states held in pinned memory               */
+  int32_t d2h_copies, h2d_copies; /* checkpoint transfers of the last step        */
+  int32_t kernel_launches;    /* kernels launched by the last step                */
+  size_t event_bytes;         /* event pools + spike masks (scale with T)         */
+} snn_memory_stats;
+snn_status snn_memory_stats_get(const snn_net* net, snn_memory_stats* out);
+
+/* Device time of the last step per pass of Fig. 1, measured with CUDA events on the main stream
+ * when the step ran with SNN_FLAG_TIME_PHASES, and the kernels launched in each.  BWD is the
+ * surrogate-gradient step kernel, DW the sparse outer-product weight-gradient kernel. */
+typedef enum { SNN_PHASE_FWD = 0, SNN_PHASE_REFWD1 = 1, SNN_PHASE_REFWD2 = 2, SNN_PHASE_BWD = 3,
+               SNN_PHASE_DW = 4, SNN_PHASE_READOUT = 5, SNN_N_PHASES = 6 } snn_phase;
+typedef struct {
+  float ms[SNN_N_PHASES];
+  int32_t launches[SNN_N_PHASES];
+} snn_phase_times;
+snn_status snn_phase_times_get(const snn_net* net, snn_phase_times* out);
+
+const char* snn_last_error(const snn_net* net); /* owned by net; valid until the next call */
+
+/* ---- schedule (host only) --------------------------------------------------------------
+ * The execution trace of Fig. 1 as a list of segment operations over numbered state slots.
+ * FWD / REFWD1 / REFWD2 compute V_{t0+1} .. V_{t1} from V_{t0} held in in_slot; V_t is
+ * written to local slot buf_slot + (t-t0-1) % buf_len and, if keep_every > 0 and
+ * (t-t0) % keep_every == 0, also to local slot keep_slot + (t-t0)/keep_every - 1.
+ * FWD generates and stores the events; REFWD* replays the stored events.
+ * BWD back-propagates t = t1 .. t0+1 with V_t in local slot buf_slot + (t-t0-1).
+ * D2H copies local slot in_slot to remote slot remote_slot; H2D the reverse into keep_slot.
+ * ZERO clears local slot keep_slot (the initial state). */
+typedef enum { SNN_OP_FWD = 0, SNN_OP_REFWD1 = 1, SNN_OP_REFWD2 = 2, SNN_OP_BWD = 3,
+               SNN_OP_D2H = 4, SNN_OP_H2D = 5, SNN_OP_ZERO = 6 } snn_op_kind;
+typedef struct {
+  int32_t kind, t0, t1;
+  int32_t in_slot, buf_slot, buf_len;
+  int32_t keep_every, keep_slot, remote_slot;
+} snn_op;
+/* Writes up to max_ops operations to ops (may be NULL to query) and the totals.
+ * Pure host function: usable without a GPU. */
+snn_status snn_plan(int32_t T, const snn_ckpt* ckpt, snn_op* ops, int32_t max_ops, int32_t* n_ops,
+                    int32_t* n_local_slots, int32_t* n_remote_slots);
+
+/* ---- spike compaction on its own ("Spike Generation": dense state -> sparse events) -----
+ * For each of n_rows rows of n_words uint32 spike words (device), writes the ascending list
+ * of set-bit indices to idx_out[row * capacity ..] (device) and its length to count_out[row]
+ * (device).  Entries beyond capacity are dropped but still counted. */
+snn_status snn_compact_spikes(const uint32_t* masks, int32_t n_rows, int32_t n_words, uint32_t* idx_out,
+                              int32_t capacity, uint32_t* count_out, void* stream);
+
+/* ---- where the last step left its events (for inspection) -------------------------------
+ * layer 0 = input, 1..L = hidden.  List (layer, t, b), t = 1..T, is
+ * pool[b * pool_capacity + offsets[t * B + b] .. offsets[(t+1) * B + b]).  Offsets are byte
+ * offsets into device_ws. */
+typedef struct {
+  size_t offsets_off;  /* uint32 [(T+2)][B]                                   */
+  size_t pool_off;     /* uint32 [B][pool_capacity] neuron indices            */
+  size_t values_off;   /* fp32  [B][pool_capacity] (graded cell), else 0      */
+  size_t pool_capacity;
+  size_t mask_off;     /* uint32 [(T+1)][B][mask_words] (hidden layers), else 0 */
+  int32_t mask_words;
+} snn_event_layout;
+snn_status snn_get_event_layout(const snn_net* net, int32_t layer, snn_event_layout* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNN_H_ */

@@ -1,0 +1,576 @@
+// C ABI and executor: validates arguments, carves the caller's workspaces, and runs the
+// schedule of Fig. 1 (forward, recomputation passes, backward, checkpoint copies) as kernel
+// launches on the main stream and copies on the side stream.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/snn.h"
+#include "kernels.cuh"
+
+using namespace snnk;
+
+struct snn_net {
+  std::vector<int32_t> sizes;  // N_0, N_1..N_L, N_out
+  int L = 0;
+  float tau = 0, theta = 0, beta = 0, scale = 0, alpha = 0;
+  int surrogate = 0, cell = 0;
+  std::string err;
+  size_t dev_peak = 0, pin_peak = 0;
+  snn_memory_stats stats{};
+  // layout of the last step, for inspection
+  std::vector<snn_event_layout> ev_layout;
+  cudaEvent_t ev_main = nullptr, ev_slot[2] = {nullptr, nullptr};
+  std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
+  snn_phase_times phases{};
+};
+
+namespace {
+
+snn_status fail(snn_net* net, snn_status st, const char* fmt, ...) {
+  if (net) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    net->err = buf;
+  }
+  return st;
+}
+
+constexpr size_t ALIGN = 256;
+size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct Layout {
+  size_t status, logits, dlogits, g_out, counts, carry[2], in_stage, tg_stage;
+  size_t off[MAXL + 1], pool[MAXL + 1], mask[MAXL + 1];
+  uint32_t cap[MAXL + 1];
+  int words[MAXL + 1];
+  size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
+  size_t event_bytes, total;
+  int n_local, n_remote;
+};
+
+bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float max_activity, Layout& lo,
+                    std::string& why) {
+  const int L = net->L;
+  const auto& sz = net->sizes;
+  int n_ops = 0;
+  if (snn_plan(T, ck, nullptr, 0, &n_ops, &lo.n_local, &lo.n_remote) != SNN_OK) {
+    why = "invalid checkpoint intervals";
+    return false;
+  }
+  size_t cur = 0;
+  auto take = [&](size_t bytes) { size_t o = cur; cur = align_up(cur + bytes); return o; };
+  const int N_L = sz[L], N_out = sz[L + 1];
+  size_t sumN = 0;
+  for (int l = 1; l <= L; ++l) { lo.layer_off[l] = (size_t)B * sumN; sumN += sz[l]; }
+  lo.state_bytes = 4 * (size_t)B * sumN;
+  lo.status = take(256);
+  lo.logits = take(4 * (size_t)B * N_out);
+  lo.dlogits = take(4 * (size_t)B * N_out);
+  lo.g_out = take(4 * (size_t)B * N_L);
+  lo.counts = take(4 * (size_t)B * N_L);
+  lo.carry[0] = take(lo.state_bytes);
+  lo.carry[1] = take(lo.state_bytes);
+  lo.words[0] = (sz[0] + 31) / 32;
+  lo.in_stage = take(4 * (size_t)T * B * lo.words[0]);
+  lo.tg_stage = take(4 * (size_t)B);
+  const size_t ev0 = cur;
+  for (int l = 0; l <= L; ++l) {
+    lo.words[l] = (sz[l] + 31) / 32;
+    const double want = std::ceil((double)max_activity * sz[l] * T) + sz[l];
+    if (want > 4.0e9) { why = "event pool per sample exceeds 32-bit offsets"; return false; }
+    lo.cap[l] = (uint32_t)want;
+    lo.off[l] = take(4 * (size_t)(T + 2) * B);
+    lo.pool[l] = take(4 * (size_t)B * lo.cap[l]);
+    lo.mask[l] = l == 0 ? 0 : take(4 * (size_t)(T + 1) * B * lo.words[l]);
+  }
+  lo.event_bytes = cur - ev0;
+  lo.slots = take((size_t)lo.n_local * lo.state_bytes);
+  lo.total = cur;
+  return true;
+}
+
+#define CUDA_TRY(expr)                                                                         \
+  do {                                                                                         \
+    cudaError_t e_ = (expr);                                                                   \
+    if (e_ != cudaSuccess)                                                                     \
+      return fail(net, SNN_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_));          \
+  } while (0)
+
+}  // namespace
+
+extern "C" snn_status snn_create(const snn_config* cfg, snn_net** out) {
+  if (!cfg || !out || !cfg->sizes || cfg->n_sizes < 3) return SNN_ERR_INVALID_ARG;
+  const int L = cfg->n_sizes - 2;
+  if (L > SNN_MAX_LAYERS) return SNN_ERR_UNSUPPORTED;
+  for (int i = 0; i < cfg->n_sizes; ++i)
+    if (cfg->sizes[i] < 1) return SNN_ERR_INVALID_ARG;
+  for (int l = 1; l <= L; ++l)
+    if (cfg->sizes[l] % 4 != 0 || cfg->sizes[l] > SNN_MAX_NEURONS) return SNN_ERR_UNSUPPORTED;
+  if (cfg->sizes[0] > SNN_MAX_NEURONS) return SNN_ERR_UNSUPPORTED;
+  if (!(cfg->tau_mem > 0) || !(cfg->surrogate_beta > 0)) return SNN_ERR_INVALID_ARG;
+  if (cfg->surrogate != SNN_SURR_FAST_SIGMOID && cfg->surrogate != SNN_SURR_SIGMOID) return SNN_ERR_INVALID_ARG;
+  if (cfg->cell != SNN_CELL_LIF && cfg->cell != SNN_CELL_GRADED) return SNN_ERR_INVALID_ARG;
+  snn_net* n = new snn_net();
+  n->sizes.assign(cfg->sizes, cfg->sizes + cfg->n_sizes);
+  n->L = L;
+  n->tau = cfg->tau_mem; n->theta = cfg->threshold; n->beta = cfg->surrogate_beta;
+  n->scale = cfg->readout_scale; n->surrogate = cfg->surrogate; n->cell = cfg->cell;
+  n->alpha = (float)std::exp(-1.0 / (double)cfg->tau_mem);
+  *out = n;
+  return SNN_OK;
+}
+
+extern "C" void snn_destroy(snn_net* net) {
+  if (!net) return;
+  if (net->ev_main) cudaEventDestroy(net->ev_main);
+  for (auto& e : net->ev_slot)
+    if (e) cudaEventDestroy(e);
+  for (auto& e : net->timing_events) cudaEventDestroy(e);
+  delete net;
+}
+
+extern "C" float snn_alpha(const snn_net* net) { return net ? net->alpha : 0.f; }
+
+extern "C" const char* snn_last_error(const snn_net* net) { return net ? net->err.c_str() : "null net"; }
+
+extern "C" snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
+                                          float max_activity, size_t* device_bytes, size_t* pinned_bytes) {
+  if (!net || !ckpt || T < 1 || B < 1 || !(max_activity > 0.f) || max_activity > 1.f) return SNN_ERR_INVALID_ARG;
+  Layout lo;
+  std::string why;
+  if (!compute_layout(net, T, B, ckpt, max_activity, lo, why))
+    return fail(const_cast<snn_net*>(net), SNN_ERR_INVALID_ARG, "%s", why.c_str());
+  if (device_bytes) *device_bytes = lo.total;
+  if (pinned_bytes) *pinned_bytes = (size_t)lo.n_remote * lo.state_bytes;
+  return SNN_OK;
+}
+
+extern "C" snn_status snn_peak_memory(const snn_net* net, size_t* device_peak_bytes, size_t* pinned_peak_bytes) {
+  if (!net) return SNN_ERR_INVALID_ARG;
+  if (device_peak_bytes) *device_peak_bytes = net->dev_peak;
+  if (pinned_peak_bytes) *pinned_peak_bytes = net->pin_peak;
+  return SNN_OK;
+}
+
+extern "C" snn_status snn_memory_stats_get(const snn_net* net, snn_memory_stats* out) {
+  if (!net || !out) return SNN_ERR_INVALID_ARG;
+  *out = net->stats;
+  return SNN_OK;
+}
+
+extern "C" snn_status snn_phase_times_get(const snn_net* net, snn_phase_times* out) {
+  if (!net || !out) return SNN_ERR_INVALID_ARG;
+  *out = net->phases;
+  return SNN_OK;
+}
+
+extern "C" snn_status snn_get_event_layout(const snn_net* net, int32_t layer, snn_event_layout* out) {
+  if (!net || !out || layer < 0 || layer >= (int)net->ev_layout.size()) return SNN_ERR_INVALID_ARG;
+  *out = net->ev_layout[layer];
+  return SNN_OK;
+}
+
+extern "C" snn_status snn_compact_spikes(const uint32_t* masks, int32_t n_rows, int32_t n_words, uint32_t* idx_out,
+                                         int32_t capacity, uint32_t* count_out, void* stream) {
+  if (n_rows < 0 || n_words < 0 || capacity < 0) return SNN_ERR_INVALID_ARG;
+  if (n_words > MAX_WORDS) return SNN_ERR_UNSUPPORTED;
+  if (n_rows == 0) return SNN_OK;
+  if (!masks && n_words > 0) return SNN_ERR_INVALID_ARG;
+  if (!count_out || (!idx_out && capacity > 0)) return SNN_ERR_INVALID_ARG;
+  compact_rows_kernel<<<n_rows, FWD_THREADS, 0, (cudaStream_t)stream>>>(masks, n_words, idx_out, capacity, count_out);
+  return cudaGetLastError() == cudaSuccess ? SNN_OK : SNN_ERR_CUDA;
+}
+
+namespace {
+
+struct Exec {
+  snn_net* net;
+  const snn_step_args* a;
+  Layout lo;
+  char* ws;
+  cudaStream_t main, side;
+  int L, B, T;
+  int launches = 0, d2h = 0, h2d = 0;
+  int carry_cur = 0;
+  bool slot_pending[2] = {false, false};
+  bool remote_tier;
+  bool timed = false;
+  struct Span { int phase, ev0, ev1, launches; };
+  std::vector<Span> spans;
+  int ev_used = 0;
+
+  // Brackets [begin_span, end_span) on the main stream with two events of the net's pool.
+  int begin_span(int phase) {
+    if (!timed) return -1;
+    auto& pool_ev = net->timing_events;
+    while ((int)pool_ev.size() < ev_used + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { timed = false; return -1; }
+      pool_ev.push_back(e);
+    }
+    cudaEventRecord(pool_ev[ev_used], main);
+    spans.push_back(Span{phase, ev_used, ev_used + 1, launches});
+    ev_used += 2;
+    return (int)spans.size() - 1;
+  }
+  void end_span(int id) {
+    if (id < 0) return;
+    cudaEventRecord(net->timing_events[spans[id].ev1], main);
+    spans[id].launches = launches - spans[id].launches;
+  }
+  void collect_spans() {
+    net->phases = snn_phase_times{};
+    for (const Span& sp : spans) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, net->timing_events[sp.ev0], net->timing_events[sp.ev1]) == cudaSuccess)
+        net->phases.ms[sp.phase] += ms;
+      net->phases.launches[sp.phase] += sp.launches;
+    }
+  }
+
+  template <class Tp> Tp* at(size_t off) const { return reinterpret_cast<Tp*>(ws + off); }
+  float* slot(int s, int l) const { return at<float>(lo.slots + (size_t)s * lo.state_bytes) + lo.layer_off[l]; }
+  float* carry(int which, int l) const { return at<float>(lo.carry[which]) + lo.layer_off[l]; }
+  const uint32_t* in_mask(int t) const {  // spikes of the input at step t (t >= 1)
+    const uint32_t* base = (a->flags & SNN_FLAG_INPUT_ON_HOST) ? at<uint32_t>(lo.in_stage)
+                                                               : reinterpret_cast<const uint32_t*>(a->input);
+    return base + (size_t)(t - 1) * B * lo.words[0];
+  }
+  uint32_t* mask(int l, int t) const { return at<uint32_t>(lo.mask[l]) + (size_t)t * B * lo.words[l]; }
+  uint32_t* off(int l, int t) const { return at<uint32_t>(lo.off[l]) + (size_t)t * B; }
+  uint32_t* pool(int l) const { return at<uint32_t>(lo.pool[l]); }
+
+  snn_status wait_slot(int s) {
+    if (remote_tier && s >= 0 && s < 2 && slot_pending[s]) {
+      CUDA_TRY(cudaStreamWaitEvent(main, net->ev_slot[s], 0));
+      slot_pending[s] = false;
+    }
+    return SNN_OK;
+  }
+
+  void fill_fwd_layer(FwdLayer& f, int l, int t, const snn_op& op, bool gen) {
+    const auto& sz = net->sizes;
+    const int t0 = op.t0;
+    f.mode = 1;
+    f.W_ff = a->W_ff[l - 1];
+    f.W_rec = a->W_rec[l - 1];
+    f.N_pre = sz[l - 1]; f.N = sz[l]; f.W_pre = lo.words[l - 1]; f.W = lo.words[l];
+    f.V_prev = t - 1 == t0 ? slot(op.in_slot, l) : slot(op.buf_slot + (t - 1 - t0 - 1) % op.buf_len, l);
+    f.V_out = slot(op.buf_slot + (t - t0 - 1) % op.buf_len, l);
+    f.V_keep = (op.keep_every > 0 && (t - t0) % op.keep_every == 0)
+                   ? slot(op.keep_slot + (t - t0) / op.keep_every - 1, l) : nullptr;
+    f.V_dbg = (gen && a->debug_V && a->debug_V[l - 1]) ? a->debug_V[l - 1] + (size_t)t * B * sz[l] : nullptr;
+    f.ff_mask = l == 1 ? in_mask(t) : mask(l - 1, t);
+    f.rec_mask = mask(l, t - 1);
+    f.out_mask = mask(l, t);
+    f.ff_pool = pool(l - 1); f.ff_off = off(l - 1, t); f.ff_cap = lo.cap[l - 1];
+    f.rec_pool = pool(l); f.rec_off = off(l, t - 1); f.rec_cap = lo.cap[l];
+    f.counts = (gen && l == L) ? at<uint32_t>(lo.counts) : nullptr;
+    f.write_ff_list = l == 1;
+  }
+
+  dim3 fwd_grid() const {
+    int maxN = 0;
+    for (int l = 1; l <= L; ++l) maxN = std::max(maxN, net->sizes[l]);
+    return dim3((maxN + FWD_COLS - 1) / FWD_COLS, B, L);
+  }
+
+  snn_status launch_fwd(const FwdParams& p, bool gen) {
+    if (gen) fwd_step_kernel<true><<<fwd_grid(), FWD_THREADS, 0, main>>>(p);
+    else fwd_step_kernel<false><<<fwd_grid(), FWD_THREADS, 0, main>>>(p);
+    ++launches;
+    CUDA_TRY(cudaGetLastError());
+    return SNN_OK;
+  }
+
+  // FWD / REFWD1 / REFWD2: layer wavefront, layer l runs l-1 steps behind layer 1.
+  snn_status run_forward(const snn_op& op, bool gen) {
+    if (wait_slot(op.in_slot) != SNN_OK || wait_slot(op.keep_slot) != SNN_OK) return SNN_ERR_CUDA;
+    const int n = op.t1 - op.t0;
+    const int span = begin_span(op.kind == SNN_OP_FWD ? SNN_PHASE_FWD
+                                : op.kind == SNN_OP_REFWD1 ? SNN_PHASE_REFWD1 : SNN_PHASE_REFWD2);
+    FwdParams p;
+    std::memset(&p, 0, sizeof p);
+    p.B = B; p.alpha = net->alpha; p.theta = net->theta; p.status = at<uint32_t>(lo.status);
+    for (int s = 1; s <= n + L - 1; ++s) {
+      for (int l = 1; l <= L; ++l) {
+        const int t = op.t0 + s - (l - 1);
+        if (t <= op.t0 || t > op.t1) p.lay[l - 1].mode = 0;
+        else fill_fwd_layer(p.lay[l - 1], l, t, op, gen);
+      }
+      if (launch_fwd(p, gen) != SNN_OK) return SNN_ERR_CUDA;
+    }
+    end_span(span);
+    return SNN_OK;
+  }
+
+  // After the last forward step: store the event lists of the final spikes.
+  snn_status run_flush() {
+    FwdParams p;
+    std::memset(&p, 0, sizeof p);
+    p.B = B; p.alpha = net->alpha; p.theta = net->theta; p.status = at<uint32_t>(lo.status);
+    for (int l = 1; l <= L; ++l) {
+      FwdLayer& f = p.lay[l - 1];
+      f.mode = 2; f.N = net->sizes[l]; f.W = lo.words[l];
+      f.rec_mask = mask(l, T); f.rec_pool = pool(l); f.rec_off = off(l, T); f.rec_cap = lo.cap[l];
+    }
+    return launch_fwd(p, true);
+  }
+
+  snn_status run_readout() {
+    const int N_L = net->sizes[L], N_out = net->sizes[L + 1];
+    const uint32_t* counts = at<uint32_t>(lo.counts);
+    const int32_t* targets = (a->flags & SNN_FLAG_INPUT_ON_HOST) ? at<int32_t>(lo.tg_stage) : a->targets;
+    const int span = begin_span(SNN_PHASE_READOUT);
+    readout_logits_kernel<<<B, 256, 8 * N_out * sizeof(float), main>>>(counts, a->W_out, N_L, N_out, net->scale,
+                                                                       at<float>(lo.logits));
+    softmax_loss_kernel<<<1, 256, B * sizeof(float), main>>>(at<float>(lo.logits), targets, B, N_out,
+                                                             at<float>(lo.dlogits), at<float>(lo.status) + 1);
+    launches += 2;
+    if (!(a->flags & SNN_FLAG_FORWARD_ONLY)) {
+      readout_gout_kernel<<<(unsigned)(((size_t)B * N_L + 255) / 256), 256, 0, main>>>(
+          a->W_out, at<float>(lo.dlogits), B, N_L, N_out, net->scale, at<float>(lo.g_out));
+      readout_dwout_kernel<<<(unsigned)(((size_t)N_L * N_out + 255) / 256), 256, 0, main>>>(
+          counts, at<float>(lo.dlogits), B, N_L, N_out, net->scale, a->dW_out);
+      launches += 2;
+    }
+    end_span(span);
+    CUDA_TRY(cudaGetLastError());
+    return SNN_OK;
+  }
+
+  template <int U> void launch_dw(const DwArgs& d) {
+    dim3 grid((d.N + 128 * U - 1) / (128 * U), (d.N_pre + 31) / 32);
+    dw_kernel<U><<<grid, 256, 0, main>>>(d);
+    ++launches;
+  }
+  void run_dw(const DwArgs& d) {
+    if (d.N >= 4096) launch_dw<4>(d);
+    else if (d.N >= 256) launch_dw<2>(d);
+    else launch_dw<1>(d);
+  }
+
+  // BWD: layer wavefront, layer l runs L-l steps behind the last layer; then the weight
+  // gradients of the whole segment.
+  snn_status run_backward(const snn_op& op) {
+    const auto& sz = net->sizes;
+    const int n = op.t1 - op.t0;
+    BwdParams p;
+    std::memset(&p, 0, sizeof p);
+    p.B = B; p.alpha = net->alpha; p.theta = net->theta; p.beta = net->beta;
+    p.surrogate = net->surrogate; p.cell = net->cell;
+    int maxN = 0;
+    for (int l = 1; l <= L; ++l) maxN = std::max(maxN, sz[l]);
+    int span = begin_span(SNN_PHASE_BWD);
+    for (int s = 0; s <= n + L - 2; ++s) {
+      for (int l = L; l >= 1; --l) {
+        BwdLayer& f = p.lay[l - 1];
+        const int lag = L - l, t = op.t1 - (s - lag);
+        if (s < lag || t <= op.t0) { f.mode = 0; continue; }
+        f.mode = 1;
+        f.N = sz[l]; f.N_post = l < L ? sz[l + 1] : 0;
+        f.W_rec = a->W_rec[l - 1];
+        f.W_ffa = l < L ? a->W_ff[l] : nullptr;
+        f.V_delta = slot(op.buf_slot + (t - op.t0 - 1), l);
+        f.d_next = t == op.t1 ? carry(carry_cur, l) : slot(op.buf_slot + (t - op.t0), l);
+        f.d_above = l < L ? slot(op.buf_slot + (t - op.t0 - 1), l + 1) : nullptr;
+        f.g_out = l == L ? at<float>(lo.g_out) : nullptr;
+        f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
+      }
+      if (B <= 8) {
+        dim3 grid((maxN + BWD_WARPS * 4 - 1) / (BWD_WARPS * 4), 1, L);
+        bwd_step_kernel<8, 4><<<grid, BWD_WARPS * 32, 0, main>>>(p);
+      } else {
+        dim3 grid((maxN + BWD_WARPS * 2 - 1) / (BWD_WARPS * 2), 1, L);
+        bwd_step_kernel<16, 2><<<grid, BWD_WARPS * 32, 0, main>>>(p);
+      }
+      ++launches;
+    }
+    carry_cur ^= 1;
+    end_span(span);
+    span = begin_span(SNN_PHASE_DW);
+    for (int l = 1; l <= L; ++l) {
+      DwArgs d;
+      d.B = B; d.n_steps = n; d.N = sz[l];
+      d.delta0 = slot(op.buf_slot, l);
+      d.slot_stride = lo.state_bytes / 4;
+      d.dW = a->dW_ff[l - 1]; d.N_pre = sz[l - 1]; d.Wm = lo.words[l - 1];
+      d.mask_row0 = l == 1 ? in_mask(op.t0 + 1) : mask(l - 1, op.t0 + 1);
+      run_dw(d);
+      d.dW = a->dW_rec[l - 1]; d.N_pre = sz[l]; d.Wm = lo.words[l];
+      d.mask_row0 = mask(l, op.t0);
+      run_dw(d);
+    }
+    end_span(span);
+    CUDA_TRY(cudaGetLastError());
+    return SNN_OK;
+  }
+
+  snn_status run_copy(const snn_op& op) {
+    char* remote = static_cast<char*>(a->pinned_ws) + (size_t)op.remote_slot * lo.state_bytes;
+    const bool to_host = op.kind == SNN_OP_D2H;
+    const int s = to_host ? op.in_slot : op.keep_slot;
+    char* local = ws + lo.slots + (size_t)s * lo.state_bytes;
+    // the copy starts after everything issued so far on the main stream
+    CUDA_TRY(cudaEventRecord(net->ev_main, main));
+    CUDA_TRY(cudaStreamWaitEvent(side, net->ev_main, 0));
+    if (to_host) { CUDA_TRY(cudaMemcpyAsync(remote, local, lo.state_bytes, cudaMemcpyDeviceToHost, side)); ++d2h; }
+    else { CUDA_TRY(cudaMemcpyAsync(local, remote, lo.state_bytes, cudaMemcpyHostToDevice, side)); ++h2d; }
+    CUDA_TRY(cudaEventRecord(net->ev_slot[s], side));
+    slot_pending[s] = true;
+    return SNN_OK;
+  }
+};
+
+}  // namespace
+
+extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float* loss_host_out) {
+  if (!net) return SNN_ERR_INVALID_ARG;
+  if (!a || !loss_host_out) return fail(net, SNN_ERR_INVALID_ARG, "null argument");
+  const int L = net->L, T = a->T, B = a->B;
+  const bool fwd_only = (a->flags & SNN_FLAG_FORWARD_ONLY) != 0;
+  if (T < 1 || B < 1) return fail(net, SNN_ERR_INVALID_ARG, "T and B must be >= 1");
+  if (B > 65535) return fail(net, SNN_ERR_UNSUPPORTED, "batch above 65535");
+  if (!a->input || !a->targets || !a->W_ff || !a->W_rec || !a->W_out || !a->device_ws)
+    return fail(net, SNN_ERR_INVALID_ARG, "null pointer in arguments");
+  if (!fwd_only && (!a->dW_ff || !a->dW_rec || !a->dW_out))
+    return fail(net, SNN_ERR_INVALID_ARG, "null gradient pointer");
+  for (int l = 0; l < L; ++l) {
+    if (!a->W_ff[l] || !a->W_rec[l]) return fail(net, SNN_ERR_INVALID_ARG, "null weight pointer");
+    if (!fwd_only && (!a->dW_ff[l] || !a->dW_rec[l])) return fail(net, SNN_ERR_INVALID_ARG, "null gradient pointer");
+    if ((reinterpret_cast<uintptr_t>(a->W_ff[l]) | reinterpret_cast<uintptr_t>(a->W_rec[l])) % 16 != 0)
+      return fail(net, SNN_ERR_INVALID_ARG, "weights must be 16-byte aligned");
+    if (!fwd_only &&
+        (reinterpret_cast<uintptr_t>(a->dW_ff[l]) | reinterpret_cast<uintptr_t>(a->dW_rec[l])) % 16 != 0)
+      return fail(net, SNN_ERR_INVALID_ARG, "gradients must be 16-byte aligned");
+  }
+  if (net->cell != SNN_CELL_LIF) return fail(net, SNN_ERR_UNSUPPORTED, "graded cell: not available in this build");
+  if (a->input_format != SNN_INPUT_BITS) return fail(net, SNN_ERR_UNSUPPORTED, "LIF cell takes bit-packed input");
+  if (!(a->max_activity > 0.f) || a->max_activity > 1.f) return fail(net, SNN_ERR_INVALID_ARG, "max_activity not in (0, 1]");
+  if (reinterpret_cast<uintptr_t>(a->device_ws) % ALIGN != 0)
+    return fail(net, SNN_ERR_INVALID_ARG, "device workspace must be 256-byte aligned");
+
+  Exec ex;
+  ex.net = net; ex.a = a; ex.L = L; ex.B = B; ex.T = T;
+  std::string why;
+  if (!compute_layout(net, T, B, &a->ckpt, a->max_activity, ex.lo, why))
+    return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
+  const Layout& lo = ex.lo;
+  const size_t pinned_need = (size_t)lo.n_remote * lo.state_bytes;
+  if (a->device_ws_bytes < lo.total)
+    return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL, "device workspace %zu < %zu bytes", a->device_ws_bytes, lo.total);
+  if (pinned_need > 0 && (!a->pinned_ws || a->pinned_ws_bytes < pinned_need))
+    return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL, "pinned workspace %zu < %zu bytes", a->pinned_ws_bytes, pinned_need);
+  std::vector<snn_op> ops;
+  {
+    int n_ops = 0;
+    snn_plan(T, &a->ckpt, nullptr, 0, &n_ops, nullptr, nullptr);
+    ops.resize(n_ops);
+    snn_plan(T, &a->ckpt, ops.data(), n_ops, &n_ops, nullptr, nullptr);
+  }
+  ex.ws = static_cast<char*>(a->device_ws);
+  ex.main = (cudaStream_t)a->main_stream;
+  ex.side = a->side_stream ? (cudaStream_t)a->side_stream : ex.main;
+  ex.remote_tier = lo.n_remote > 0;
+  ex.timed = (a->flags & SNN_FLAG_TIME_PHASES) != 0;
+  if (!net->ev_main) {
+    CUDA_TRY(cudaEventCreateWithFlags(&net->ev_main, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[0], cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[1], cudaEventDisableTiming));
+  }
+  cudaStream_t ms = ex.main;
+  const auto& sz = net->sizes;
+
+  // ---- start-of-step state: status, counts, delta carry, list offsets, spikes at t = 0, gradients
+  CUDA_TRY(cudaMemsetAsync(ex.ws + lo.status, 0, 256, ms));
+  CUDA_TRY(cudaMemsetAsync(ex.ws + lo.counts, 0, 4 * (size_t)B * sz[L], ms));
+  CUDA_TRY(cudaMemsetAsync(ex.ws + lo.carry[0], 0, lo.state_bytes, ms));
+  CUDA_TRY(cudaMemsetAsync(ex.ws + lo.carry[1], 0, lo.state_bytes, ms));
+  for (int l = 0; l <= L; ++l) {
+    CUDA_TRY(cudaMemsetAsync(ex.ws + lo.off[l], 0, 4 * (size_t)2 * B, ms));
+    if (l > 0) CUDA_TRY(cudaMemsetAsync(ex.ws + lo.mask[l], 0, 4 * (size_t)B * lo.words[l], ms));
+  }
+  if (!fwd_only) {
+    for (int l = 1; l <= L; ++l) {
+      CUDA_TRY(cudaMemsetAsync(a->dW_ff[l - 1], 0, 4 * (size_t)sz[l - 1] * sz[l], ms));
+      CUDA_TRY(cudaMemsetAsync(a->dW_rec[l - 1], 0, 4 * (size_t)sz[l] * sz[l], ms));
+    }
+  }
+  if (a->flags & SNN_FLAG_INPUT_ON_HOST) {
+    CUDA_TRY(cudaMemcpyAsync(ex.ws + lo.in_stage, a->input, 4 * (size_t)T * B * lo.words[0], cudaMemcpyHostToDevice, ms));
+    CUDA_TRY(cudaMemcpyAsync(ex.ws + lo.tg_stage, a->targets, 4 * (size_t)B, cudaMemcpyHostToDevice, ms));
+  }
+
+  int last_fwd = -1;
+  for (int i = 0; i < (int)ops.size(); ++i)
+    if (ops[i].kind == SNN_OP_FWD) last_fwd = i;
+  snn_status st = SNN_OK;
+  for (int i = 0; i < (int)ops.size() && st == SNN_OK; ++i) {
+    const snn_op& op = ops[i];
+    switch (op.kind) {
+      case SNN_OP_ZERO:
+        st = ex.wait_slot(op.keep_slot);
+        if (st == SNN_OK)
+          CUDA_TRY(cudaMemsetAsync(ex.ws + lo.slots + (size_t)op.keep_slot * lo.state_bytes, 0, lo.state_bytes, ms));
+        break;
+      case SNN_OP_FWD:
+        st = ex.run_forward(op, true);
+        if (st == SNN_OK && i == last_fwd) {
+          st = ex.run_flush();
+          if (st == SNN_OK) st = ex.run_readout();
+        }
+        break;
+      case SNN_OP_REFWD1:
+      case SNN_OP_REFWD2:
+        st = ex.run_forward(op, false);
+        break;
+      case SNN_OP_BWD:
+        st = ex.run_backward(op);
+        break;
+      case SNN_OP_D2H:
+      case SNN_OP_H2D:
+        st = ex.run_copy(op);
+        break;
+      default:
+        st = fail(net, SNN_ERR_INVALID_ARG, "unknown op");
+    }
+    if (fwd_only && i == last_fwd) break;
+  }
+  // ---- finish: everything on both streams, then status and loss
+  cudaError_t e1 = cudaStreamSynchronize(ex.side);
+  cudaError_t e2 = cudaStreamSynchronize(ex.main);
+  if (st != SNN_OK) return st;
+  if (e1 != cudaSuccess || e2 != cudaSuccess)
+    return fail(net, SNN_ERR_CUDA, "stream synchronize failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
+  uint32_t host_status[2] = {0, 0};
+  CUDA_TRY(cudaMemcpy(host_status, ex.ws + lo.status, 8, cudaMemcpyDeviceToHost));
+  std::memcpy(loss_host_out, &host_status[1], 4);
+
+  if (a->flags & SNN_FLAG_TIME_PHASES) ex.collect_spans();
+  net->dev_peak = lo.total;
+  net->pin_peak = pinned_need;
+  net->stats.state_bytes = lo.state_bytes;
+  net->stats.local_state_slots = lo.n_local;
+  net->stats.remote_state_slots = lo.n_remote;
+  net->stats.d2h_copies = ex.d2h;
+  net->stats.h2d_copies = ex.h2d;
+  net->stats.kernel_launches = ex.launches;
+  net->stats.event_bytes = lo.event_bytes;
+  net->ev_layout.assign(L + 1, snn_event_layout{});
+  for (int l = 0; l <= L; ++l) {
+    snn_event_layout& e = net->ev_layout[l];
+    e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = 0; e.pool_capacity = lo.cap[l];
+    e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];
+  }
+  if (host_status[0] & STATUS_EVENT_OVERFLOW)
+    return fail(net, SNN_ERR_EVENT_OVERFLOW, "more events than max_activity=%g allows", (double)a->max_activity);
+  return SNN_OK;
+}

@@ -64,11 +64,11 @@ WORKLOADS: Dict[str, Workload] = {
     "c1": Workload("c1", (64, 128, 10), T=100, B=4, p_in=0.05, seed=0, strategy=STANDARD,
                    g_ff=(1.0,), g_rec=(1.0,), readout_scale=1.0),
     "c2": Workload("c2", (512, 1024, 1024, 20), T=1000, B=32, p_in=0.03, seed=1, strategy=CHUNK,
-                   chunk_size=32, g_ff=(1.0, 1.0), g_rec=(1.0, 1.0)),
+                   chunk_size=32, g_ff=(2.49, 1.34), g_rec=(1.0, 1.0)),
     "c3": Workload("c3", (512, 2048, 2048, 20), T=10000, B=16, p_in=0.02, seed=2, strategy=REMOTE,
-                   chunk_size=64, g_ff=(1.0, 1.0), g_rec=(1.0, 1.0)),
+                   chunk_size=64, g_ff=(3.08, 1.32), g_rec=(1.0, 1.0)),
     "c4": Workload("c4", (1024, 8192, 8192, 8192, 100), T=2000, B=8, p_in=0.02, seed=3, strategy=DOUBLE,
-                   chunk_size=16, remote_chunk_size=256, g_ff=(1.0, 1.0, 1.0), g_rec=(1.0, 1.0, 1.0)),
+                   chunk_size=16, remote_chunk_size=256, g_ff=(2.9, 1.36, 1.32), g_rec=(1.0, 1.0, 1.0)),
     "c5": Workload("c5", (1024, 4096, 4096, 50), T=4096, B=16, p_in=0.10, seed=4, strategy=DOUBLE,
                    chunk_size=16, remote_chunk_size=256, cell=CELL_GRADED, g_ff=(1.0, 1.0),
                    g_rec=(0.3, 0.3)),

@@ -1,0 +1,262 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Spike trains and event lists bit-exact; membranes <= 1e-5 absolute; gradients
+<= 1e-4 of the tensor's largest entry; every checkpointing strategy bit-identical to STANDARD."""
+import ctypes as C
+import math
+
+import numpy as np
+import pytest
+
+import snn_workloads as wl
+from gpu_helpers import (V_ATOL, assert_grads_close, lists_from_dense, make_session, run_oracle)
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def sb():
+    from paper_2412_11810_b200 import binding
+    return binding
+
+
+# ---------------------------------------------------------------- spike compaction on its own
+@pytest.mark.parametrize("n_rows,n", [(1, 1), (7, 31), (5, 32), (33, 100), (64, 1000), (3, 4096), (2, 65536), (0, 64)])
+def test_compaction_bit_exact(orc32, n_rows, n):
+    rng = np.random.default_rng(n + n_rows)
+    v = rng.standard_normal((max(n_rows, 1), n)).astype(np.float32)
+    if n_rows >= 3:
+        v[0] = -1.0   # empty row
+        v[1] = 2.0    # full row
+    v = v[:n_rows]
+    theta = 0.5
+    dense = (v > np.float32(theta))
+    words = wl.pack_bits(dense) if n_rows else np.zeros((0, (n + 31) // 32), np.uint32)
+    cap = n
+    dm = torch.from_numpy(words.view(np.int32).copy()).cuda()
+    idx = torch.full((max(n_rows, 1), cap), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((max(n_rows, 1),), -1, dtype=torch.int32, device="cuda")
+    sb().snn_compact_spikes(dm.data_ptr(), n_rows, words.shape[1], idx.data_ptr(), cap, cnt.data_ptr(), 0)
+    torch.cuda.synchronize()
+    idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+    for r in range(n_rows):
+        ref = orc32.compact(v[r], theta)          # brute force: for i: if v[i] > theta: push(i)
+        assert cnt[r] == len(ref)
+        assert np.array_equal(idx[r, :cnt[r]], ref)
+        assert np.all(idx[r, cnt[r]:] == -1)
+
+
+def test_compaction_capacity_clamps(orc32):
+    words = np.full((2, 4), 0xFFFFFFFF, np.uint32)
+    dm = torch.from_numpy(words.view(np.int32)).cuda()
+    idx = torch.full((2, 10), -1, dtype=torch.int32, device="cuda")
+    guard = torch.full((16,), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    sb().snn_compact_spikes(dm.data_ptr(), 2, 4, idx.data_ptr(), 10, cnt.data_ptr(), 0)
+    torch.cuda.synchronize()
+    assert np.all(cnt.cpu().numpy() == 128)
+    assert np.array_equal(idx.cpu().numpy(), np.tile(np.arange(10, dtype=np.int32), (2, 1)))
+    assert np.all(guard.cpu().numpy() == -7)
+
+
+# ---------------------------------------------------------------- forward: membranes, spikes, events
+def _check_forward(orc32, w, d):
+    ref = run_oracle(orc32, w, d, do_backward=False)
+    s, bits, targets = make_session(w, d)
+    loss = s.train_step(bits, targets, forward_only=True, keep_V=True, max_activity=1.0)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    for l in range(w.L):
+        V = s.debug_V[l].cpu().numpy()
+        assert np.abs(V[1:] - ref["V"][l][1:]).max() <= V_ATOL
+        assert np.array_equal(V[1:], ref["V"][l][1:]), "canonical operation order: expected bit-equal"
+        words = s.spike_words(l + 1)
+        assert np.array_equal(wl.unpack_bits(words, w.sizes[l + 1]), ref["S"][l].astype(np.uint8))
+    # event lists: input (layer 0) and every hidden layer, every (t, b)
+    dense = [d["input_dense"]] + [r[1:] for r in ref["S"]]
+    for layer in range(w.L + 1):
+        off, pool = s.events(layer)
+        want = lists_from_dense(dense[layer])
+        for t in range(1, w.T + 1):
+            for b in range(w.B):
+                got = pool[b, off[t, b]:off[t + 1, b]]
+                assert np.array_equal(got, want[t - 1][b]), (layer, t, b)
+    s.close()
+    return ref
+
+
+def test_forward_tiny_bit_exact(orc32):
+    w = wl.small()
+    _check_forward(orc32, w, wl.make(w))
+
+
+def test_forward_ragged_sizes_bit_exact(orc32):
+    # hidden sizes that are multiples of 4 but not of 32 or 128, input not a multiple of 32,
+    # several column tiles (N > 512) and more than 1024 events per list
+    w = wl.small(sizes=(70, 3000, 36, 7), T=9, B=2, p_in=0.5, g_ff=(3.0, 6.0), g_rec=(1.0, 1.0), seed=3)
+    ref = _check_forward(orc32, w, wl.make(w))
+    assert ref["S"][0][1:].mean() > 0.1
+
+
+def test_forward_c1_bit_exact(orc32):
+    w = wl.WORKLOADS["c1"]
+    ref = _check_forward(orc32, w, wl.make(w))
+    assert ref["S"][0].sum() > 0
+
+
+# ---------------------------------------------------------------- gradients and strategies
+STRATS = [(1, 4, 0), (1, 1, 0), (1, 13, 0), (1, 40, 0), (2, 4, 0), (2, 1, 0), (2, 5, 0), (3, 2, 6), (3, 3, 3),
+          (3, 1, 4), (3, 2, 26), (3, 13, 13)]
+
+
+def _bits(t):
+    return [x.cpu().numpy().view(np.uint32).copy() for x in t]
+
+
+def test_gradients_and_all_strategies_tiny(orc32):
+    w = wl.small()
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    s, bits, targets = make_session(w, d)
+    loss = s.train_step(bits, targets, strategy=0, max_activity=1.0)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    assert s.stats().local_state_slots == w.T + 1
+    for strat, K, R in STRATS:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        loss2 = s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0)
+        assert loss2 == loss
+        for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(a, b), f"strategy {strat} K={K} R={R} differs from STANDARD"
+        st = s.stats()
+        Kc = min(K, w.T)
+        if strat == 1:
+            assert st.local_state_slots == Kc + math.ceil(w.T / K) and st.d2h_copies == 0
+        elif strat == 2:
+            assert st.local_state_slots == Kc + 2
+            assert st.d2h_copies == st.h2d_copies == math.ceil(w.T / K)
+        else:
+            assert st.local_state_slots == Kc + math.ceil(min(R, w.T) / K) + 1
+            assert st.d2h_copies == st.h2d_copies == math.ceil(w.T / R)
+        dev, pin = s.peak_memory()
+        assert pin == st.remote_state_slots * st.state_bytes
+    s.close()
+
+
+@pytest.mark.parametrize("T", [1, 2])
+def test_degenerate_sequence_lengths(orc32, T):
+    w = wl.small(T=T)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    s, bits, targets = make_session(w, d)
+    for strat, K, R in [(0, 0, 0), (1, 1, 0), (2, 3, 0), (3, 1, 2)]:
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0)
+        assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
+def test_silent_and_saturated_networks(orc32):
+    from dataclasses import replace
+    for theta in (1e30, -1e30):
+        w = replace(wl.small(T=3), theta=theta)
+        d = wl.make(w)
+        ref = run_oracle(orc32, w, d)
+        s, bits, targets = make_session(w, d)
+        loss = s.train_step(bits, targets, strategy=1, chunk_size=2, max_activity=1.0)
+        if theta > 0:
+            assert abs(loss - math.log(w.sizes[-1])) < 1e-6
+        assert_grads_close(s.gradients(), ref)
+        s.close()
+
+
+def test_sigmoid_surrogate(orc32):
+    from oracle.oracle import SURR_SIGMOID, NetSpec, leak_from_tau
+    from paper_2412_11810_b200 import Session
+    w = wl.small()
+    d = wl.make(w)
+    spec = NetSpec(w.sizes, leak_from_tau(w.tau_mem), w.theta, 4.0, w.scale(), surrogate=SURR_SIGMOID)
+    ref = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
+    s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate=1, surrogate_beta=4.0,
+                readout_scale=w.scale())
+    s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    s.train_step(d["input_bits"], d["targets"], strategy=3, chunk_size=2, remote_chunk_size=4, max_activity=1.0)
+    assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
+def test_c1_gradients_all_strategies(orc32):
+    w = wl.WORKLOADS["c1"]
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    s, bits, targets = make_session(w, d)
+    loss = s.train_step(bits, targets, strategy=0)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 10, 0), (2, 7, 0), (3, 4, 16)]:
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R)
+        for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(a, b)
+    s.close()
+
+
+def test_medium_network_several_tiles(orc32):
+    # two layers wider than one column tile, batch above the backward kernel's batch tile,
+    # ragged segments in both tiers
+    w = wl.small(sizes=(96, 640, 1040, 12), T=37, B=19, p_in=0.05, g_ff=(2.5, 1.4), g_rec=(1.0, 1.0), seed=5)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    act = [float(s_[1:].mean()) for s_ in ref["S"]]
+    assert all(0.005 < a < 0.5 for a in act), act
+    s, bits, targets = make_session(w, d)
+    s.train_step(bits, targets, strategy=0)
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 6, 0), (2, 8, 0), (3, 3, 12)]:
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R)
+        for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(a, b)
+    s.close()
+
+
+def test_host_input_path_matches_device_input(orc32):
+    w = wl.small()
+    d = wl.make(w)
+    s, bits, targets = make_session(w, d)
+    l0 = s.train_step(bits, targets, strategy=1, chunk_size=4, max_activity=1.0)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    l1 = s.train_step(d["input_bits"], d["targets"], strategy=1, chunk_size=4, max_activity=1.0)
+    assert l0 == l1
+    for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+        assert np.array_equal(a, b)
+    s.close()
+
+
+# ---------------------------------------------------------------- errors reported, nothing faults
+def test_errors_are_reported(orc32):
+    b = sb()
+    w = wl.small()
+    d = wl.make(w)
+    s, bits, targets = make_session(w, d)
+    with pytest.raises(b.SnnError) as e:
+        s.train_step(bits, targets, strategy=3, chunk_size=4, remote_chunk_size=6)
+    assert e.value.status == b.SNN_ERR_INVALID_ARG
+    # far fewer event slots than the activity needs: reported, never written out of bounds
+    with pytest.raises(b.SnnError) as e:
+        s.train_step(bits, targets, strategy=0, max_activity=1e-4)
+    assert e.value.status == b.SNN_ERR_EVENT_OVERFLOW
+    # workspace too small: rejected before any launch
+    s.train_step(bits, targets, strategy=0, max_activity=0.5)
+    ck = s.ckpt(0)
+    need, _ = b.snn_workspace_query(s.net, w.T, w.B, ck, 0.5)
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    a = b.snn_step_args()
+    a.T, a.B, a.input, a.targets = w.T, w.B, bits.data_ptr(), targets.data_ptr()
+    wff = b.ptr_array([x.data_ptr() for x in s.W_ff]); wrec = b.ptr_array([x.data_ptr() for x in s.W_rec])
+    gff = b.ptr_array([x.data_ptr() for x in s.dW_ff]); grec = b.ptr_array([x.data_ptr() for x in s.dW_rec])
+    a.W_ff, a.W_rec, a.W_out, a.dW_ff, a.dW_rec, a.dW_out = wff, wrec, s.W_out.data_ptr(), gff, grec, s.dW_out.data_ptr()
+    a.device_ws, a.device_ws_bytes = small.data_ptr(), small.numel()
+    a.ckpt, a.max_activity = ck, 0.5
+    loss = C.c_float()
+    assert b.lib.snn_train_step(s.net, C.byref(a), C.byref(loss)) == b.SNN_ERR_WORKSPACE_TOO_SMALL
+    s.close()
