@@ -238,7 +238,7 @@ def run_ours(args, rank, world):
         K0 = w.chunk_size if w.strategy in (1, 2) else max(1, int(round(T ** 0.5)))
         Kd, Rd = (w.chunk_size, w.remote_chunk_size) if w.strategy == 3 else (16, 256)
         alt = {0: (0, 0), 1: (K0, 0), 2: (K0, 0), 3: (Kd, Rd)}
-        for strat, (K, R) in alt.items():
+        for strat, (K, R) in ([] if args.no_strategies else alt.items()):
             kws = dict(strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=args.max_activity)
             s.train_step(bits, targets, **kws)
             tms = []
@@ -301,6 +301,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--max-activity", type=float, default=0.25)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-strategies", action="store_true", help="skip the per-strategy table")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
