@@ -138,6 +138,30 @@ typedef struct {
  * before any kernel is launched; SNN_ERR_EVENT_OVERFLOW, SNN_ERR_CUDA after. */
 snn_status snn_train_step(snn_net* net, const snn_step_args* args, float* loss_host_out);
 
+/* The same training step for callers that cannot allocate device memory at all.
+ * (The paper has no counterpart: this entry point exists for embedding only.)
+ * Some hosts of this library own no allocator they may call when a step is due: a C program
+ * that links the library without PyTorch, a process whose device memory has been handed over
+ * entirely to another component's pool, or a service under a fixed memory budget where a
+ * cudaMalloc at step time could fail, or would stall every stream of the device while it runs.
+ * For them the device workspace is not passed in: the library uses a buffer of
+ * SNN_STATIC_WORKSPACE_BYTES that is part of its own device image.  Every GPU that loads the
+ * library holds those bytes until the process exits, whether this entry point is used or not.
+ *   - args->device_ws and args->device_ws_bytes are ignored; inputs, targets, weights, gradient
+ *     buffers, the pinned workspace (REMOTE / DOUBLE) and the streams are passed as usual.
+ *   - A step whose snn_workspace_query device size exceeds SNN_STATIC_WORKSPACE_BYTES is
+ *     rejected with SNN_ERR_WORKSPACE_TOO_SMALL before anything runs.
+ *   - The call allocates and frees no device or pinned memory.  The first call on a device looks
+ *     up the address of the built-in buffer (once per device, with that device current); make
+ *     that first call outside any stream capture.  Like snn_train_step it creates a few CUDA
+ *     events the first time a net is used.
+ *   - All calls on one device share the one buffer.  It keeps whatever the previous call left;
+ *     the step clears everything it needs to start from zero.  Two calls that overlap on the GPU
+ *     (different host threads, different nets, different streams) race on it: serialise them.
+ * Results are those of snn_train_step, bit for bit. */
+#define SNN_STATIC_WORKSPACE_BYTES (32u << 20)
+snn_status snn_train_step_static(snn_net* net, const snn_step_args* args, float* loss_host_out);
+
 /* High-water marks of the last train step: bytes of the device workspace and of the pinned
  * workspace actually used, and the part of the former that scales with the paper's M_s
  * (number of dense states held locally times bytes per state; Eqs. 2, 4, 6, 11). */

@@ -26,7 +26,8 @@ STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "rem
 
 EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_train_step", "snn_peak_memory",
            "snn_memory_stats_get", "snn_last_error", "snn_plan", "snn_compact_spikes", "snn_get_event_layout",
-           "snn_phase_times_get"]
+           "snn_phase_times_get", "snn_train_step_static"]
+SNN_STATIC_WORKSPACE_BYTES = 32 << 20
 
 
 class snn_config(C.Structure):
@@ -82,6 +83,7 @@ def _load() -> C.CDLL:
     lib.snn_workspace_query.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(snn_ckpt), C.c_float,
                                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.snn_train_step.argtypes = [C.c_void_p, C.POINTER(snn_step_args), C.POINTER(C.c_float)]
+    lib.snn_train_step_static.argtypes = [C.c_void_p, C.POINTER(snn_step_args), C.POINTER(C.c_float)]
     lib.snn_peak_memory.argtypes = [C.c_void_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.snn_memory_stats_get.argtypes = [C.c_void_p, C.POINTER(snn_memory_stats)]
     lib.snn_last_error.argtypes = [C.c_void_p]
@@ -136,6 +138,14 @@ def snn_workspace_query(net, T: int, B: int, ckpt: snn_ckpt, max_activity: float
 def snn_train_step(net, args: snn_step_args) -> float:
     loss = C.c_float()
     _check(lib.snn_train_step(net, C.byref(args), C.byref(loss)), net)
+    return loss.value
+
+
+def snn_train_step_static(net, args: snn_step_args) -> float:
+    """snn_train_step on the library's built-in device workspace: for hosts that cannot allocate
+    device memory themselves (args.device_ws is ignored).  See include/snn.h for the limits."""
+    loss = C.c_float()
+    _check(lib.snn_train_step_static(net, C.byref(args), C.byref(loss)), net)
     return loss.value
 
 

@@ -574,3 +574,50 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     return fail(net, SNN_ERR_EVENT_OVERFLOW, "more events than max_activity=%g allows", (double)a->max_activity);
   return SNN_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Training step on the library's own, statically reserved device workspace, for callers that
+// have no way to allocate device memory when the step is due (no PyTorch in the process, the
+// whole device already given to another pool, or a fixed budget under which cudaMalloc could
+// fail or stall the device).  The buffer lives in the device image of this library: every GPU
+// that loads it holds SNN_STATIC_WORKSPACE_BYTES until exit.
+//
+// The array's name is only a handle in host code; the device address that kernels and copies
+// need comes from cudaGetSymbolAddress, looked up once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_workspace[SNN_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_workspace_addr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" snn_status snn_train_step_static(snn_net* net, const snn_step_args* args, float* loss_host_out) {
+  if (!net) return SNN_ERR_INVALID_ARG;
+  if (!args || !loss_host_out) return fail(net, SNN_ERR_INVALID_ARG, "null argument");
+  if (args->T < 1 || args->B < 1) return fail(net, SNN_ERR_INVALID_ARG, "T and B must be >= 1");
+  if (!(args->max_activity > 0.f) || args->max_activity > 1.f)
+    return fail(net, SNN_ERR_INVALID_ARG, "max_activity not in (0, 1]");
+  // size check first: nothing runs for a step that does not fit the built-in buffer
+  Layout lo;
+  std::string why;
+  if (!compute_layout(net, args->T, args->B, &args->ckpt, args->max_activity, lo, why))
+    return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
+  if (lo.total > (size_t)SNN_STATIC_WORKSPACE_BYTES)
+    return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL,
+                "this step needs %zu bytes of device workspace; the built-in workspace holds %zu "
+                "(use snn_train_step with a caller-provided workspace)",
+                lo.total, (size_t)SNN_STATIC_WORKSPACE_BYTES);
+  int dev = -1;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(net, SNN_ERR_UNSUPPORTED, "device index %d out of range", dev);
+  if (!g_static_workspace_addr[dev]) {  // first call on this device: resolve the buffer's device address
+    void* p = nullptr;
+    CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
+    if (!p) return fail(net, SNN_ERR_CUDA, "built-in workspace has no device address");
+    g_static_workspace_addr[dev] = p;
+  }
+  snn_step_args a = *args;
+  a.device_ws = g_static_workspace_addr[dev];
+  a.device_ws_bytes = (size_t)SNN_STATIC_WORKSPACE_BYTES;
+  return snn_train_step(net, &a, loss_host_out);
+}
