@@ -7,10 +7,13 @@
 // first, then recurrent events, each list in ascending presynaptic index, one fused
 // multiply-add for the leak, one subtraction for the reset.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace snnk {
+
+namespace cg = cooperative_groups;
 
 constexpr int MAXL = 8;
 constexpr int FWD_THREADS = 128;            // each thread owns 4 adjacent neurons of one sample
@@ -21,19 +24,53 @@ constexpr uint32_t STATUS_EVENT_OVERFLOW = 1u;
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 
+// 128-bit read-only load that does not allocate in L1: weight rows are streamed once per CTA.
+__device__ __forceinline__ float4 ldg4_stream(const float* p) {
+  float4 v;
+  asm("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+      : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
+// 16-byte asynchronous copy global -> shared (bypasses L1 and the register file).  Copies are
+// grouped with cp_async_commit; cp_async_wait<N> returns when at most N groups are pending.
+// Each thread only ever reads back the bytes it copied itself, so no barrier is needed.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr uint32_t REC_TAG = 0x80000000u;  // list entry names a row of W_rec (else of W_ff)
+
+// A row of spike words made of two parts that is addressed as one: the feed-forward source
+// (layer below, this step) followed by the recurrent source (own layer, previous step).
+struct WordPair {
+  const uint32_t* a; int n_a;
+  const uint32_t* b; int n_b;
+  __device__ __forceinline__ int size() const { return n_a + n_b; }
+  __device__ __forceinline__ uint32_t get(int w) const { return w < n_a ? a[w] : b[w - n_a]; }
+  __device__ __forceinline__ uint32_t first_index(int w) const {
+    return w < n_a ? (uint32_t)w * 32u : ((uint32_t)(w - n_a) * 32u) | REC_TAG;
+  }
+};
+
 // ------------------------------------------------------------------------------------------
 // Spike compaction ("Spike Generation" in its sparse representation): spike words -> ascending
 // index list.  Step 1: exclusive prefix sum of the per-word popcounts over the whole row.
-// Returns the number of set bits; s_pref[w] = number of set bits in words [0, w).
+// s_pref[w] = number of set bits in words [0, w), for w = 0 .. size() (the last one = total).
 template <int NT>
-__device__ uint32_t prefix_popcounts(const uint32_t* __restrict__ words, int n_words, uint32_t* s_pref,
-                                     uint32_t* s_warp) {
+__device__ uint32_t prefix_popcounts(const WordPair& wp, uint32_t* s_pref, uint32_t* s_warp) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_words = wp.size();
   const int wpt = (n_words + NT - 1) / NT;
   const int w0 = tid * wpt;
   uint32_t sum = 0;
   for (int i = 0; i < wpt; ++i)
-    if (w0 + i < n_words) sum += __popc(words[w0 + i]);
+    if (w0 + i < n_words) sum += __popc(wp.get(w0 + i));
   uint32_t inc = sum;
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
@@ -52,40 +89,51 @@ __device__ uint32_t prefix_popcounts(const uint32_t* __restrict__ words, int n_w
   }
   uint32_t ex = base + inc - sum;
   for (int i = 0; i < wpt; ++i)
-    if (w0 + i < n_words) { s_pref[w0 + i] = ex; ex += __popc(words[w0 + i]); }
+    if (w0 + i < n_words) { s_pref[w0 + i] = ex; ex += __popc(wp.get(w0 + i)); }
+  if (tid == 0) s_pref[n_words] = total;
   __syncthreads();
   return total;
 }
 
 // Step 2a: the part [c0, c0 + LIST_CHUNK) of the list into shared memory.
 template <int NT>
-__device__ void fill_chunk_from_words(const uint32_t* __restrict__ words, int n_words, const uint32_t* s_pref,
-                                      uint32_t c0, uint32_t* s_list) {
+__device__ void fill_chunk_from_words(const WordPair& wp, const uint32_t* s_pref, uint32_t c0, uint32_t* s_list) {
+  const int n_words = wp.size();
   for (int w = threadIdx.x; w < n_words; w += NT) {
-    uint32_t bits = words[w];
+    uint32_t bits = wp.get(w);
     if (!bits) continue;
     uint32_t p = s_pref[w];
     if (p >= c0 + LIST_CHUNK || p + __popc(bits) <= c0) continue;
+    const uint32_t first = wp.first_index(w);
     while (bits) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
-      if (p >= c0 && p < c0 + LIST_CHUNK) s_list[p - c0] = (uint32_t)(w * 32 + bit);
+      if (p >= c0 && p < c0 + LIST_CHUNK) s_list[p - c0] = first + bit;
       ++p;
     }
   }
 }
 
-// Step 2b: the whole list to global memory (entries past the capacity are dropped).
+// Step 2b: the lists to global memory (entries past the room left in a pool are dropped).
+// Part a goes to dst_a (if not null), part b to dst_b; n_a_bits = set bits of part a.
 template <int NT>
-__device__ void write_list_from_words(const uint32_t* __restrict__ words, int n_words, const uint32_t* s_pref,
-                                      uint32_t* __restrict__ dst, uint32_t room) {
+__device__ void write_lists_from_words(const WordPair& wp, const uint32_t* s_pref, uint32_t n_a_bits,
+                                       uint32_t* __restrict__ dst_a, uint32_t room_a,
+                                       uint32_t* __restrict__ dst_b, uint32_t room_b) {
+  const int n_words = wp.size();
   for (int w = threadIdx.x; w < n_words; w += NT) {
-    uint32_t bits = words[w];
+    uint32_t bits = wp.get(w);
     uint32_t p = s_pref[w];
+    const bool in_a = w < wp.n_a;
+    uint32_t* dst = in_a ? dst_a : dst_b;
+    if (!dst) continue;
+    const uint32_t room = in_a ? room_a : room_b;
+    if (!in_a) p -= n_a_bits;
+    const uint32_t first = wp.first_index(w) & ~REC_TAG;
     while (bits) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
-      if (p < room) dst[p] = (uint32_t)(w * 32 + bit);
+      if (p < room) dst[p] = first + bit;
       ++p;
     }
   }
@@ -95,12 +143,13 @@ __device__ void write_list_from_words(const uint32_t* __restrict__ words, int n_
 __global__ void __launch_bounds__(FWD_THREADS)
 compact_rows_kernel(const uint32_t* __restrict__ masks, int n_words, uint32_t* __restrict__ idx_out,
                     int capacity, uint32_t* __restrict__ count_out) {
-  __shared__ uint32_t s_pref[MAX_WORDS];
+  __shared__ uint32_t s_pref[MAX_WORDS + 1];
   __shared__ uint32_t s_warp[FWD_THREADS / 32];
   const size_t row = blockIdx.x;
-  const uint32_t* words = masks + row * (size_t)n_words;
-  const uint32_t total = prefix_popcounts<FWD_THREADS>(words, n_words, s_pref, s_warp);
-  write_list_from_words<FWD_THREADS>(words, n_words, s_pref, idx_out + row * (size_t)capacity, (uint32_t)capacity);
+  WordPair wp{masks + row * (size_t)n_words, n_words, nullptr, 0};
+  const uint32_t total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
+  write_lists_from_words<FWD_THREADS>(wp, s_pref, total, idx_out + row * (size_t)capacity, (uint32_t)capacity,
+                                      nullptr, 0);
   if (threadIdx.x == 0) count_out[row] = total;
 }
 
@@ -134,63 +183,9 @@ struct FwdParams {
   uint32_t* status;
 };
 
-// Adds the rows of W named by one event list to the accumulator, in list order.
-// GEN: the list is compacted here from spike words; else it is read back from the pool.
-template <bool GEN>
-__device__ __forceinline__ void accumulate_list(const uint32_t* __restrict__ words, int n_words,
-                                                uint32_t* __restrict__ pool, uint32_t* __restrict__ off,
-                                                uint32_t cap, bool write_list, int B, int b,
-                                                const float* __restrict__ W, int N, int col, bool active,
-                                                float4& acc, uint32_t* s_list, uint32_t* s_pref,
-                                                uint32_t* s_warp, uint32_t* status) {
-  uint32_t total, start = 0;
-  uint32_t* my_pool = pool + (size_t)b * cap;
-  if (GEN) {
-    total = prefix_popcounts<FWD_THREADS>(words, n_words, s_pref, s_warp);
-    if (write_list) {
-      start = off[b];
-      const uint32_t room = cap - start;  // start <= cap always (clamped below)
-      write_list_from_words<FWD_THREADS>(words, n_words, s_pref, my_pool + start, room);
-      if (threadIdx.x == 0) {
-        off[B + b] = start + (total < room ? total : room);
-        if (total > room) atomicOr(status, STATUS_EVENT_OVERFLOW);
-      }
-    }
-  } else {
-    start = off[b];
-    total = off[B + b] - start;
-  }
-  if (W == nullptr) return;
-  const float* Wc = W + col;
-  for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
-    const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
-    if (GEN) {
-      fill_chunk_from_words<FWD_THREADS>(words, n_words, s_pref, c0, s_list);
-    } else {
-      for (int i = threadIdx.x; i < n; i += FWD_THREADS) s_list[i] = my_pool[start + c0 + i];
-    }
-    __syncthreads();
-    if (active) {
-      int e = 0;
-      for (; e + 8 <= n; e += 8) {
-        float4 w[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) w[u] = ldg4(Wc + (size_t)s_list[e + u] * N);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          acc.x = __fadd_rn(acc.x, w[u].x); acc.y = __fadd_rn(acc.y, w[u].y);
-          acc.z = __fadd_rn(acc.z, w[u].z); acc.w = __fadd_rn(acc.w, w[u].w);
-        }
-      }
-      for (; e < n; ++e) {
-        const float4 w = ldg4(Wc + (size_t)s_list[e] * N);
-        acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
-        acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
-      }
-    }
-    __syncthreads();
-  }
-}
+constexpr int GATHER_ROWS = 8;     // weight rows per copy group
+constexpr int GATHER_STAGES = 5;   // copy groups in flight per thread (40 rows, 80 KB per CTA)
+constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
 template <bool GEN>
 __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_constant__ FwdParams p) {
@@ -201,32 +196,109 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   const int b = blockIdx.y, B = p.B;
   const bool tile0 = blockIdx.x == 0;
   __shared__ uint32_t s_list[LIST_CHUNK];
-  __shared__ uint32_t s_pref[MAX_WORDS];
+  __shared__ uint32_t s_pref[GEN ? 2 * MAX_WORDS + 1 : 1];
   __shared__ uint32_t s_warp[FWD_THREADS / 32];
+  extern __shared__ float4 s_stage[];   // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
   const int col = col0 + threadIdx.x * 4;
   const bool active = col < L.N;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool step = L.mode == 1;
+  if (!step && !(GEN && tile0)) return;
 
-  if (L.mode == 2) {  // after the last step: only store the list of the final spikes
-    if (GEN && tile0)
-      accumulate_list<true>(L.rec_mask + (size_t)b * L.W, L.W, L.rec_pool, L.rec_off, L.rec_cap, true, B, b,
-                            nullptr, L.N, col, false, acc, s_list, s_pref, s_warp, p.status);
-    return;
+  // issue the loads the epilogue needs before anything else
+  float4 vp = make_float4(0.f, 0.f, 0.f, 0.f);
+  uint32_t pw = 0;
+  if (step && active) {
+    vp = *reinterpret_cast<const float4*>(L.V_prev + (size_t)b * L.N + col);
+    pw = L.rec_mask[(size_t)b * L.W + (col >> 5)] >> (col & 31);
   }
-  // feed-forward events: layer below, same step
-  accumulate_list<GEN>(GEN ? L.ff_mask + (size_t)b * L.W_pre : nullptr, L.W_pre, L.ff_pool, L.ff_off, L.ff_cap,
-                       tile0 && L.write_ff_list, B, b, L.W_ff, L.N, col, active, acc, s_list, s_pref, s_warp,
-                       p.status);
-  // recurrent events: own layer, previous step
-  accumulate_list<GEN>(GEN ? L.rec_mask + (size_t)b * L.W : nullptr, L.W, L.rec_pool, L.rec_off, L.rec_cap, tile0,
-                       B, b, L.W_rec, L.N, col, active, acc, s_list, s_pref, s_warp, p.status);
 
-  // leak, reset by subtraction of the previous step's own spike, threshold
+  // ---- the two event lists of this step as one: feed-forward events, then recurrent events
+  uint32_t n_ff, total, s_ff = 0, s_rec = 0;
+  uint32_t* const ff_pool = L.ff_pool + (size_t)b * L.ff_cap;
+  uint32_t* const rec_pool = L.rec_pool + (size_t)b * L.rec_cap;
+  WordPair wp{nullptr, 0, nullptr, 0};
+  if (GEN) {
+    wp = WordPair{step ? L.ff_mask + (size_t)b * L.W_pre : nullptr, step ? L.W_pre : 0,
+                  L.rec_mask + (size_t)b * L.W, L.W};
+    total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
+    n_ff = s_pref[wp.n_a];
+    if (tile0) {  // this CTA appends the lists to the event pools
+      const bool wr_ff = step && L.write_ff_list;
+      s_rec = L.rec_off[b];
+      if (wr_ff) s_ff = L.ff_off[b];
+      const uint32_t room_ff = wr_ff ? L.ff_cap - s_ff : 0, room_rec = L.rec_cap - s_rec;
+      write_lists_from_words<FWD_THREADS>(wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff,
+                                          rec_pool + s_rec, room_rec);
+      if (threadIdx.x == 0) {
+        const uint32_t n_rec = total - n_ff;
+        L.rec_off[B + b] = s_rec + (n_rec < room_rec ? n_rec : room_rec);
+        if (wr_ff) L.ff_off[B + b] = s_ff + (n_ff < room_ff ? n_ff : room_ff);
+        if (n_rec > room_rec || (wr_ff && n_ff > room_ff)) atomicOr(p.status, STATUS_EVENT_OVERFLOW);
+      }
+    }
+    if (!step) return;
+  } else {
+    s_ff = L.ff_off[b]; n_ff = L.ff_off[B + b] - s_ff;
+    s_rec = L.rec_off[b]; total = n_ff + (L.rec_off[B + b] - s_rec);
+  }
+
+  // ---- gather-accumulate in list order
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const float* const Wff_c = L.W_ff + col;
+  const float* const Wrec_c = L.W_rec + col;
+  for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
+    const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
+    if (GEN) {
+      fill_chunk_from_words<FWD_THREADS>(wp, s_pref, c0, s_list);
+    } else {
+      for (int i = threadIdx.x; i < n; i += FWD_THREADS) {
+        const uint32_t q = c0 + i;
+        s_list[i] = q < n_ff ? ff_pool[s_ff + q] : (rec_pool[s_rec + (q - n_ff)] | REC_TAG);
+      }
+    }
+    __syncthreads();
+    if (active) {
+      // weight rows stream through a per-thread ring of GATHER_STAGES groups of GATHER_ROWS rows:
+      // the copies of the next groups are in flight while the oldest group is added, in list order
+      float4* const ring = s_stage + threadIdx.x;
+      const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
+      auto issue = [&](int g) {
+        if (g < n_groups) {
+          float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+#pragma unroll
+          for (int u = 0; u < GATHER_ROWS; ++u) {
+            const int i = g * GATHER_ROWS + u;
+            if (i < n) {
+              const uint32_t v = s_list[i];
+              cp_async16(dst + u * FWD_THREADS, ((v & REC_TAG) ? Wrec_c : Wff_c) + (size_t)(v & ~REC_TAG) * L.N);
+            }
+          }
+        }
+        cp_async_commit();
+      };
+      for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
+      for (int g = 0; g < n_groups; ++g) {
+        issue(g + GATHER_STAGES - 1);
+        cp_async_wait<GATHER_STAGES - 1>();
+        const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+#pragma unroll
+        for (int u = 0; u < GATHER_ROWS; ++u) {
+          if (g * GATHER_ROWS + u < n) {
+            const float4 w = src[u * FWD_THREADS];
+            acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+            acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+          }
+        }
+      }
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+  }
+
+  // ---- leak, reset by subtraction of the previous step's own spike, threshold
   uint32_t nib = 0;
   if (active) {
     const size_t k = (size_t)b * L.N + col;
-    const float4 vp = *reinterpret_cast<const float4*>(L.V_prev + k);
-    const uint32_t pw = L.rec_mask[(size_t)b * L.W + (col >> 5)] >> (col & 31);
     float4 v;
     v.x = __fsub_rn(__fmaf_rn(p.alpha, vp.x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
     v.y = __fsub_rn(__fmaf_rn(p.alpha, vp.y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
@@ -261,8 +333,13 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
 // ------------------------------------------------------------------------------------------
 // Backward step: delta^l_t = g_S sigma'(V^l_t - theta) + alpha delta^l_{t+1}, with
 // g_S = g_out + W_ff^{l+1} delta^{l+1}_t + W_rec^l delta^l_{t+1} - theta delta^l_{t+1}.
-// A warp owns R rows i of the weight matrices and all lanes split the contraction index;
-// R * BT partial sums per lane are reduced across the warp in a fixed tree.
+//
+// A CTA owns 32 rows i of the two weight matrices: 8 row groups of 4 rows, one warp per
+// (row group, group of BT samples).  The 32 lanes of a warp split the contraction index; a
+// thread-block cluster of CS CTAs splits it further (rank r takes the r-th slice of each
+// matrix).  Partial sums: per lane 4 x BT accumulators, reduced across the warp in a fixed
+// tree that leaves each lane with its own (row, sample) totals, then across the cluster through
+// distributed shared memory in rank order.  The order is fixed by (N, CS) alone.
 struct BwdLayer {
   const float* W_rec;     // [N][N]
   const float* W_ffa;     // W_ff of the layer above [N][N_post] or null
@@ -282,7 +359,9 @@ struct BwdParams {
   int surrogate, cell;
 };
 
-constexpr int BWD_WARPS = 4;
+constexpr int BWD_RT = 4;                 // rows per thread
+constexpr int BWD_WR = 8;                 // row groups (warps along rows) per CTA
+constexpr int BWD_TM = BWD_RT * BWD_WR;   // rows per CTA
 
 __device__ __forceinline__ float surrogate_grad(float v, float theta, float beta, int surrogate, int cell) {
   const float x = v - theta;
@@ -295,70 +374,141 @@ __device__ __forceinline__ float surrogate_grad(float v, float theta, float beta
   return beta * s * (1.f - s);
 }
 
-// Sum over the warp of 32 per-lane values; on return lane i holds the total of value i.
-__device__ __forceinline__ float warp_transpose_reduce(float (&v)[32], int lane) {
+// Sum over the warp of NV per-lane values; on return lane i holds the totals of values
+// i * NV/32 .. (i+1) * NV/32 - 1 in v[0 .. NV/32).
+template <int NV>
+__device__ __forceinline__ void warp_transpose_reduce(float (&v)[NV], int lane) {
+  int n = NV;
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) {
     const bool upper = (lane & s) != 0;
+    const int half = n / 2;
 #pragma unroll
-    for (int j = 0; j < s; ++j) {
-      const float send = upper ? v[j] : v[j + s];
-      const float keep = upper ? v[j + s] : v[j];
-      v[j] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-    }
-  }
-  return v[0];
-}
-
-template <int BT, int R>
-__device__ __forceinline__ void dot_rows(const float* __restrict__ W, int ld, int row0, int n_rows,
-                                         const float* __restrict__ d, int b0, int B, int K, int lane,
-                                         float (&acc)[32]) {
-  static_assert(BT * R == 32, "one value per lane after the reduction");
-  if (W == nullptr) return;
-  for (int k = lane * 4; k < K; k += 128) {
-    float4 w[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-      w[r] = row0 + r < n_rows ? ldg4(W + (size_t)(row0 + r) * ld + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int bb = 0; bb < BT; ++bb) {
-      const float4 dv = b0 + bb < B ? ldg4(d + (size_t)(b0 + bb) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        float a = acc[r * BT + bb];
-        a = fmaf(w[r].x, dv.x, a); a = fmaf(w[r].y, dv.y, a);
-        a = fmaf(w[r].z, dv.z, a); a = fmaf(w[r].w, dv.w, a);
-        acc[r * BT + bb] = a;
+    for (int j = 0; j < NV / 2; ++j) {
+      if (j < half) {
+        const float send = upper ? v[j] : v[j + half];
+        const float keep = upper ? v[j + half] : v[j];
+        v[j] = keep + __shfl_xor_sync(0xffffffffu, send, s);
       }
     }
+    n = half;
   }
 }
 
-template <int BT, int R>
-__global__ void __launch_bounds__(BWD_WARPS * 32) bwd_step_kernel(const __grid_constant__ BwdParams p) {
+constexpr int BWD_STAGES = 4;   // weight-row groups (4 rows x 512 B per warp) in flight per warp
+
+__device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer& L, int i, int b, float sum) {
+  if (i >= L.N || b >= p.B) return;
+  const size_t k = (size_t)b * L.N + i;
+  const float dn = L.d_next[k];
+  float g = sum + (L.g_out ? L.g_out[k] : 0.f);
+  if (p.cell == 0) g = fmaf(-p.theta, dn, g);
+  const float sp = surrogate_grad(L.V_delta[k], p.theta, p.beta, p.surrogate, p.cell);
+  const float dl = fmaf(g, sp, p.alpha * dn);
+  L.V_delta[k] = dl;
+  if (L.carry_out) L.carry_out[k] = dl;
+}
+
+// BT samples per thread (8 or 16), WB sample groups per CTA; launched with cluster size CS along x:
+// blockIdx.x = row_tile * CS + rank.
+template <int BT, int WB>
+__global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
+  constexpr int NT = 32 * BWD_WR * WB, NV = BWD_RT * BT, VPL = NV / 32, NWARP = BWD_WR * WB, BP = BT * WB;
+  constexpr int STAGE_F4 = (BWD_TM + BP) * 32;      // float4 per stage: 32 weight rows + BP delta rows, 128 k each
+  cg::cluster_group cluster = cg::this_cluster();
+  const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const BwdLayer& L = p.lay[blockIdx.z];
-  if (L.mode == 0) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int row0 = (blockIdx.x * BWD_WARPS + warp) * R;
-  if (row0 >= L.N) return;
-  for (int b0 = 0; b0 < p.B; b0 += BT) {
-    float acc[32];
+  if (L.mode == 0) return;                          // same for the whole cluster
+  const int tile_row0 = (blockIdx.x / CS) * BWD_TM;
+  if (tile_row0 >= L.N) return;                     // same for the whole cluster
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wr = warp % BWD_WR, wb = warp / BWD_WR;
+  const int row0 = tile_row0 + wr * BWD_RT;
+  __shared__ float s_part[NWARP * NV];
+  extern __shared__ float4 s_tiles[];               // [BWD_STAGES][BWD_TM + BP][32]
+  // this rank's slice of each contraction range, in units of 4 floats
+  const int q_rec = L.N / 4, q_ff = L.W_ffa ? L.N_post / 4 : 0;
+  const int lo_rec = (int)((long long)q_rec * rank / CS) * 4, hi_rec = (int)((long long)q_rec * (rank + 1) / CS) * 4;
+  const int lo_ff = (int)((long long)q_ff * rank / CS) * 4, hi_ff = (int)((long long)q_ff * (rank + 1) / CS) * 4;
+  // One chunk = 128 consecutive k of one matrix: a [32 rows][128] tile of W and a [BP][128] tile of
+  // delta.  Chunks run over this rank's slice of W_ff(l+1) first, then of W_rec, k ascending.  The
+  // tiles of the next BWD_STAGES-1 chunks are in flight (cp.async) while one chunk is multiplied.
+  const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
+  const int rlast = L.N - 1, blast = p.B - 1;
+  auto locate = [&](int it, const float*& W, const float*& d, int& ld, int& k0, int& hi) {
+    if (it < it_ff) { W = L.W_ffa; d = L.d_above; ld = L.N_post; k0 = lo_ff + it * 128; hi = hi_ff; }
+    else { W = L.W_rec; d = L.d_next; ld = L.N; k0 = lo_rec + (it - it_ff) * 128; hi = hi_rec; }
+  };
+
+  for (int bp0 = 0; bp0 < p.B; bp0 += BP) {
+    auto issue = [&](int it) {
+      if (it < it_all) {
+        const float* W; const float* d; int ld, k0, hi;
+        locate(it, W, d, ld, k0, hi);
+        float4* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F4;
+        for (int q = tid; q < STAGE_F4; q += NT) {
+          const int rr = q >> 5, k = k0 + 4 * (q & 31);
+          if (k < hi) {
+            // rows and samples past the end are clamped to the last valid one; their sums are never used
+            const float* src = rr < BWD_TM
+                                   ? W + (size_t)(tile_row0 + rr < rlast ? tile_row0 + rr : rlast) * ld + k
+                                   : d + (size_t)(bp0 + rr - BWD_TM < blast ? bp0 + rr - BWD_TM : blast) * ld + k;
+            cp_async16(st + q, src);
+          }
+        }
+      }
+      cp_async_commit();
+    };
+    float acc[NV];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-    dot_rows<BT, R>(L.W_ffa, L.N_post, row0, L.N, L.d_above, b0, p.B, L.N_post, lane, acc);
-    dot_rows<BT, R>(L.W_rec, L.N, row0, L.N, L.d_next, b0, p.B, L.N, lane, acc);
-    const float sum = warp_transpose_reduce(acc, lane);
-    const int i = row0 + lane / BT, b = b0 + lane % BT;
-    if (i < L.N && b < p.B) {
-      const size_t k = (size_t)b * L.N + i;
-      const float dn = L.d_next[k];
-      float g = sum + (L.g_out ? L.g_out[k] : 0.f);
-      if (p.cell == 0) g = fmaf(-p.theta, dn, g);
-      const float sp = surrogate_grad(L.V_delta[k], p.theta, p.beta, p.surrogate, p.cell);
-      const float dl = fmaf(g, sp, p.alpha * dn);
-      L.V_delta[k] = dl;
-      if (L.carry_out) L.carry_out[k] = dl;
+    for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+    for (int it = 0; it < BWD_STAGES - 1; ++it) issue(it);
+    for (int it = 0; it < it_all; ++it) {
+      cp_async_wait<BWD_STAGES - 2>();   // this thread's copies of chunk `it` have landed
+      __syncthreads();                   // ... everybody's have, and chunk it-1 has been consumed
+      issue(it + BWD_STAGES - 1);        // refills the stage chunk it-1 used
+      const float* W; const float* d; int ld, k0, hi;
+      locate(it, W, d, ld, k0, hi);
+      if (k0 + 4 * lane < hi) {
+        const float4* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F4 + lane;
+        float4 w[BWD_RT];
+#pragma unroll
+        for (int r = 0; r < BWD_RT; ++r) w[r] = st[(wr * BWD_RT + r) * 32];
+#pragma unroll
+        for (int bb = 0; bb < BT; ++bb) {
+          const float4 dv = st[(BWD_TM + wb * BT + bb) * 32];
+#pragma unroll
+          for (int r = 0; r < BWD_RT; ++r) {
+            float a = acc[r * BT + bb];
+            a = fmaf(w[r].x, dv.x, a); a = fmaf(w[r].y, dv.y, a);
+            a = fmaf(w[r].z, dv.z, a); a = fmaf(w[r].w, dv.w, a);
+            acc[r * BT + bb] = a;
+          }
+        }
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();   // the stages are free again for the next pass over the samples
+    const int b0 = bp0 + wb * BT;
+    warp_transpose_reduce<NV>(acc, lane);
+    if (CS == 1) {
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) {
+        const int idx = lane * VPL + j;
+        bwd_epilogue(p, L, row0 + idx / BT, b0 + idx % BT, acc[j]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) s_part[warp * NV + lane * VPL + j] = acc[j];
+      cluster.sync();
+      // every rank finishes a share of the tile: totals summed over the ranks in rank order
+      for (int e = rank + CS * tid; e < NWARP * NV; e += CS * NT) {
+        float sum = 0.f;
+        for (int r = 0; r < CS; ++r) sum += cluster.map_shared_rank(s_part, r)[e];
+        const int w = e / NV, idx = e % NV;
+        bwd_epilogue(p, L, tile_row0 + (w % BWD_WR) * BWD_RT + idx / BT, bp0 + (w / BWD_WR) * BT + idx % BT, sum);
+      }
+      cluster.sync();  // nobody leaves or overwrites s_part while another rank still reads it
     }
   }
 }
@@ -367,7 +517,10 @@ __global__ void __launch_bounds__(BWD_WARPS * 32) bwd_step_kernel(const __grid_c
 // Sparse outer-product weight gradient over a run of steps t = t1 .. t0+1:
 //   dW[j, :] += delta_t[b, :]   for every (t, b) in which presynaptic neuron j was active,
 // accumulated per element in the fixed order t descending, b ascending, starting from the
-// value already in dW.  A CTA owns 32 presynaptic rows (one spike word) and a column tile.
+// value already in dW.  A CTA owns 8 presynaptic rows (one warp each) and a column tile.
+// The (t, b) pairs are scanned in windows of DW_WINDOW: the warps first compact, by ballot
+// over the spike words, the list of pairs in which their row was active, then stream the
+// listed delta rows with DW_BATCH loads in flight, adding them in list order.
 struct DwArgs {
   float* dW;                 // [N_pre][N]
   const uint32_t* mask_row0; // spike words of the presynaptic layer for t = t0+1: [(t-t0-1)][B][Wm]
@@ -376,66 +529,95 @@ struct DwArgs {
   int N_pre, N, Wm, B, n_steps;
 };
 
+constexpr int DW_ROWS = 8;        // rows (warps) per CTA
+constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
+constexpr int DW_GROUP = 4;       // delta rows per copy group
+constexpr int DW_STAGES = 4;      // copy groups in flight per warp
+
 template <int U>
-__global__ void __launch_bounds__(256) dw_kernel(const DwArgs a) {
-  __shared__ uint32_t s_words[256];
+__global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
+  __shared__ uint32_t s_words[DW_WINDOW];
+  __shared__ uint32_t s_ev[DW_ROWS][DW_WINDOW];   // per row: indices of the pairs in which it was active
+  extern __shared__ float4 s_ring[];              // [DW_ROWS][DW_STAGES][DW_GROUP][U][32]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int wc = blockIdx.y;                 // spike word column = 32 presynaptic rows
-  const int rowb = wc * 32 + warp * 4;       // this warp's 4 rows
+  const int row = blockIdx.y * DW_ROWS + warp;
+  const int wc = (blockIdx.y * DW_ROWS) >> 5;               // spike word column of these rows
+  const int bit = ((blockIdx.y * DW_ROWS) & 31) + warp;     // this row's bit in it
   const int colb = blockIdx.x * (128 * U) + lane * 4;
-  float4 acc[4][U];
+  const bool row_ok = row < a.N_pre;
+  float4 acc[U];
 #pragma unroll
-  for (int r = 0; r < 4; ++r)
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int c = colb + u * 128;
-      acc[r][u] = (rowb + r < a.N_pre && c < a.N)
-                      ? *reinterpret_cast<const float4*>(a.dW + (size_t)(rowb + r) * a.N + c)
-                      : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+  for (int u = 0; u < U; ++u) {
+    const int c = colb + u * 128;
+    acc[u] = (row_ok && c < a.N) ? *reinterpret_cast<const float4*>(a.dW + (size_t)row * a.N + c)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float4* const ring = s_ring + (size_t)(threadIdx.x >> 5) * DW_STAGES * DW_GROUP * U * 32 + lane;
   const int n_pairs = a.n_steps * a.B;
-  for (int p0 = 0; p0 < n_pairs; p0 += 256) {
+  for (int p0 = 0; p0 < n_pairs; p0 += DW_WINDOW) {
+    const int lim = n_pairs - p0 < DW_WINDOW ? n_pairs - p0 : DW_WINDOW;
     __syncthreads();
-    {
-      const int pr = p0 + threadIdx.x;
-      uint32_t w = 0;
-      if (pr < n_pairs) {
-        const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;   // ts = t - t0 - 1, t descending
-        w = a.mask_row0[((size_t)ts * a.B + b) * a.Wm + wc];
-      }
-      s_words[threadIdx.x] = w;
+    for (int i = threadIdx.x; i < lim; i += 32 * DW_ROWS) {
+      const int pr = p0 + i;
+      const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;   // ts = t - t0 - 1, t descending
+      s_words[i] = a.mask_row0[((size_t)ts * a.B + b) * a.Wm + wc];
     }
     __syncthreads();
-    const int lim = n_pairs - p0 < 256 ? n_pairs - p0 : 256;
+    // this warp's row: ascending list of the window's pairs in which it was active
+    int n_ev = 0;
     for (int sb = 0; sb < lim; sb += 32) {
-      const uint32_t wd = s_words[sb + lane] >> (warp * 4);
+      const bool on = sb + lane < lim && ((s_words[sb + lane] >> bit) & 1u);
+      const uint32_t m = __ballot_sync(0xffffffffu, on);
+      if (on) s_ev[warp][n_ev + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(p0 + sb + lane);
+      n_ev += __popc(m);
+    }
+    __syncwarp();
+    if (row_ok) {
+      // the listed delta rows stream through a per-warp ring of DW_STAGES groups of DW_GROUP rows
+      const int n_groups = (n_ev + DW_GROUP - 1) / DW_GROUP;
+      auto issue = [&](int g) {
+        if (g < n_groups) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        uint32_t m = __ballot_sync(0xffffffffu, (wd >> r) & 1u);
-        while (m) {
-          const int q = __ffs(m) - 1;
-          m &= m - 1;
-          const int pr = p0 + sb + q;
-          const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
-          const float* d = a.delta0 + (size_t)ts * a.slot_stride + (size_t)b * a.N + colb;
+          for (int q = 0; q < DW_GROUP; ++q) {
+            const int e = g * DW_GROUP + q;
+            if (e < n_ev) {
+              const int pr = (int)s_ev[warp][e];
+              const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
+              const float* d = a.delta0 + (size_t)ts * a.slot_stride + (size_t)b * a.N + colb;
 #pragma unroll
-          for (int u = 0; u < U; ++u)
-            if (colb + u * 128 < a.N) {
-              const float4 dv = ldg4(d + u * 128);
-              acc[r][u].x += dv.x; acc[r][u].y += dv.y; acc[r][u].z += dv.z; acc[r][u].w += dv.w;
+              for (int u = 0; u < U; ++u)
+                if (colb + u * 128 < a.N) cp_async16(ring + (((g % DW_STAGES) * DW_GROUP + q) * U + u) * 32, d + u * 128);
             }
+          }
+        }
+        cp_async_commit();
+      };
+      for (int g = 0; g < DW_STAGES - 1; ++g) issue(g);
+      for (int g = 0; g < n_groups; ++g) {
+        issue(g + DW_STAGES - 1);
+        cp_async_wait<DW_STAGES - 1>();
+#pragma unroll
+        for (int q = 0; q < DW_GROUP; ++q) {
+          if (g * DW_GROUP + q < n_ev) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+              if (colb + u * 128 < a.N) {
+                const float4 dv = ring[(((g % DW_STAGES) * DW_GROUP + q) * U + u) * 32];
+                acc[u].x += dv.x; acc[u].y += dv.y; acc[u].z += dv.z; acc[u].w += dv.w;
+              }
+          }
         }
       }
+      cp_async_wait<0>();
     }
   }
-#pragma unroll
-  for (int r = 0; r < 4; ++r)
+  if (row_ok) {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int c = colb + u * 128;
-      if (rowb + r < a.N_pre && c < a.N)
-        *reinterpret_cast<float4*>(a.dW + (size_t)(rowb + r) * a.N + c) = acc[r][u];
+      if (c < a.N) *reinterpret_cast<float4*>(a.dW + (size_t)row * a.N + c) = acc[u];
     }
+  }
 }
 
 // ------------------------------------------------------------------------------------------

@@ -284,8 +284,8 @@ struct Exec {
   }
 
   snn_status launch_fwd(const FwdParams& p, bool gen) {
-    if (gen) fwd_step_kernel<true><<<fwd_grid(), FWD_THREADS, 0, main>>>(p);
-    else fwd_step_kernel<false><<<fwd_grid(), FWD_THREADS, 0, main>>>(p);
+    if (gen) fwd_step_kernel<true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+    else fwd_step_kernel<false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
     ++launches;
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
@@ -348,13 +348,24 @@ struct Exec {
   }
 
   template <int U> void launch_dw(const DwArgs& d) {
-    dim3 grid((d.N + 128 * U - 1) / (128 * U), (d.N_pre + 31) / 32);
-    dw_kernel<U><<<grid, 256, 0, main>>>(d);
+    dim3 grid((d.N + 128 * U - 1) / (128 * U), (d.N_pre + DW_ROWS - 1) / DW_ROWS);
+    dw_kernel<U><<<grid, 32 * DW_ROWS, (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4), main>>>(d);
     ++launches;
   }
+  template <int BT, int WB> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles * CS, 1, L);
+    cfg.blockDim = dim3(32 * BWD_WR * WB);
+    cfg.stream = main;
+    cfg.dynamicSmemBytes = (size_t)BWD_STAGES * (BWD_TM + BT * WB) * 32 * sizeof(float4);
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, bwd_step_kernel<BT, WB>, p);
+  }
   void run_dw(const DwArgs& d) {
-    if (d.N >= 4096) launch_dw<4>(d);
-    else if (d.N >= 256) launch_dw<2>(d);
+    if (d.N >= 512) launch_dw<2>(d);
     else launch_dw<1>(d);
   }
 
@@ -369,6 +380,15 @@ struct Exec {
     p.surrogate = net->surrogate; p.cell = net->cell;
     int maxN = 0;
     for (int l = 1; l <= L; ++l) maxN = std::max(maxN, sz[l]);
+    // cluster size along the contraction index: enough CTAs to fill the GPU, at least one full
+    // warp pass (128 values) per rank; a function of the network sizes only
+    const int tiles = (maxN + BWD_TM - 1) / BWD_TM;
+    int minN = maxN;
+    for (int l = 1; l <= L; ++l) minN = std::min(minN, sz[l]);
+    // (one wave: two 256-thread CTAs or one 512-thread CTA per SM on 148 SMs)
+    const int wave = B <= 16 ? 296 : 148;
+    int CS = 1;
+    while (CS < 8 && tiles * L * CS * 2 <= wave && minN / (4 * CS * 2) >= 32) CS *= 2;
     int span = begin_span(SNN_PHASE_BWD);
     for (int s = 0; s <= n + L - 2; ++s) {
       for (int l = L; l >= 1; --l) {
@@ -385,13 +405,11 @@ struct Exec {
         f.g_out = l == L ? at<float>(lo.g_out) : nullptr;
         f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
       }
-      if (B <= 8) {
-        dim3 grid((maxN + BWD_WARPS * 4 - 1) / (BWD_WARPS * 4), 1, L);
-        bwd_step_kernel<8, 4><<<grid, BWD_WARPS * 32, 0, main>>>(p);
-      } else {
-        dim3 grid((maxN + BWD_WARPS * 2 - 1) / (BWD_WARPS * 2), 1, L);
-        bwd_step_kernel<16, 2><<<grid, BWD_WARPS * 32, 0, main>>>(p);
-      }
+      cudaError_t le;
+      if (B <= 8) le = launch_bwd<8, 1>(p, tiles, CS);
+      else if (B <= 16) le = launch_bwd<16, 1>(p, tiles, CS);
+      else le = launch_bwd<16, 2>(p, tiles, CS);
+      if (le != cudaSuccess) return fail(net, SNN_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(le));
       ++launches;
     }
     carry_cur ^= 1;
@@ -485,6 +503,21 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     CUDA_TRY(cudaEventCreateWithFlags(&net->ev_main, cudaEventDisableTiming));
     CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[0], cudaEventDisableTiming));
     CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[1], cudaEventDisableTiming));
+  }
+  {
+    static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
+    if (!smem_opt_in) {
+      const int dw1 = (int)(DW_ROWS * DW_STAGES * DW_GROUP * 1 * 32 * sizeof(float4));
+      auto bwd_smem = [](int bp) { return (int)(BWD_STAGES * (BWD_TM + bp) * 32 * sizeof(float4)); };
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(8)));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(16)));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(32)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1));
+      smem_opt_in = true;
+    }
   }
   cudaStream_t ms = ex.main;
   const auto& sz = net->sizes;
