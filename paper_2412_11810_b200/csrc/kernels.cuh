@@ -527,18 +527,22 @@ struct DwArgs {
   const float* delta0;       // delta of step t0+1: delta(t, b) = delta0 + (t-t0-1) * slot_stride + b * N
   size_t slot_stride;        // floats between consecutive steps
   int N_pre, N, Wm, B, n_steps;
+  int window;                // (t, b) pairs compacted at a time: min(n_steps * B rounded up to 32, DW_WINDOW)
 };
 
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
 constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
 constexpr int DW_GROUP = 4;       // delta rows per copy group
-constexpr int DW_STAGES = 4;      // copy groups in flight per warp
+constexpr int DW_STAGES = 2;      // copy groups in flight per warp
 
 template <int U>
 __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
-  __shared__ uint32_t s_words[DW_WINDOW];
-  __shared__ uint32_t s_ev[DW_ROWS][DW_WINDOW];   // per row: indices of the pairs in which it was active
-  extern __shared__ float4 s_ring[];              // [DW_ROWS][DW_STAGES][DW_GROUP][U][32]
+  // dynamic shared memory: copy ring [DW_ROWS][DW_STAGES][DW_GROUP][U][32] float4, then the spike
+  // words of one window [window] and the per-row lists of active pairs [DW_ROWS][window]
+  extern __shared__ float4 s_ring[];
+  const int window = a.window;
+  uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_ring + (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32);
+  uint32_t* const s_evw = s_words + window + (size_t)(threadIdx.x >> 5) * window;   // this warp's list
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row = blockIdx.y * DW_ROWS + warp;
   const int wc = (blockIdx.y * DW_ROWS) >> 5;               // spike word column of these rows
@@ -554,8 +558,8 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
   }
   float4* const ring = s_ring + (size_t)(threadIdx.x >> 5) * DW_STAGES * DW_GROUP * U * 32 + lane;
   const int n_pairs = a.n_steps * a.B;
-  for (int p0 = 0; p0 < n_pairs; p0 += DW_WINDOW) {
-    const int lim = n_pairs - p0 < DW_WINDOW ? n_pairs - p0 : DW_WINDOW;
+  for (int p0 = 0; p0 < n_pairs; p0 += window) {
+    const int lim = n_pairs - p0 < window ? n_pairs - p0 : window;
     __syncthreads();
     for (int i = threadIdx.x; i < lim; i += 32 * DW_ROWS) {
       const int pr = p0 + i;
@@ -568,7 +572,7 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
     for (int sb = 0; sb < lim; sb += 32) {
       const bool on = sb + lane < lim && ((s_words[sb + lane] >> bit) & 1u);
       const uint32_t m = __ballot_sync(0xffffffffu, on);
-      if (on) s_ev[warp][n_ev + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(p0 + sb + lane);
+      if (on) s_evw[n_ev + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(p0 + sb + lane);
       n_ev += __popc(m);
     }
     __syncwarp();
@@ -581,7 +585,7 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
           for (int q = 0; q < DW_GROUP; ++q) {
             const int e = g * DW_GROUP + q;
             if (e < n_ev) {
-              const int pr = (int)s_ev[warp][e];
+              const int pr = (int)s_evw[e];
               const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
               const float* d = a.delta0 + (size_t)ts * a.slot_stride + (size_t)b * a.N + colb;
 #pragma unroll

@@ -347,9 +347,13 @@ struct Exec {
     return SNN_OK;
   }
 
-  template <int U> void launch_dw(const DwArgs& d) {
+  template <int U> void launch_dw(DwArgs d) {
     dim3 grid((d.N + 128 * U - 1) / (128 * U), (d.N_pre + DW_ROWS - 1) / DW_ROWS);
-    dw_kernel<U><<<grid, 32 * DW_ROWS, (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4), main>>>(d);
+    const int pairs = d.n_steps * d.B;
+    d.window = std::min(DW_WINDOW, (pairs + 31) / 32 * 32);
+    const size_t smem = (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4) +
+                        (size_t)(DW_ROWS + 1) * d.window * sizeof(uint32_t);
+    dw_kernel<U><<<grid, 32 * DW_ROWS, smem, main>>>(d);
     ++launches;
   }
   template <int BT, int WB> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
@@ -508,14 +512,15 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
     if (!smem_opt_in) {
       const int dw1 = (int)(DW_ROWS * DW_STAGES * DW_GROUP * 1 * 32 * sizeof(float4));
+      const int dww = (int)((DW_ROWS + 1) * DW_WINDOW * sizeof(uint32_t));
       auto bwd_smem = [](int bp) { return (int)(BWD_STAGES * (BWD_TM + bp) * 32 * sizeof(float4)); };
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(16)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(32)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
       smem_opt_in = true;
     }
   }
