@@ -116,10 +116,17 @@ __device__ void fill_chunk_from_words(const WordPair& wp, const uint32_t* s_pref
 
 // Step 2b: the lists to global memory (entries past the room left in a pool are dropped).
 // Part a goes to dst_a (if not null), part b to dst_b; n_a_bits = set bits of part a.
-template <int NT>
+// Graded events also store their value (read from the dense source rows val_a / val_b) and, per
+// spike word, the number of events before it (pref_a / pref_b), which lets a reader find the
+// position of a given neuron's event without searching.
+template <int NT, bool GRADED>
 __device__ void write_lists_from_words(const WordPair& wp, const uint32_t* s_pref, uint32_t n_a_bits,
                                        uint32_t* __restrict__ dst_a, uint32_t room_a,
-                                       uint32_t* __restrict__ dst_b, uint32_t room_b) {
+                                       uint32_t* __restrict__ dst_b, uint32_t room_b,
+                                       const float* __restrict__ val_a = nullptr, float* __restrict__ vdst_a = nullptr,
+                                       uint16_t* __restrict__ pref_a = nullptr,
+                                       const float* __restrict__ val_b = nullptr, float* __restrict__ vdst_b = nullptr,
+                                       uint16_t* __restrict__ pref_b = nullptr) {
   const int n_words = wp.size();
   for (int w = threadIdx.x; w < n_words; w += NT) {
     uint32_t bits = wp.get(w);
@@ -130,13 +137,52 @@ __device__ void write_lists_from_words(const WordPair& wp, const uint32_t* s_pre
     const uint32_t room = in_a ? room_a : room_b;
     if (!in_a) p -= n_a_bits;
     const uint32_t first = wp.first_index(w) & ~REC_TAG;
+    if (GRADED) (in_a ? pref_a : pref_b)[in_a ? w : w - wp.n_a] = (uint16_t)p;
     while (bits) {
       const int bit = __ffs(bits) - 1;
       bits &= bits - 1;
-      if (p < room) dst[p] = first + bit;
+      if (p < room) {
+        dst[p] = first + bit;
+        if (GRADED) (in_a ? vdst_a : vdst_b)[p] = (in_a ? val_a : val_b)[first + bit];
+      }
       ++p;
     }
   }
+}
+
+// Step 2a for graded events: the values that go with fill_chunk_from_words' indices.
+template <int NT>
+__device__ void fill_values_from_words(const WordPair& wp, const uint32_t* s_pref, uint32_t c0,
+                                       const float* __restrict__ val_a, const float* __restrict__ val_b,
+                                       float* s_val) {
+  const int n_words = wp.size();
+  for (int w = threadIdx.x; w < n_words; w += NT) {
+    uint32_t bits = wp.get(w);
+    if (!bits) continue;
+    uint32_t p = s_pref[w];
+    if (p >= c0 + LIST_CHUNK || p + __popc(bits) <= c0) continue;
+    const bool in_a = w < wp.n_a;
+    const float* src = (in_a ? val_a : val_b) + (in_a ? w : w - wp.n_a) * 32;
+    while (bits) {
+      const int bit = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (p >= c0 && p < c0 + LIST_CHUNK) s_val[p - c0] = src[bit];
+      ++p;
+    }
+  }
+}
+
+// Dense fp32 rows -> spike words (bit = value is not zero): one warp per word.
+__global__ void __launch_bounds__(256)
+dense_to_words_kernel(const float* __restrict__ dense, size_t n_rows, int N, int W, uint32_t* __restrict__ words) {
+  const size_t wid = ((size_t)blockIdx.x * 256 + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= n_rows * (size_t)W) return;
+  const size_t row = wid / W;
+  const int col = (int)(wid % W) * 32 + lane;
+  const bool on = col < N && dense[row * N + col] != 0.f;
+  const uint32_t m = __ballot_sync(0xffffffffu, on);
+  if (lane == 0) words[wid] = m;
 }
 
 // Stand-alone compaction of many rows: one CTA per row.
@@ -148,8 +194,8 @@ compact_rows_kernel(const uint32_t* __restrict__ masks, int n_words, uint32_t* _
   const size_t row = blockIdx.x;
   WordPair wp{masks + row * (size_t)n_words, n_words, nullptr, 0};
   const uint32_t total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
-  write_lists_from_words<FWD_THREADS>(wp, s_pref, total, idx_out + row * (size_t)capacity, (uint32_t)capacity,
-                                      nullptr, 0);
+  write_lists_from_words<FWD_THREADS, false>(wp, s_pref, total, idx_out + row * (size_t)capacity,
+                                             (uint32_t)capacity, nullptr, 0);
   if (threadIdx.x == 0) count_out[row] = total;
 }
 
@@ -169,7 +215,16 @@ struct FwdLayer {
   uint32_t* ff_off;           // offsets row t of the layer below: [b] start, [B + b] end
   uint32_t* rec_pool;         // own event pool [B][rec_cap]
   uint32_t* rec_off;          // own offsets row t-1
-  uint32_t* counts;           // [B][N] spike counts (last layer, generating mode) or null
+  uint32_t* counts;           // [B][N] spike counts (last layer, generating mode) or null;
+                              // the graded cell keeps the fp32 sum of its events there instead
+  // graded cell only
+  const float* ff_val_src;    // [B][N_pre] dense values of the layer below at step t   (generating mode)
+  const float* rec_val_src;   // [B][N]     own dense event values at step t-1          (generating mode)
+  float* act_out;             // [B][N]     own dense event values at step t            (generating mode)
+  float* ff_vals;             // values that go with ff_pool
+  float* rec_vals;            // values that go with rec_pool
+  uint16_t* ff_pref;          // [B][W_pre] events before each spike word, layer below at step t
+  uint16_t* rec_pref;         // [B][W]     the same for the own layer at step t-1
   uint32_t ff_cap, rec_cap;
   int N_pre, N, W_pre, W;
   int mode;                   // 0 idle, 1 step, 2 only write the list of own spikes at t-1
@@ -187,7 +242,7 @@ constexpr int GATHER_ROWS = 8;     // weight rows per copy group
 constexpr int GATHER_STAGES = 5;   // copy groups in flight per thread (40 rows, 80 KB per CTA)
 constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
-template <bool GEN>
+template <bool GEN, bool GRADED>
 __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_constant__ FwdParams p) {
   const FwdLayer& L = p.lay[blockIdx.z];
   if (L.mode == 0) return;
@@ -198,6 +253,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   __shared__ uint32_t s_list[LIST_CHUNK];
   __shared__ uint32_t s_pref[GEN ? 2 * MAX_WORDS + 1 : 1];
   __shared__ uint32_t s_warp[FWD_THREADS / 32];
+  __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
   extern __shared__ float4 s_stage[];   // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
   const int col = col0 + threadIdx.x * 4;
   const bool active = col < L.N;
@@ -209,7 +265,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   uint32_t pw = 0;
   if (step && active) {
     vp = *reinterpret_cast<const float4*>(L.V_prev + (size_t)b * L.N + col);
-    pw = L.rec_mask[(size_t)b * L.W + (col >> 5)] >> (col & 31);
+    if (!GRADED) pw = L.rec_mask[(size_t)b * L.W + (col >> 5)] >> (col & 31);
   }
 
   // ---- the two event lists of this step as one: feed-forward events, then recurrent events
@@ -227,8 +283,15 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
       s_rec = L.rec_off[b];
       if (wr_ff) s_ff = L.ff_off[b];
       const uint32_t room_ff = wr_ff ? L.ff_cap - s_ff : 0, room_rec = L.rec_cap - s_rec;
-      write_lists_from_words<FWD_THREADS>(wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff,
-                                          rec_pool + s_rec, room_rec);
+      if (GRADED)
+        write_lists_from_words<FWD_THREADS, true>(
+            wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff, rec_pool + s_rec, room_rec,
+            wr_ff ? L.ff_val_src + (size_t)b * L.N_pre : nullptr, L.ff_vals + (size_t)b * L.ff_cap + s_ff,
+            L.ff_pref + (size_t)b * L.W_pre, L.rec_val_src + (size_t)b * L.N,
+            L.rec_vals + (size_t)b * L.rec_cap + s_rec, L.rec_pref + (size_t)b * L.W);
+      else
+        write_lists_from_words<FWD_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff,
+                                                   rec_pool + s_rec, room_rec);
       if (threadIdx.x == 0) {
         const uint32_t n_rec = total - n_ff;
         L.rec_off[B + b] = s_rec + (n_rec < room_rec ? n_rec : room_rec);
@@ -250,10 +313,16 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
     const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
     if (GEN) {
       fill_chunk_from_words<FWD_THREADS>(wp, s_pref, c0, s_list);
+      if (GRADED)
+        fill_values_from_words<FWD_THREADS>(wp, s_pref, c0, L.ff_val_src + (size_t)b * L.N_pre,
+                                            L.rec_val_src + (size_t)b * L.N, s_val);
     } else {
       for (int i = threadIdx.x; i < n; i += FWD_THREADS) {
         const uint32_t q = c0 + i;
         s_list[i] = q < n_ff ? ff_pool[s_ff + q] : (rec_pool[s_rec + (q - n_ff)] | REC_TAG);
+        if (GRADED)
+          s_val[i] = q < n_ff ? L.ff_vals[(size_t)b * L.ff_cap + s_ff + q]
+                              : L.rec_vals[(size_t)b * L.rec_cap + s_rec + (q - n_ff)];
       }
     }
     __syncthreads();
@@ -285,8 +354,14 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
         for (int u = 0; u < GATHER_ROWS; ++u) {
           if (g * GATHER_ROWS + u < n) {
             const float4 w = src[u * FWD_THREADS];
-            acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
-            acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+            if (GRADED) {   // one fused multiply-add per event and neuron
+              const float sv = s_val[g * GATHER_ROWS + u];
+              acc.x = __fmaf_rn(sv, w.x, acc.x); acc.y = __fmaf_rn(sv, w.y, acc.y);
+              acc.z = __fmaf_rn(sv, w.z, acc.z); acc.w = __fmaf_rn(sv, w.w, acc.w);
+            } else {        // a binary spike: the fused multiply-add is an exact plain add
+              acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+              acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+            }
           }
         }
       }
@@ -300,17 +375,33 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   if (active) {
     const size_t k = (size_t)b * L.N + col;
     float4 v;
-    v.x = __fsub_rn(__fmaf_rn(p.alpha, vp.x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
-    v.y = __fsub_rn(__fmaf_rn(p.alpha, vp.y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
-    v.z = __fsub_rn(__fmaf_rn(p.alpha, vp.z, acc.z), __fmul_rn(p.theta, (float)((pw >> 2) & 1u)));
-    v.w = __fsub_rn(__fmaf_rn(p.alpha, vp.w, acc.w), __fmul_rn(p.theta, (float)((pw >> 3) & 1u)));
+    if (GRADED) {   // leaky integrator without reset
+      v.x = __fmaf_rn(p.alpha, vp.x, acc.x); v.y = __fmaf_rn(p.alpha, vp.y, acc.y);
+      v.z = __fmaf_rn(p.alpha, vp.z, acc.z); v.w = __fmaf_rn(p.alpha, vp.w, acc.w);
+    } else {
+      v.x = __fsub_rn(__fmaf_rn(p.alpha, vp.x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
+      v.y = __fsub_rn(__fmaf_rn(p.alpha, vp.y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
+      v.z = __fsub_rn(__fmaf_rn(p.alpha, vp.z, acc.z), __fmul_rn(p.theta, (float)((pw >> 2) & 1u)));
+      v.w = __fsub_rn(__fmaf_rn(p.alpha, vp.w, acc.w), __fmul_rn(p.theta, (float)((pw >> 3) & 1u)));
+    }
     *reinterpret_cast<float4*>(L.V_out + k) = v;
     if (L.V_keep) *reinterpret_cast<float4*>(L.V_keep + k) = v;
     if (L.V_dbg) *reinterpret_cast<float4*>(L.V_dbg + k) = v;
     if (GEN) {
       nib = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) |
             (v.w > p.theta ? 8u : 0u);
-      if (L.counts && nib) {
+      if (GRADED) {
+        const float4 a = make_float4(nib & 1u ? v.x : 0.f, nib & 2u ? v.y : 0.f, nib & 4u ? v.z : 0.f,
+                                     nib & 8u ? v.w : 0.f);
+        *reinterpret_cast<float4*>(L.act_out + k) = a;
+        if (L.counts && nib) {   // time-summed events, added in step order
+          float4* c = reinterpret_cast<float4*>(L.counts + k);
+          float4 cv = *c;
+          cv.x = __fadd_rn(cv.x, a.x); cv.y = __fadd_rn(cv.y, a.y);
+          cv.z = __fadd_rn(cv.z, a.z); cv.w = __fadd_rn(cv.w, a.w);
+          *c = cv;
+        }
+      } else if (L.counts && nib) {
         uint4* c = reinterpret_cast<uint4*>(L.counts + k);
         uint4 cv = *c;
         cv.x += nib & 1u; cv.y += (nib >> 1) & 1u; cv.z += (nib >> 2) & 1u; cv.w += (nib >> 3) & 1u;
@@ -528,6 +619,11 @@ struct DwArgs {
   size_t slot_stride;        // floats between consecutive steps
   int N_pre, N, Wm, B, n_steps;
   int window;                // (t, b) pairs compacted at a time: min(n_steps * B rounded up to 32, DW_WINDOW)
+  // graded cell only: where the value of an event is found (same step indexing as mask_row0)
+  const uint32_t* off_row0;  // list offsets of the presynaptic layer [(t-t0-1)][B]
+  const uint16_t* pref_row0; // events before each spike word [(t-t0-1)][B][Wm]
+  const float* vals;         // value pool [B][cap]
+  size_t cap;
 };
 
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
@@ -535,7 +631,7 @@ constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
 constexpr int DW_GROUP = 4;       // delta rows per copy group
 constexpr int DW_STAGES = 2;      // copy groups in flight per warp
 
-template <int U>
+template <int U, bool GRADED>
 __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
   // dynamic shared memory: copy ring [DW_ROWS][DW_STAGES][DW_GROUP][U][32] float4, then the spike
   // words of one window [window] and the per-row lists of active pairs [DW_ROWS][window]
@@ -543,6 +639,8 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
   const int window = a.window;
   uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_ring + (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32);
   uint32_t* const s_evw = s_words + window + (size_t)(threadIdx.x >> 5) * window;   // this warp's list
+  float* const s_valw = reinterpret_cast<float*>(s_words + (size_t)(DW_ROWS + 1) * window) +
+                        (size_t)(threadIdx.x >> 5) * window;                         // and its values (graded)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row = blockIdx.y * DW_ROWS + warp;
   const int wc = (blockIdx.y * DW_ROWS) >> 5;               // spike word column of these rows
@@ -572,7 +670,18 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
     for (int sb = 0; sb < lim; sb += 32) {
       const bool on = sb + lane < lim && ((s_words[sb + lane] >> bit) & 1u);
       const uint32_t m = __ballot_sync(0xffffffffu, on);
-      if (on) s_evw[n_ev + __popc(m & ((1u << lane) - 1u))] = (uint32_t)(p0 + sb + lane);
+      if (on) {
+        const int slot = n_ev + __popc(m & ((1u << lane) - 1u));
+        const int pr = p0 + sb + lane;
+        s_evw[slot] = (uint32_t)pr;
+        if (GRADED) {   // the event's value: list start + events before its word + events before it in the word
+          const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
+          const size_t rowi = (size_t)ts * a.B + b;
+          const uint32_t pos = a.off_row0[rowi] + a.pref_row0[rowi * a.Wm + wc] +
+                               __popc(s_words[sb + lane] & ((1u << bit) - 1u));
+          s_valw[slot] = pos < a.cap ? a.vals[(size_t)b * a.cap + pos] : 0.f;
+        }
+      }
       n_ev += __popc(m);
     }
     __syncwarp();
@@ -607,7 +716,13 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
             for (int u = 0; u < U; ++u)
               if (colb + u * 128 < a.N) {
                 const float4 dv = ring[(((g % DW_STAGES) * DW_GROUP + q) * U + u) * 32];
-                acc[u].x += dv.x; acc[u].y += dv.y; acc[u].z += dv.z; acc[u].w += dv.w;
+                if (GRADED) {
+                  const float sv = s_valw[g * DW_GROUP + q];
+                  acc[u].x = fmaf(sv, dv.x, acc[u].x); acc[u].y = fmaf(sv, dv.y, acc[u].y);
+                  acc[u].z = fmaf(sv, dv.z, acc[u].z); acc[u].w = fmaf(sv, dv.w, acc[u].w);
+                } else {
+                  acc[u].x += dv.x; acc[u].y += dv.y; acc[u].z += dv.z; acc[u].w += dv.w;
+                }
               }
           }
         }
@@ -628,8 +743,8 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
 // Readout: logits = scale * c W_out, mean soft-max cross-entropy, and the gradients that
 // leave it.  One small dense product per training step; plain fp32.
 __global__ void __launch_bounds__(256)
-readout_logits_kernel(const uint32_t* __restrict__ counts, const float* __restrict__ W_out, int N_L, int N_out,
-                      float scale, float* __restrict__ logits) {
+readout_logits_kernel(const uint32_t* __restrict__ counts, int counts_are_float, const float* __restrict__ W_out,
+                      int N_L, int N_out, float scale, float* __restrict__ logits) {
   extern __shared__ float s_part[];  // [8][N_out]
   const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int k = lane; k < N_out; k += 32) s_part[warp * N_out + k] = 0.f;
@@ -637,7 +752,7 @@ readout_logits_kernel(const uint32_t* __restrict__ counts, const float* __restri
   for (int i = warp; i < N_L; i += 8) {
     const uint32_t c = counts[(size_t)b * N_L + i];
     if (!c) continue;
-    const float cf = (float)c;
+    const float cf = counts_are_float ? __uint_as_float(c) : (float)c;
     for (int k = lane; k < N_out; k += 32) s_part[warp * N_out + k] = fmaf(cf, W_out[(size_t)i * N_out + k], s_part[warp * N_out + k]);
   }
   __syncthreads();
@@ -687,13 +802,16 @@ readout_gout_kernel(const float* __restrict__ W_out, const float* __restrict__ d
 
 // dW_out[i, k] = scale * sum_b c[b, i] dlogits[b, k]
 __global__ void __launch_bounds__(256)
-readout_dwout_kernel(const uint32_t* __restrict__ counts, const float* __restrict__ dlogits, int B, int N_L,
-                     int N_out, float scale, float* __restrict__ dW_out) {
+readout_dwout_kernel(const uint32_t* __restrict__ counts, int counts_are_float, const float* __restrict__ dlogits,
+                     int B, int N_L, int N_out, float scale, float* __restrict__ dW_out) {
   const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
   if (idx >= (size_t)N_L * N_out) return;
   const int i = (int)(idx / N_out), k = (int)(idx % N_out);
   float s = 0.f;
-  for (int b = 0; b < B; ++b) s = fmaf((float)counts[(size_t)b * N_L + i], dlogits[(size_t)b * N_out + k], s);
+  for (int b = 0; b < B; ++b) {
+    const uint32_t c = counts[(size_t)b * N_L + i];
+    s = fmaf(counts_are_float ? __uint_as_float(c) : (float)c, dlogits[(size_t)b * N_out + k], s);
+  }
   dW_out[idx] = scale * s;
 }
 

@@ -49,6 +49,7 @@ size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 struct Layout {
   size_t status, logits, dlogits, g_out, counts, carry[2], in_stage, tg_stage;
   size_t off[MAXL + 1], pool[MAXL + 1], mask[MAXL + 1];
+  size_t vals[MAXL + 1], pref[MAXL + 1], act[MAXL + 1], in_words;   // graded cell only
   uint32_t cap[MAXL + 1];
   int words[MAXL + 1];
   size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
@@ -79,7 +80,9 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.carry[0] = take(lo.state_bytes);
   lo.carry[1] = take(lo.state_bytes);
   lo.words[0] = (sz[0] + 31) / 32;
-  lo.in_stage = take(4 * (size_t)T * B * lo.words[0]);
+  const bool graded = net->cell == SNN_CELL_GRADED;
+  lo.in_stage = take(4 * (size_t)T * B * (graded ? sz[0] : lo.words[0]));
+  lo.in_words = graded ? take(4 * (size_t)T * B * lo.words[0]) : 0;
   lo.tg_stage = take(4 * (size_t)B);
   const size_t ev0 = cur;
   for (int l = 0; l <= L; ++l) {
@@ -90,6 +93,9 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     lo.off[l] = take(4 * (size_t)(T + 2) * B);
     lo.pool[l] = take(4 * (size_t)B * lo.cap[l]);
     lo.mask[l] = l == 0 ? 0 : take(4 * (size_t)(T + 1) * B * lo.words[l]);
+    lo.vals[l] = graded ? take(4 * (size_t)B * lo.cap[l]) : 0;
+    lo.pref[l] = graded ? take(2 * (size_t)(T + 2) * B * lo.words[l]) : 0;
+    lo.act[l] = (graded && l > 0) ? take(4 * (size_t)2 * B * sz[l]) : 0;
   }
   lo.event_bytes = cur - ev0;
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
@@ -239,11 +245,18 @@ struct Exec {
   template <class Tp> Tp* at(size_t off) const { return reinterpret_cast<Tp*>(ws + off); }
   float* slot(int s, int l) const { return at<float>(lo.slots + (size_t)s * lo.state_bytes) + lo.layer_off[l]; }
   float* carry(int which, int l) const { return at<float>(lo.carry[which]) + lo.layer_off[l]; }
-  const uint32_t* in_mask(int t) const {  // spikes of the input at step t (t >= 1)
-    const uint32_t* base = (a->flags & SNN_FLAG_INPUT_ON_HOST) ? at<uint32_t>(lo.in_stage)
-                                                               : reinterpret_cast<const uint32_t*>(a->input);
+  bool graded() const { return net->cell == SNN_CELL_GRADED; }
+  const void* in_base() const { return (a->flags & SNN_FLAG_INPUT_ON_HOST) ? (const void*)(ws + lo.in_stage) : a->input; }
+  const uint32_t* in_mask(int t) const {  // spike words of the input at step t (t >= 1)
+    const uint32_t* base = graded() ? at<uint32_t>(lo.in_words) : reinterpret_cast<const uint32_t*>(in_base());
     return base + (size_t)(t - 1) * B * lo.words[0];
   }
+  const float* in_dense(int t) const {   // graded input values at step t
+    return reinterpret_cast<const float*>(in_base()) + (size_t)(t - 1) * B * net->sizes[0];
+  }
+  float* vals(int l) const { return at<float>(lo.vals[l]); }
+  uint16_t* pref(int l, int t) const { return at<uint16_t>(lo.pref[l]) + (size_t)t * B * lo.words[l]; }
+  float* act(int l, int parity) const { return at<float>(lo.act[l]) + (size_t)parity * B * net->sizes[l]; }
   uint32_t* mask(int l, int t) const { return at<uint32_t>(lo.mask[l]) + (size_t)t * B * lo.words[l]; }
   uint32_t* off(int l, int t) const { return at<uint32_t>(lo.off[l]) + (size_t)t * B; }
   uint32_t* pool(int l) const { return at<uint32_t>(lo.pool[l]); }
@@ -275,6 +288,13 @@ struct Exec {
     f.rec_pool = pool(l); f.rec_off = off(l, t - 1); f.rec_cap = lo.cap[l];
     f.counts = (gen && l == L) ? at<uint32_t>(lo.counts) : nullptr;
     f.write_ff_list = l == 1;
+    if (graded()) {
+      f.ff_val_src = l == 1 ? in_dense(t) : act(l - 1, t & 1);
+      f.rec_val_src = act(l, (t - 1) & 1);
+      f.act_out = act(l, t & 1);
+      f.ff_vals = vals(l - 1); f.rec_vals = vals(l);
+      f.ff_pref = pref(l - 1, t); f.rec_pref = pref(l, t - 1);
+    }
   }
 
   dim3 fwd_grid() const {
@@ -284,8 +304,13 @@ struct Exec {
   }
 
   snn_status launch_fwd(const FwdParams& p, bool gen) {
-    if (gen) fwd_step_kernel<true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
-    else fwd_step_kernel<false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+    if (graded()) {
+      if (gen) fwd_step_kernel<true, true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+      else fwd_step_kernel<false, true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+    } else {
+      if (gen) fwd_step_kernel<true, false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+      else fwd_step_kernel<false, false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
+    }
     ++launches;
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
@@ -321,6 +346,7 @@ struct Exec {
       FwdLayer& f = p.lay[l - 1];
       f.mode = 2; f.N = net->sizes[l]; f.W = lo.words[l];
       f.rec_mask = mask(l, T); f.rec_pool = pool(l); f.rec_off = off(l, T); f.rec_cap = lo.cap[l];
+      if (graded()) { f.rec_val_src = act(l, T & 1); f.rec_vals = vals(l); f.rec_pref = pref(l, T); }
     }
     return launch_fwd(p, true);
   }
@@ -330,7 +356,8 @@ struct Exec {
     const uint32_t* counts = at<uint32_t>(lo.counts);
     const int32_t* targets = (a->flags & SNN_FLAG_INPUT_ON_HOST) ? at<int32_t>(lo.tg_stage) : a->targets;
     const int span = begin_span(SNN_PHASE_READOUT);
-    readout_logits_kernel<<<B, 256, 8 * N_out * sizeof(float), main>>>(counts, a->W_out, N_L, N_out, net->scale,
+    const int cf = graded() ? 1 : 0;
+    readout_logits_kernel<<<B, 256, 8 * N_out * sizeof(float), main>>>(counts, cf, a->W_out, N_L, N_out, net->scale,
                                                                        at<float>(lo.logits));
     softmax_loss_kernel<<<1, 256, B * sizeof(float), main>>>(at<float>(lo.logits), targets, B, N_out,
                                                              at<float>(lo.dlogits), at<float>(lo.status) + 1);
@@ -339,7 +366,7 @@ struct Exec {
       readout_gout_kernel<<<(unsigned)(((size_t)B * N_L + 255) / 256), 256, 0, main>>>(
           a->W_out, at<float>(lo.dlogits), B, N_L, N_out, net->scale, at<float>(lo.g_out));
       readout_dwout_kernel<<<(unsigned)(((size_t)N_L * N_out + 255) / 256), 256, 0, main>>>(
-          counts, at<float>(lo.dlogits), B, N_L, N_out, net->scale, a->dW_out);
+          counts, cf, at<float>(lo.dlogits), B, N_L, N_out, net->scale, a->dW_out);
       launches += 2;
     }
     end_span(span);
@@ -352,8 +379,9 @@ struct Exec {
     const int pairs = d.n_steps * d.B;
     d.window = std::min(DW_WINDOW, (pairs + 31) / 32 * 32);
     const size_t smem = (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4) +
-                        (size_t)(DW_ROWS + 1) * d.window * sizeof(uint32_t);
-    dw_kernel<U><<<grid, 32 * DW_ROWS, smem, main>>>(d);
+                        (size_t)(2 * DW_ROWS + 1) * d.window * sizeof(uint32_t);
+    if (graded()) dw_kernel<U, true><<<grid, 32 * DW_ROWS, smem, main>>>(d);
+    else dw_kernel<U, false><<<grid, 32 * DW_ROWS, smem, main>>>(d);
     ++launches;
   }
   template <int BT, int WB> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
@@ -426,9 +454,12 @@ struct Exec {
       d.slot_stride = lo.state_bytes / 4;
       d.dW = a->dW_ff[l - 1]; d.N_pre = sz[l - 1]; d.Wm = lo.words[l - 1];
       d.mask_row0 = l == 1 ? in_mask(op.t0 + 1) : mask(l - 1, op.t0 + 1);
+      d.off_row0 = nullptr; d.pref_row0 = nullptr; d.vals = nullptr; d.cap = 0;
+      if (graded()) { d.off_row0 = off(l - 1, op.t0 + 1); d.pref_row0 = pref(l - 1, op.t0 + 1); d.vals = vals(l - 1); d.cap = lo.cap[l - 1]; }
       run_dw(d);
       d.dW = a->dW_rec[l - 1]; d.N_pre = sz[l]; d.Wm = lo.words[l];
       d.mask_row0 = mask(l, op.t0);
+      if (graded()) { d.off_row0 = off(l, op.t0); d.pref_row0 = pref(l, op.t0); d.vals = vals(l); d.cap = lo.cap[l]; }
       run_dw(d);
     }
     end_span(span);
@@ -474,8 +505,10 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
         (reinterpret_cast<uintptr_t>(a->dW_ff[l]) | reinterpret_cast<uintptr_t>(a->dW_rec[l])) % 16 != 0)
       return fail(net, SNN_ERR_INVALID_ARG, "gradients must be 16-byte aligned");
   }
-  if (net->cell != SNN_CELL_LIF) return fail(net, SNN_ERR_UNSUPPORTED, "graded cell: not available in this build");
-  if (a->input_format != SNN_INPUT_BITS) return fail(net, SNN_ERR_UNSUPPORTED, "LIF cell takes bit-packed input");
+  if (net->cell == SNN_CELL_LIF && a->input_format != SNN_INPUT_BITS)
+    return fail(net, SNN_ERR_UNSUPPORTED, "the LIF cell takes bit-packed input (SNN_INPUT_BITS)");
+  if (net->cell == SNN_CELL_GRADED && a->input_format != SNN_INPUT_DENSE)
+    return fail(net, SNN_ERR_UNSUPPORTED, "the graded cell takes dense fp32 input (SNN_INPUT_DENSE)");
   if (!(a->max_activity > 0.f) || a->max_activity > 1.f) return fail(net, SNN_ERR_INVALID_ARG, "max_activity not in (0, 1]");
   if (reinterpret_cast<uintptr_t>(a->device_ws) % ALIGN != 0)
     return fail(net, SNN_ERR_INVALID_ARG, "device workspace must be 256-byte aligned");
@@ -512,15 +545,19 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
     if (!smem_opt_in) {
       const int dw1 = (int)(DW_ROWS * DW_STAGES * DW_GROUP * 1 * 32 * sizeof(float4));
-      const int dww = (int)((DW_ROWS + 1) * DW_WINDOW * sizeof(uint32_t));
+      const int dww = (int)((2 * DW_ROWS + 1) * DW_WINDOW * sizeof(uint32_t));
       auto bwd_smem = [](int bp) { return (int)(BWD_STAGES * (BWD_TM + bp) * 32 * sizeof(float4)); };
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(16)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(32)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
       smem_opt_in = true;
     }
   }
@@ -543,10 +580,19 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     }
   }
   if (a->flags & SNN_FLAG_INPUT_ON_HOST) {
-    CUDA_TRY(cudaMemcpyAsync(ex.ws + lo.in_stage, a->input, 4 * (size_t)T * B * lo.words[0], cudaMemcpyHostToDevice, ms));
+    CUDA_TRY(cudaMemcpyAsync(ex.ws + lo.in_stage, a->input,
+                             4 * (size_t)T * B * (net->cell == SNN_CELL_GRADED ? sz[0] : lo.words[0]),
+                             cudaMemcpyHostToDevice, ms));
     CUDA_TRY(cudaMemcpyAsync(ex.ws + lo.tg_stage, a->targets, 4 * (size_t)B, cudaMemcpyHostToDevice, ms));
   }
 
+  if (net->cell == SNN_CELL_GRADED) {   // spike words of the dense input, all steps at once
+    const size_t n_rows = (size_t)T * B, n_warps = n_rows * lo.words[0];
+    dense_to_words_kernel<<<(unsigned)((n_warps * 32 + 255) / 256), 256, 0, ms>>>(
+        reinterpret_cast<const float*>(ex.in_base()), n_rows, sz[0], lo.words[0], ex.at<uint32_t>(lo.in_words));
+    ++ex.launches;
+    CUDA_TRY(cudaGetLastError());
+  }
   int last_fwd = -1;
   for (int i = 0; i < (int)ops.size(); ++i)
     if (ops[i].kind == SNN_OP_FWD) last_fwd = i;
@@ -605,7 +651,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   net->ev_layout.assign(L + 1, snn_event_layout{});
   for (int l = 0; l <= L; ++l) {
     snn_event_layout& e = net->ev_layout[l];
-    e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = 0; e.pool_capacity = lo.cap[l];
+    e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = lo.vals[l]; e.pool_capacity = lo.cap[l];
     e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];
   }
   if (host_status[0] & STATUS_EVENT_OVERFLOW)

@@ -22,6 +22,7 @@ class Session:
             raise RuntimeError("a CUDA device is required: this library has no CPU path")
         self.sizes = [int(s) for s in sizes]
         self.L = len(self.sizes) - 2
+        self.cell = cell
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.net = sb.snn_create(self.sizes, tau_mem, threshold, surrogate, surrogate_beta, cell, readout_scale)
@@ -81,12 +82,15 @@ class Session:
     def train_step(self, input_bits, targets, strategy: int = sb.SNN_STANDARD, chunk_size: int = 0,
                    remote_chunk_size: int = 0, max_activity: float = 0.25, forward_only: bool = False,
                    keep_V: bool = False, time_phases: bool = False) -> float:
-        """input_bits: uint32 [T][B][ceil(N_0/32)] as a CUDA tensor (int32 storage) or a pinned host
-        tensor / numpy array (then it is copied to the device inside the call); targets alike."""
+        """input_bits: uint32 [T][B][ceil(N_0/32)] spike words (LIF cell; int32 storage) or float32
+        [T][B][N_0] dense values (graded cell), as a CUDA tensor or as a pinned host tensor / numpy
+        array (then it is copied to the device inside the call); targets alike."""
         on_host = not (isinstance(input_bits, torch.Tensor) and input_bits.is_cuda)
         if on_host:
             if not isinstance(input_bits, torch.Tensor):
-                input_bits = torch.from_numpy(np.ascontiguousarray(input_bits).view(np.int32)).pin_memory()
+                arr = np.ascontiguousarray(input_bits)
+                arr = arr.astype(np.float32, copy=False) if self.cell == sb.SNN_CELL_GRADED else arr.view(np.int32)
+                input_bits = torch.from_numpy(arr).pin_memory()
             if not isinstance(targets, torch.Tensor):
                 targets = torch.from_numpy(np.ascontiguousarray(targets, np.int32)).pin_memory()
         T, B = int(input_bits.shape[0]), int(input_bits.shape[1])
@@ -101,7 +105,8 @@ class Session:
             dbg = sb.ptr_array([t.data_ptr() for t in self.debug_V])
         a = sb.snn_step_args()
         a.T, a.B = T, B
-        a.input, a.input_format, a.targets = input_bits.data_ptr(), sb.SNN_INPUT_BITS, targets.data_ptr()
+        fmt = sb.SNN_INPUT_DENSE if self.cell == sb.SNN_CELL_GRADED else sb.SNN_INPUT_BITS
+        a.input, a.input_format, a.targets = input_bits.data_ptr(), fmt, targets.data_ptr()
         wff = sb.ptr_array([w.data_ptr() for w in self.W_ff]); wrec = sb.ptr_array([w.data_ptr() for w in self.W_rec])
         gff = sb.ptr_array([w.data_ptr() for w in self.dW_ff]); grec = sb.ptr_array([w.data_ptr() for w in self.dW_rec])
         a.W_ff, a.W_rec, a.W_out = wff, wrec, self.W_out.data_ptr()

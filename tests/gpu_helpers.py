@@ -23,7 +23,10 @@ def make_session(w, d):
     s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate_beta=w.beta, cell=w.cell,
                 readout_scale=w.scale())
     s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
-    bits = torch.from_numpy(d["input_bits"].view(np.int32)).to(s.device)
+    if w.cell == wl.CELL_GRADED:
+        bits = torch.from_numpy(d["input_dense"]).to(s.device)
+    else:
+        bits = torch.from_numpy(d["input_bits"].view(np.int32)).to(s.device)
     targets = torch.from_numpy(d["targets"]).to(s.device)
     return s, bits, targets
 

@@ -260,3 +260,95 @@ def test_errors_are_reported(orc32):
     loss = C.c_float()
     assert b.lib.snn_train_step(s.net, C.byref(a), C.byref(loss)) == b.SNN_ERR_WORKSPACE_TOO_SMALL
     s.close()
+
+
+# ---------------------------------------------------------------- graded (thresholded-ReLU) cell
+def _graded(**kw):
+    a = dict(cell=wl.CELL_GRADED, theta=0.3, g_ff=(1.2, 0.8), g_rec=(0.3, 0.3), p_in=0.3)
+    a.update(kw)
+    return wl.small(**a)
+
+
+def test_graded_forward_bit_exact(orc32):
+    w = _graded(sizes=(37, 640, 36, 7), T=11, B=3, seed=21)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d, do_backward=False)
+    frac = [float((x[1:] != 0).mean()) for x in ref["S"]]
+    assert all(0.05 < f < 0.8 for f in frac), frac
+    s, x, targets = make_session(w, d)
+    loss = s.train_step(x, targets, forward_only=True, keep_V=True, max_activity=1.0)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    for l in range(w.L):
+        V = s.debug_V[l].cpu().numpy()
+        assert np.array_equal(V[1:], ref["V"][l][1:])
+        assert np.array_equal(wl.unpack_bits(s.spike_words(l + 1), w.sizes[l + 1]), (ref["S"][l] != 0).astype(np.uint8))
+    # event lists with their values, input included
+    sb_ = sb()
+    dense = [d["input_dense"]] + [r[1:] for r in ref["S"]]
+    for layer in range(w.L + 1):
+        off, pool = s.events(layer)
+        e = sb_.snn_get_event_layout(s.net, layer)
+        vals = s.device_ws[e.values_off:e.values_off + 4 * w.B * e.pool_capacity].view(torch.float32).cpu().numpy()
+        vals = vals.reshape(w.B, e.pool_capacity)
+        for t in range(1, w.T + 1):
+            for b in range(w.B):
+                idx = np.flatnonzero(dense[layer][t - 1, b])
+                assert np.array_equal(pool[b, off[t, b]:off[t + 1, b]], idx)
+                assert np.array_equal(vals[b, off[t, b]:off[t + 1, b]], dense[layer][t - 1, b, idx])
+    s.close()
+
+
+def test_graded_gradients_and_strategies(orc32):
+    w = _graded(sizes=(37, 640, 132, 7), T=23, B=5, seed=22)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    s, x, targets = make_session(w, d)
+    loss = s.train_step(x, targets, strategy=0, max_activity=1.0)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 4, 0), (1, 1, 0), (2, 5, 0), (3, 2, 6), (3, 3, 3)]:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        assert s.train_step(x, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0) == loss
+        for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(a, b), (strat, K, R)
+    # host input path
+    assert s.train_step(d["input_dense"], d["targets"], strategy=3, chunk_size=2, remote_chunk_size=6,
+                        max_activity=1.0) == loss
+    for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+        assert np.array_equal(a, b)
+    s.close()
+
+
+def test_graded_with_unit_events_equals_lif_without_reset(orc32):
+    """Every input value 1 and a threshold no hidden neuron reaches: the graded kernels then do
+    exactly what the spiking kernels do on the same input words (no hidden event, no reset)."""
+    from dataclasses import replace
+    w = wl.small(sizes=(40, 260, 8), T=9, B=3, p_in=0.3, seed=23)
+    d = wl.make(w)
+    wl_lif = replace(w, theta=1e30)
+    s1, bits, targets = make_session(wl_lif, d)
+    s1.train_step(bits, targets, forward_only=True, keep_V=True, max_activity=1.0)
+    V_lif = s1.debug_V[0].cpu().numpy()
+    s1.close()
+    wg = replace(w, theta=1e30, cell=wl.CELL_GRADED)
+    dg = dict(d, input_dense=(d["input_dense"] != 0).astype(np.float32))
+    s2, x, targets = make_session(wg, dg)
+    s2.train_step(x, targets, forward_only=True, keep_V=True, max_activity=1.0)
+    assert np.array_equal(s2.debug_V[0].cpu().numpy(), V_lif)
+    s2.close()
+
+
+def test_cell_and_input_format_must_match():
+    b = sb()
+    w = wl.small()
+    d = wl.make(w)
+    from dataclasses import replace
+    s, x, targets = make_session(replace(w, cell=wl.CELL_GRADED), d)
+    a_bits = torch.from_numpy(d["input_bits"].view(np.int32)).cuda()
+    s.cell = b.SNN_CELL_LIF      # makes the session pass SNN_INPUT_BITS to a graded net
+    with pytest.raises(b.SnnError) as e:
+        s.train_step(a_bits, targets)
+    assert e.value.status == b.SNN_ERR_UNSUPPORTED
+    s.close()
