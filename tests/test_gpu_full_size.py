@@ -24,7 +24,7 @@ def _bits(tensors):
 def _check_prefix_spikes(s, w_full, ref, n_steps):
     for l in range(w_full.L):
         words = s.spike_words(l + 1)[:n_steps + 1]
-        assert np.array_equal(wl.unpack_bits(words, w_full.sizes[l + 1]), ref["S"][l][:n_steps + 1].astype(np.uint8))
+        assert np.array_equal(wl.unpack_bits(words, w_full.sizes[l + 1]), (ref["S"][l][:n_steps + 1] != 0).astype(np.uint8))
 
 
 def test_c2_whole_workload_against_oracle(orc32):
@@ -46,13 +46,13 @@ def test_c2_whole_workload_against_oracle(orc32):
     s.close()
 
 
-@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32)])
+@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32), ("c5", 60, 16, 32)])
 def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     w_full = wl.WORKLOADS[name]
     w = w_full.with_T(T_short)
     d = wl.make(w)
     ref = run_oracle(orc32, w, d)
-    assert all(0.01 < float(x[T_short // 2:].mean()) < 0.15 for x in ref["S"])
+    assert all(0.01 < float((x[T_short // 2:] != 0).mean()) < 0.2 for x in ref["S"])
     s, bits, targets = make_session(w, d)
     loss = s.train_step(bits, targets, strategy=w_full.strategy, chunk_size=K, remote_chunk_size=R)
     assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
@@ -61,12 +61,15 @@ def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     s.close()
 
 
-@pytest.mark.parametrize("name,T_prefix", [("c3", 60), ("c4", 12)])
+@pytest.mark.parametrize("name,T_prefix", [("c3", 60), ("c4", 12), ("c5", 40)])
 def test_full_length_properties(orc32, name, T_prefix):
     w = wl.WORKLOADS[name]
     d = wl.make(w, dense_input=False)
     # oracle forward on the first steps of the very same input (dense copy of the prefix only)
-    prefix = wl.unpack_bits(d["input_bits"][:T_prefix], w.sizes[0]).astype(np.float32)
+    if w.cell == wl.CELL_GRADED:
+        prefix = d["input_dense"][:T_prefix]
+    else:
+        prefix = wl.unpack_bits(d["input_bits"][:T_prefix], w.sizes[0]).astype(np.float32)
     dp = dict(d, input_dense=prefix)
     ref = run_oracle(orc32, w.with_T(T_prefix), dp, do_backward=False)
     s, bits, targets = make_session(w, d)
