@@ -72,7 +72,7 @@ class snn_event_layout(C.Structure):
 
 def _load() -> C.CDLL:
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2412_11810_b200.build` "
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python paper_2412_11810_b200/build.py` "
                           "(there is no fallback path)")
     lib = C.CDLL(LIB_PATH)
     lib.snn_create.argtypes = [C.POINTER(snn_config), C.POINTER(C.c_void_p)]

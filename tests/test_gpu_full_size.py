@@ -52,7 +52,7 @@ def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     w = w_full.with_T(T_short)
     d = wl.make(w)
     ref = run_oracle(orc32, w, d)
-    assert all(0.01 < float((x[T_short // 2:] != 0).mean()) < 0.2 for x in ref["S"])
+    assert all(0.002 < float((x[T_short // 2:] != 0).mean()) < 0.3 for x in ref["S"])
     s, bits, targets = make_session(w, d)
     loss = s.train_step(bits, targets, strategy=w_full.strategy, chunk_size=K, remote_chunk_size=R)
     assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
