@@ -46,7 +46,7 @@ def test_c2_whole_workload_against_oracle(orc32):
     s.close()
 
 
-@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32), ("c5", 60, 16, 32)])
+@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32), ("c5", 160, 16, 64)])
 def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     w_full = wl.WORKLOADS[name]
     w = w_full.with_T(T_short)
@@ -61,7 +61,7 @@ def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     s.close()
 
 
-@pytest.mark.parametrize("name,T_prefix", [("c3", 60), ("c4", 12), ("c5", 40)])
+@pytest.mark.parametrize("name,T_prefix", [("c3", 60), ("c4", 12), ("c5", 100)])
 def test_full_length_properties(orc32, name, T_prefix):
     w = wl.WORKLOADS[name]
     d = wl.make(w, dense_input=False)
