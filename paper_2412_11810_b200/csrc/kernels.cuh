@@ -44,6 +44,12 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// Programmatic dependent launch: every step kernel lets the next launch of the stream start early
+// (its CTAs become resident and run their prologue while this grid drains) and waits for the
+// previous grid to have completed, with its writes visible, before it touches global memory.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 constexpr uint32_t REC_TAG = 0x80000000u;  // list entry names a row of W_rec (else of W_ff)
 
 // A row of spike words made of two parts that is addressed as one: the feed-forward source
@@ -244,6 +250,7 @@ constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREAD
 
 template <bool GEN, bool GRADED>
 __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_constant__ FwdParams p) {
+  pdl_launch_dependents();
   const FwdLayer& L = p.lay[blockIdx.z];
   if (L.mode == 0) return;
   const int col0 = blockIdx.x * FWD_COLS;
@@ -260,6 +267,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   const bool step = L.mode == 1;
   if (!step && !(GEN && tile0)) return;
 
+  pdl_wait();
   // issue the loads the epilogue needs before anything else
   float4 vp = make_float4(0.f, 0.f, 0.f, 0.f);
   uint32_t pw = 0;
@@ -506,6 +514,7 @@ template <int BT, int WB>
 __global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
   constexpr int NT = 32 * BWD_WR * WB, NV = BWD_RT * BT, VPL = NV / 32, NWARP = BWD_WR * WB, BP = BT * WB;
   constexpr int STAGE_F4 = (BWD_TM + BP) * 32;      // float4 per stage: 32 weight rows + BP delta rows, 128 k each
+  pdl_launch_dependents();
   cg::cluster_group cluster = cg::this_cluster();
   const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const BwdLayer& L = p.lay[blockIdx.z];
@@ -531,6 +540,7 @@ __global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_ke
     else { W = L.W_rec; d = L.d_next; ld = L.N; k0 = lo_rec + (it - it_ff) * 128; hi = hi_rec; }
   };
 
+  pdl_wait();
   for (int bp0 = 0; bp0 < p.B; bp0 += BP) {
     auto issue = [&](int it) {
       if (it < it_all) {
@@ -616,9 +626,7 @@ struct DwArgs {
   float* dW;                 // [N_pre][N]
   const uint32_t* mask_row0; // spike words of the presynaptic layer for t = t0+1: [(t-t0-1)][B][Wm]
   const float* delta0;       // delta of step t0+1: delta(t, b) = delta0 + (t-t0-1) * slot_stride + b * N
-  size_t slot_stride;        // floats between consecutive steps
-  int N_pre, N, Wm, B, n_steps;
-  int window;                // (t, b) pairs compacted at a time: min(n_steps * B rounded up to 32, DW_WINDOW)
+  int N_pre, N, Wm;
   // graded cell only: where the value of an event is found (same step indexing as mask_row0)
   const uint32_t* off_row0;  // list offsets of the presynaptic layer [(t-t0-1)][B]
   const uint16_t* pref_row0; // events before each spike word [(t-t0-1)][B][Wm]
@@ -626,22 +634,43 @@ struct DwArgs {
   size_t cap;
 };
 
+// All weight matrices of a segment in one launch: blockIdx.z selects the matrix.
+struct DwParams {
+  DwArgs m[2 * MAXL];
+  size_t slot_stride;        // floats between consecutive steps (multiple of 4)
+  int B, n_steps;
+  int window;                // (t, b) pairs compacted at a time: min(n_steps * B rounded up to 32, DW_WINDOW)
+};
+
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
 constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
 constexpr int DW_GROUP = 4;       // delta rows per copy group
 constexpr int DW_STAGES = 2;      // copy groups in flight per warp
 
+// shared memory of dw_kernel in bytes for a window of `window` pairs
+template <int U, bool GRADED> constexpr size_t dw_smem_bytes(int window) {
+  return (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4) +
+         (size_t)window * sizeof(uint32_t) * (2 + DW_ROWS + (GRADED ? 1 + DW_ROWS : 0));
+}
+
 template <int U, bool GRADED>
-__global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
-  // dynamic shared memory: copy ring [DW_ROWS][DW_STAGES][DW_GROUP][U][32] float4, then the spike
-  // words of one window [window] and the per-row lists of active pairs [DW_ROWS][window]
+__global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const __grid_constant__ DwParams p) {
+  pdl_launch_dependents();
+  const DwArgs& a = p.m[blockIdx.z];
+  if ((int)blockIdx.y * DW_ROWS >= a.N_pre || (int)blockIdx.x * 128 * U >= a.N) return;
+  pdl_wait();
+  // dynamic shared memory: copy ring [DW_ROWS][DW_STAGES][DW_GROUP][U][32] float4; then, per window,
+  // the spike words [window], the position of each pair's delta row in units of 16 bytes [window],
+  // and per row the list of those positions for the pairs in which the row fired [DW_ROWS][window];
+  // graded cell: also each pair's (step, sample) row index and per row the event values
   extern __shared__ float4 s_ring[];
-  const int window = a.window;
-  uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_ring + (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32);
-  uint32_t* const s_evw = s_words + window + (size_t)(threadIdx.x >> 5) * window;   // this warp's list
-  float* const s_valw = reinterpret_cast<float*>(s_words + (size_t)(DW_ROWS + 1) * window) +
-                        (size_t)(threadIdx.x >> 5) * window;                         // and its values (graded)
+  const int window = p.window, B = p.B, n_steps = p.n_steps;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_ring + (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32);
+  uint32_t* const s_off = s_words + window;
+  uint32_t* const s_evw = s_off + window + (size_t)warp * window;
+  uint32_t* const s_rowi = s_off + (size_t)(1 + DW_ROWS) * window;            // graded only
+  float* const s_valw = reinterpret_cast<float*>(s_rowi + window) + (size_t)warp * window;
   const int row = blockIdx.y * DW_ROWS + warp;
   const int wc = (blockIdx.y * DW_ROWS) >> 5;               // spike word column of these rows
   const int bit = ((blockIdx.y * DW_ROWS) & 31) + warp;     // this row's bit in it
@@ -654,32 +683,35 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
     acc[u] = (row_ok && c < a.N) ? *reinterpret_cast<const float4*>(a.dW + (size_t)row * a.N + c)
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  float4* const ring = s_ring + (size_t)(threadIdx.x >> 5) * DW_STAGES * DW_GROUP * U * 32 + lane;
-  const int n_pairs = a.n_steps * a.B;
+  float4* const ring = s_ring + (size_t)warp * DW_STAGES * DW_GROUP * U * 32 + lane;
+  const float4* const delta_c = reinterpret_cast<const float4*>(a.delta0 + colb);
+  const uint32_t stride16 = (uint32_t)(p.slot_stride / 4), n16 = (uint32_t)(a.N / 4);
+  const int n_pairs = n_steps * B;
   for (int p0 = 0; p0 < n_pairs; p0 += window) {
     const int lim = n_pairs - p0 < window ? n_pairs - p0 : window;
     __syncthreads();
     for (int i = threadIdx.x; i < lim; i += 32 * DW_ROWS) {
       const int pr = p0 + i;
-      const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;   // ts = t - t0 - 1, t descending
-      s_words[i] = a.mask_row0[((size_t)ts * a.B + b) * a.Wm + wc];
+      const int ts = n_steps - 1 - pr / B, b = pr % B;      // ts = t - t0 - 1; pairs run t descending, b ascending
+      const size_t rowi = (size_t)ts * B + b;
+      s_words[i] = a.mask_row0[rowi * a.Wm + wc];
+      s_off[i] = (uint32_t)ts * stride16 + (uint32_t)b * n16;
+      if (GRADED) s_rowi[i] = (uint32_t)rowi;
     }
     __syncthreads();
-    // this warp's row: ascending list of the window's pairs in which it was active
+    // this warp's row: the window's pairs in which it fired, in pair order
     int n_ev = 0;
     for (int sb = 0; sb < lim; sb += 32) {
-      const bool on = sb + lane < lim && ((s_words[sb + lane] >> bit) & 1u);
+      const uint32_t wd = sb + lane < lim ? s_words[sb + lane] : 0u;
+      const bool on = (wd >> bit) & 1u;
       const uint32_t m = __ballot_sync(0xffffffffu, on);
       if (on) {
         const int slot = n_ev + __popc(m & ((1u << lane) - 1u));
-        const int pr = p0 + sb + lane;
-        s_evw[slot] = (uint32_t)pr;
+        s_evw[slot] = s_off[sb + lane];
         if (GRADED) {   // the event's value: list start + events before its word + events before it in the word
-          const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
-          const size_t rowi = (size_t)ts * a.B + b;
-          const uint32_t pos = a.off_row0[rowi] + a.pref_row0[rowi * a.Wm + wc] +
-                               __popc(s_words[sb + lane] & ((1u << bit) - 1u));
-          s_valw[slot] = pos < a.cap ? a.vals[(size_t)b * a.cap + pos] : 0.f;
+          const size_t rowi = s_rowi[sb + lane];
+          const uint32_t pos = a.off_row0[rowi] + a.pref_row0[rowi * a.Wm + wc] + __popc(wd & ((1u << bit) - 1u));
+          s_valw[slot] = pos < a.cap ? a.vals[(rowi % B) * a.cap + pos] : 0.f;
         }
       }
       n_ev += __popc(m);
@@ -694,12 +726,10 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const DwArgs a) {
           for (int q = 0; q < DW_GROUP; ++q) {
             const int e = g * DW_GROUP + q;
             if (e < n_ev) {
-              const int pr = (int)s_evw[e];
-              const int ts = a.n_steps - 1 - pr / a.B, b = pr % a.B;
-              const float* d = a.delta0 + (size_t)ts * a.slot_stride + (size_t)b * a.N + colb;
+              const float4* d = delta_c + s_evw[e];
 #pragma unroll
               for (int u = 0; u < U; ++u)
-                if (colb + u * 128 < a.N) cp_async16(ring + (((g % DW_STAGES) * DW_GROUP + q) * U + u) * 32, d + u * 128);
+                if (colb + u * 128 < a.N) cp_async16(ring + (((g % DW_STAGES) * DW_GROUP + q) * U + u) * 32, d + u * 32);
             }
           }
         }

@@ -297,6 +297,26 @@ struct Exec {
     }
   }
 
+  // Launch with programmatic stream serialization (the kernels call griddepcontrol.wait before they
+  // touch global memory), optionally as thread-block clusters of cluster_x CTAs along x.
+  template <class P> cudaError_t launch_pdl(void (*kernel)(P), dim3 grid, dim3 block, size_t smem, const P& params,
+                                            int cluster_x = 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cudaLaunchAttribute at[2];
+    int n = 0;
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 0) {
+      at[n].id = cudaLaunchAttributeClusterDimension;
+      at[n].val.clusterDim.x = cluster_x; at[n].val.clusterDim.y = 1; at[n].val.clusterDim.z = 1;
+      ++n;
+    }
+    cfg.attrs = at; cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, params);
+  }
+
   dim3 fwd_grid() const {
     int maxN = 0;
     for (int l = 1; l <= L; ++l) maxN = std::max(maxN, net->sizes[l]);
@@ -304,13 +324,9 @@ struct Exec {
   }
 
   snn_status launch_fwd(const FwdParams& p, bool gen) {
-    if (graded()) {
-      if (gen) fwd_step_kernel<true, true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
-      else fwd_step_kernel<false, true><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
-    } else {
-      if (gen) fwd_step_kernel<true, false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
-      else fwd_step_kernel<false, false><<<fwd_grid(), FWD_THREADS, FWD_DYN_SMEM, main>>>(p);
-    }
+    void (*k)(FwdParams) = graded() ? (gen ? fwd_step_kernel<true, true> : fwd_step_kernel<false, true>)
+                                    : (gen ? fwd_step_kernel<true, false> : fwd_step_kernel<false, false>);
+    CUDA_TRY(launch_pdl(k, fwd_grid(), dim3(FWD_THREADS), FWD_DYN_SMEM, p));
     ++launches;
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
@@ -374,31 +390,17 @@ struct Exec {
     return SNN_OK;
   }
 
-  template <int U> void launch_dw(DwArgs d) {
-    dim3 grid((d.N + 128 * U - 1) / (128 * U), (d.N_pre + DW_ROWS - 1) / DW_ROWS);
+  template <int U> void launch_dw(DwParams& d, int maxN, int maxNpre) {
+    dim3 grid((maxN + 128 * U - 1) / (128 * U), (maxNpre + DW_ROWS - 1) / DW_ROWS, 2 * L);
     const int pairs = d.n_steps * d.B;
     d.window = std::min(DW_WINDOW, (pairs + 31) / 32 * 32);
-    const size_t smem = (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4) +
-                        (size_t)(2 * DW_ROWS + 1) * d.window * sizeof(uint32_t);
-    if (graded()) dw_kernel<U, true><<<grid, 32 * DW_ROWS, smem, main>>>(d);
-    else dw_kernel<U, false><<<grid, 32 * DW_ROWS, smem, main>>>(d);
+    if (graded()) launch_pdl(dw_kernel<U, true>, grid, dim3(32 * DW_ROWS), dw_smem_bytes<U, true>(d.window), d);
+    else launch_pdl(dw_kernel<U, false>, grid, dim3(32 * DW_ROWS), dw_smem_bytes<U, false>(d.window), d);
     ++launches;
   }
   template <int BT, int WB> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(tiles * CS, 1, L);
-    cfg.blockDim = dim3(32 * BWD_WR * WB);
-    cfg.stream = main;
-    cfg.dynamicSmemBytes = (size_t)BWD_STAGES * (BWD_TM + BT * WB) * 32 * sizeof(float4);
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, bwd_step_kernel<BT, WB>, p);
-  }
-  void run_dw(const DwArgs& d) {
-    if (d.N >= 512) launch_dw<2>(d);
-    else launch_dw<1>(d);
+    return launch_pdl(bwd_step_kernel<BT, WB>, dim3(tiles * CS, 1, L), dim3(32 * BWD_WR * WB),
+                      (size_t)BWD_STAGES * (BWD_TM + BT * WB) * 32 * sizeof(float4), p, CS);
   }
 
   // BWD: layer wavefront, layer l runs L-l steps behind the last layer; then the weight
@@ -447,20 +449,33 @@ struct Exec {
     carry_cur ^= 1;
     end_span(span);
     span = begin_span(SNN_PHASE_DW);
-    for (int l = 1; l <= L; ++l) {
-      DwArgs d;
-      d.B = B; d.n_steps = n; d.N = sz[l];
-      d.delta0 = slot(op.buf_slot, l);
-      d.slot_stride = lo.state_bytes / 4;
-      d.dW = a->dW_ff[l - 1]; d.N_pre = sz[l - 1]; d.Wm = lo.words[l - 1];
-      d.mask_row0 = l == 1 ? in_mask(op.t0 + 1) : mask(l - 1, op.t0 + 1);
-      d.off_row0 = nullptr; d.pref_row0 = nullptr; d.vals = nullptr; d.cap = 0;
-      if (graded()) { d.off_row0 = off(l - 1, op.t0 + 1); d.pref_row0 = pref(l - 1, op.t0 + 1); d.vals = vals(l - 1); d.cap = lo.cap[l - 1]; }
-      run_dw(d);
-      d.dW = a->dW_rec[l - 1]; d.N_pre = sz[l]; d.Wm = lo.words[l];
-      d.mask_row0 = mask(l, op.t0);
-      if (graded()) { d.off_row0 = off(l, op.t0); d.pref_row0 = pref(l, op.t0); d.vals = vals(l); d.cap = lo.cap[l]; }
-      run_dw(d);
+    // All 2L weight gradients of the segment in one launch.  Row positions are kept in units of 16 bytes in
+    // 32 bits, so a very long segment (STANDARD) is cut into runs of steps, latest steps first: the order of
+    // additions per element (t descending, b ascending) is unchanged.
+    const size_t stride16 = lo.state_bytes / 16;
+    const int max_run = (int)std::min<size_t>((size_t)n, (0xffffffffull - (size_t)B * maxN / 4) / stride16);
+    int maxNpre = sz[0];
+    for (int l = 1; l <= L; ++l) maxNpre = std::max(maxNpre, sz[l]);
+    for (int hi = n; hi > 0; hi -= max_run) {
+      const int lo_s = std::max(0, hi - max_run);   // steps t0+lo_s+1 .. t0+hi
+      const int ta = op.t0 + lo_s;
+      DwParams d;
+      std::memset(&d, 0, sizeof d);
+      d.B = B; d.n_steps = hi - lo_s; d.slot_stride = lo.state_bytes / 4;
+      for (int l = 1; l <= L; ++l) {
+        DwArgs& f = d.m[2 * (l - 1)];
+        f.N = sz[l]; f.delta0 = slot(op.buf_slot + lo_s, l);
+        f.dW = a->dW_ff[l - 1]; f.N_pre = sz[l - 1]; f.Wm = lo.words[l - 1];
+        f.mask_row0 = l == 1 ? in_mask(ta + 1) : mask(l - 1, ta + 1);
+        if (graded()) { f.off_row0 = off(l - 1, ta + 1); f.pref_row0 = pref(l - 1, ta + 1); f.vals = vals(l - 1); f.cap = lo.cap[l - 1]; }
+        DwArgs& r = d.m[2 * (l - 1) + 1];
+        r.N = sz[l]; r.delta0 = f.delta0;
+        r.dW = a->dW_rec[l - 1]; r.N_pre = sz[l]; r.Wm = lo.words[l];
+        r.mask_row0 = mask(l, ta);
+        if (graded()) { r.off_row0 = off(l, ta); r.pref_row0 = pref(l, ta); r.vals = vals(l); r.cap = lo.cap[l]; }
+      }
+      if (maxN >= 4096) launch_dw<2>(d, maxN, maxNpre);
+      else launch_dw<1>(d, maxN, maxNpre);
     }
     end_span(span);
     CUDA_TRY(cudaGetLastError());
@@ -544,8 +559,6 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   {
     static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
     if (!smem_opt_in) {
-      const int dw1 = (int)(DW_ROWS * DW_STAGES * DW_GROUP * 1 * 32 * sizeof(float4));
-      const int dww = (int)((2 * DW_ROWS + 1) * DW_WINDOW * sizeof(uint32_t));
       auto bwd_smem = [](int bp) { return (int)(BWD_STAGES * (BWD_TM + bp) * 32 * sizeof(float4)); };
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
@@ -554,10 +567,10 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(16)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(32)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dw1 + dww));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * dw1 + dww));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, true>(DW_WINDOW)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, true>(DW_WINDOW)));
       smem_opt_in = true;
     }
   }

@@ -70,8 +70,8 @@ WORKLOADS: Dict[str, Workload] = {
     "c4": Workload("c4", (1024, 8192, 8192, 8192, 100), T=2000, B=8, p_in=0.02, seed=3, strategy=DOUBLE,
                    chunk_size=16, remote_chunk_size=256, g_ff=(2.9, 1.36, 1.32), g_rec=(1.0, 1.0, 1.0)),
     "c5": Workload("c5", (1024, 4096, 4096, 50), T=4096, B=16, p_in=0.10, seed=4, strategy=DOUBLE,
-                   chunk_size=16, remote_chunk_size=256, cell=CELL_GRADED, g_ff=(0.38, 0.16),
-                   g_rec=(0.2, 0.2)),
+                   chunk_size=16, remote_chunk_size=256, cell=CELL_GRADED, g_ff=(0.703, 0.113),
+                   g_rec=(0.05, 0.05)),
 }
 
 

@@ -46,15 +46,21 @@ def test_c2_whole_workload_against_oracle(orc32):
     s.close()
 
 
-@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32), ("c5", 160, 16, 64)])
+@pytest.mark.parametrize("name,T_short,K,R", [("c3", 300, 64, 0), ("c4", 40, 16, 32), ("c5", 100, 16, 64)])
 def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     w_full = wl.WORKLOADS[name]
+    if name == "c5":
+        # the graded workload needs hundreds of steps to reach its stationary activity; for a short
+        # sequence the feed-forward gains are raised so that both layers are busy from the start
+        from dataclasses import replace
+        w_full = replace(w_full, g_ff=(1.0, 0.5))
     w = w_full.with_T(T_short)
     d = wl.make(w)
     ref = run_oracle(orc32, w, d)
-    assert all(0.002 < float((x[T_short // 2:] != 0).mean()) < 0.3 for x in ref["S"])
+    assert all(0.01 < float((x[T_short // 2:] != 0).mean()) < 0.6 for x in ref["S"])
     s, bits, targets = make_session(w, d)
-    loss = s.train_step(bits, targets, strategy=w_full.strategy, chunk_size=K, remote_chunk_size=R)
+    loss = s.train_step(bits, targets, strategy=w_full.strategy, chunk_size=K, remote_chunk_size=R,
+                        max_activity=0.6 if name == "c5" else 0.25)
     assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
     _check_prefix_spikes(s, w, ref, T_short)
     assert_grads_close(s.gradients(), ref)
