@@ -286,6 +286,13 @@ def run_ours(args, rank, world):
             "gpu_launches": int(stats.kernel_launches) * args.steps,
             "roofline": roof,
             "phases_ms": {k: v[0] for k, v in ph.items()}, "phase_launches": {k: v[1] for k, v in ph.items()},
+            "host_link": None if not stats.d2h_copies else {
+                "bytes_per_copy": int(stats.state_bytes), "d2h_copies": int(stats.d2h_copies),
+                "h2d_copies": int(stats.h2d_copies),
+                "d2h_gbs": stats.state_bytes * stats.d2h_copies / (ph["d2h"][0] / 1e3) / 1e9 if ph["d2h"][0] > 0 else None,
+                "h2d_gbs": stats.state_bytes * stats.h2d_copies / (ph["h2d"][0] / 1e3) / 1e9 if ph["h2d"][0] > 0 else None,
+                "copy_ms_per_step": ph["d2h"][0] + ph["h2d"][0],
+                "note": "CUDA events on the side stream around every checkpoint copy; copies overlap the passes"},
             "peak_memory": {"device_bytes": dev_peak, "pinned_bytes": pin_peak,
                             "local_state_slots": stats.local_state_slots, "state_bytes": stats.state_bytes,
                             "event_bytes": stats.event_bytes},

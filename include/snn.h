@@ -178,9 +178,11 @@ snn_status snn_memory_stats_get(const snn_net* net, snn_memory_stats* out);
 
 /* Device time of the last step per pass of Fig. 1, measured with CUDA events on the main stream
  * when the step ran with SNN_FLAG_TIME_PHASES, and the kernels launched in each.  BWD is the
- * surrogate-gradient step kernel, DW the sparse outer-product weight-gradient kernel. */
+ * surrogate-gradient step kernel, DW the sparse outer-product weight-gradient kernel; D2H and H2D are the
+ * checkpoint copies, timed on the side stream (their `launches` count copies; they overlap the passes). */
 typedef enum { SNN_PHASE_FWD = 0, SNN_PHASE_REFWD1 = 1, SNN_PHASE_REFWD2 = 2, SNN_PHASE_BWD = 3,
-               SNN_PHASE_DW = 4, SNN_PHASE_READOUT = 5, SNN_N_PHASES = 6 } snn_phase;
+               SNN_PHASE_DW = 4, SNN_PHASE_READOUT = 5, SNN_PHASE_D2H = 6, SNN_PHASE_H2D = 7,
+               SNN_N_PHASES = 8 } snn_phase;
 typedef struct {
   float ms[SNN_N_PHASES];
   int32_t launches[SNN_N_PHASES];

@@ -120,6 +120,28 @@ __device__ void fill_chunk_from_words(const WordPair& wp, const uint32_t* s_pref
   }
 }
 
+// Step 2a for the gather: instead of the indices, the address of each listed weight row (at the
+// CTA's first column) goes to shared memory, so that issuing a row copy is one load and one add.
+template <int NT>
+__device__ void fill_rows_from_words(const WordPair& wp, const uint32_t* s_pref, uint32_t c0,
+                                     const float* Wa_tile, const float* Wb_tile, int N, const float** s_row) {
+  const int n_words = wp.size();
+  for (int w = threadIdx.x; w < n_words; w += NT) {
+    uint32_t bits = wp.get(w);
+    if (!bits) continue;
+    uint32_t p = s_pref[w];
+    if (p >= c0 + LIST_CHUNK || p + __popc(bits) <= c0) continue;
+    const bool in_a = w < wp.n_a;
+    const float* base = (in_a ? Wa_tile : Wb_tile) + (size_t)((in_a ? w : w - wp.n_a) * 32) * N;
+    while (bits) {
+      const int bit = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (p >= c0 && p < c0 + LIST_CHUNK) s_row[p - c0] = base + (size_t)bit * N;
+      ++p;
+    }
+  }
+}
+
 // Step 2b: the lists to global memory (entries past the room left in a pool are dropped).
 // Part a goes to dst_a (if not null), part b to dst_b; n_a_bits = set bits of part a.
 // Graded events also store their value (read from the dense source rows val_a / val_b) and, per
@@ -257,7 +279,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   if (col0 >= L.N) return;
   const int b = blockIdx.y, B = p.B;
   const bool tile0 = blockIdx.x == 0;
-  __shared__ uint32_t s_list[LIST_CHUNK];
+  __shared__ const float* s_row[LIST_CHUNK];   // addresses of the listed weight rows at this CTA's first column
   __shared__ uint32_t s_pref[GEN ? 2 * MAX_WORDS + 1 : 1];
   __shared__ uint32_t s_warp[FWD_THREADS / 32];
   __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
@@ -315,19 +337,20 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
 
   // ---- gather-accumulate in list order
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  const float* const Wff_c = L.W_ff + col;
-  const float* const Wrec_c = L.W_rec + col;
+  const float* const Wff_tile = L.W_ff + col0;
+  const float* const Wrec_tile = L.W_rec + col0;
   for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
     const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
     if (GEN) {
-      fill_chunk_from_words<FWD_THREADS>(wp, s_pref, c0, s_list);
+      fill_rows_from_words<FWD_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
       if (GRADED)
         fill_values_from_words<FWD_THREADS>(wp, s_pref, c0, L.ff_val_src + (size_t)b * L.N_pre,
                                             L.rec_val_src + (size_t)b * L.N, s_val);
     } else {
       for (int i = threadIdx.x; i < n; i += FWD_THREADS) {
         const uint32_t q = c0 + i;
-        s_list[i] = q < n_ff ? ff_pool[s_ff + q] : (rec_pool[s_rec + (q - n_ff)] | REC_TAG);
+        s_row[i] = q < n_ff ? Wff_tile + (size_t)ff_pool[s_ff + q] * L.N
+                            : Wrec_tile + (size_t)rec_pool[s_rec + (q - n_ff)] * L.N;
         if (GRADED)
           s_val[i] = q < n_ff ? L.ff_vals[(size_t)b * L.ff_cap + s_ff + q]
                               : L.rec_vals[(size_t)b * L.rec_cap + s_rec + (q - n_ff)];
@@ -339,38 +362,44 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
       // the copies of the next groups are in flight while the oldest group is added, in list order
       float4* const ring = s_stage + threadIdx.x;
       const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
+      const int lane_col = threadIdx.x * 4;
       auto issue = [&](int g) {
         if (g < n_groups) {
           float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+          const float* const* rows = s_row + g * GATHER_ROWS;
+          if ((g + 1) * GATHER_ROWS <= n) {
 #pragma unroll
-          for (int u = 0; u < GATHER_ROWS; ++u) {
-            const int i = g * GATHER_ROWS + u;
-            if (i < n) {
-              const uint32_t v = s_list[i];
-              cp_async16(dst + u * FWD_THREADS, ((v & REC_TAG) ? Wrec_c : Wff_c) + (size_t)(v & ~REC_TAG) * L.N);
-            }
+            for (int u = 0; u < GATHER_ROWS; ++u) cp_async16(dst + u * FWD_THREADS, rows[u] + lane_col);
+          } else {
+#pragma unroll
+            for (int u = 0; u < GATHER_ROWS; ++u)
+              if (g * GATHER_ROWS + u < n) cp_async16(dst + u * FWD_THREADS, rows[u] + lane_col);
           }
         }
         cp_async_commit();
+      };
+      auto add_row = [&](const float4 w, int i) {
+        if (GRADED) {   // one fused multiply-add per event and neuron
+          const float sv = s_val[i];
+          acc.x = __fmaf_rn(sv, w.x, acc.x); acc.y = __fmaf_rn(sv, w.y, acc.y);
+          acc.z = __fmaf_rn(sv, w.z, acc.z); acc.w = __fmaf_rn(sv, w.w, acc.w);
+        } else {        // a binary spike: the fused multiply-add is an exact plain add
+          acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+          acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+        }
       };
       for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
       for (int g = 0; g < n_groups; ++g) {
         issue(g + GATHER_STAGES - 1);
         cp_async_wait<GATHER_STAGES - 1>();
         const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+        if ((g + 1) * GATHER_ROWS <= n) {
 #pragma unroll
-        for (int u = 0; u < GATHER_ROWS; ++u) {
-          if (g * GATHER_ROWS + u < n) {
-            const float4 w = src[u * FWD_THREADS];
-            if (GRADED) {   // one fused multiply-add per event and neuron
-              const float sv = s_val[g * GATHER_ROWS + u];
-              acc.x = __fmaf_rn(sv, w.x, acc.x); acc.y = __fmaf_rn(sv, w.y, acc.y);
-              acc.z = __fmaf_rn(sv, w.z, acc.z); acc.w = __fmaf_rn(sv, w.w, acc.w);
-            } else {        // a binary spike: the fused multiply-add is an exact plain add
-              acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
-              acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
-            }
-          }
+          for (int u = 0; u < GATHER_ROWS; ++u) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
+        } else {
+#pragma unroll
+          for (int u = 0; u < GATHER_ROWS; ++u)
+            if (g * GATHER_ROWS + u < n) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
         }
       }
       cp_async_wait<0>();

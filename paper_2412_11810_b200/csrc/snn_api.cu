@@ -214,23 +214,24 @@ struct Exec {
   int ev_used = 0;
 
   // Brackets [begin_span, end_span) on the main stream with two events of the net's pool.
-  int begin_span(int phase) {
+  int begin_span(int phase, cudaStream_t st = nullptr) {
     if (!timed) return -1;
+    if (!st) st = main;
     auto& pool_ev = net->timing_events;
     while ((int)pool_ev.size() < ev_used + 2) {
       cudaEvent_t e;
       if (cudaEventCreate(&e) != cudaSuccess) { timed = false; return -1; }
       pool_ev.push_back(e);
     }
-    cudaEventRecord(pool_ev[ev_used], main);
+    cudaEventRecord(pool_ev[ev_used], st);
     spans.push_back(Span{phase, ev_used, ev_used + 1, launches});
     ev_used += 2;
     return (int)spans.size() - 1;
   }
-  void end_span(int id) {
+  void end_span(int id, cudaStream_t st = nullptr) {
     if (id < 0) return;
-    cudaEventRecord(net->timing_events[spans[id].ev1], main);
-    spans[id].launches = launches - spans[id].launches;
+    cudaEventRecord(net->timing_events[spans[id].ev1], st ? st : main);
+    spans[id].launches = st ? 1 : launches - spans[id].launches;
   }
   void collect_spans() {
     net->phases = snn_phase_times{};
@@ -490,8 +491,10 @@ struct Exec {
     // the copy starts after everything issued so far on the main stream
     CUDA_TRY(cudaEventRecord(net->ev_main, main));
     CUDA_TRY(cudaStreamWaitEvent(side, net->ev_main, 0));
+    const int span = begin_span(to_host ? SNN_PHASE_D2H : SNN_PHASE_H2D, side);
     if (to_host) { CUDA_TRY(cudaMemcpyAsync(remote, local, lo.state_bytes, cudaMemcpyDeviceToHost, side)); ++d2h; }
     else { CUDA_TRY(cudaMemcpyAsync(local, remote, lo.state_bytes, cudaMemcpyHostToDevice, side)); ++h2d; }
+    end_span(span, side);
     CUDA_TRY(cudaEventRecord(net->ev_slot[s], side));
     slot_pending[s] = true;
     return SNN_OK;
