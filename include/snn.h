@@ -10,6 +10,10 @@
  *   REMOTE    the same schedule with the checkpoints in remote memory (Eqs. 6, 7)
  *   DOUBLE    remote checkpoints every remote_chunk_size steps, local ones every
  *             chunk_size steps recomputed by an extra pass (Eqs. 11-13)
+ *   HIERARCHICAL  checkpoints every chunk_size steps kept in remote memory and moved nb_local at a
+ *             time, the last nb_local staying local (section "Hierarchical Checkpointing", Eqs. 8-10)
+ *   DOUBLE_LOCAL  the schedule of DOUBLE with both tiers in device memory (Discussion: the purely
+ *             on-chip use of Double Checkpointing)
  * "Local" memory is device memory, "remote" memory is pinned host memory.
  *
  * General rules.  Every function returns an snn_status and never throws, aborts
@@ -43,7 +47,8 @@ typedef enum {
   SNN_ERR_UNSUPPORTED = 6
 } snn_status;
 
-typedef enum { SNN_STANDARD = 0, SNN_CHUNK = 1, SNN_REMOTE = 2, SNN_DOUBLE = 3 } snn_strategy;
+typedef enum { SNN_STANDARD = 0, SNN_CHUNK = 1, SNN_REMOTE = 2, SNN_DOUBLE = 3, SNN_HIERARCHICAL = 4,
+               SNN_DOUBLE_LOCAL = 5 } snn_strategy;
 typedef enum { SNN_CELL_LIF = 0, SNN_CELL_GRADED = 1 } snn_cell;
 typedef enum { SNN_SURR_FAST_SIGMOID = 0, SNN_SURR_SIGMOID = 1 } snn_surrogate;
 
@@ -82,15 +87,26 @@ void snn_destroy(snn_net* net);
 /* The leak alpha = exp(-1/tau_mem), evaluated in double and rounded once to fp32. */
 float snn_alpha(const snn_net* net);
 
-/* Checkpoint hyper-parameters (paper: chunk_size, Eq. 1; remote_chunk_size, Eq. 11).
- * STANDARD ignores both; CHUNK and REMOTE need chunk_size >= 1; DOUBLE needs
- * remote_chunk_size >= chunk_size >= 1 and remote_chunk_size % chunk_size == 0.
- * The sequence length need not be a multiple of either: the last segment is short. */
+/* Checkpoint hyper-parameters (paper: chunk_size, Eq. 1; remote_chunk_size, Eq. 11; nb_local, Eq. 8).
+ * STANDARD ignores all; CHUNK and REMOTE need chunk_size >= 1; DOUBLE and DOUBLE_LOCAL need
+ * remote_chunk_size >= chunk_size >= 1 and remote_chunk_size % chunk_size == 0; HIERARCHICAL needs
+ * chunk_size >= 1 and nb_local >= 1.
+ * The sequence length need not be a multiple of any of them: the last segment is short. */
 typedef struct {
   int32_t strategy; /* snn_strategy */
   int32_t chunk_size;
   int32_t remote_chunk_size;
+  int32_t nb_local;
 } snn_ckpt;
+
+/* Hyper-parameters by the rules of the paper's Hyperparameter Study: CHUNK chunk_size = sqrt(T);
+ * DOUBLE remote_chunk_size within 64 .. 256 (256 once T >= 1024, else the power of two nearest T/4,
+ * at least 4) and chunk_size = sqrt(remote_chunk_size); REMOTE the largest chunk_size whose device
+ * workspace fits device_budget_bytes (sqrt(T) if the budget is 0); HIERARCHICAL chunk_size =
+ * sqrt(T) and nb_local = sqrt(number of checkpoints).  Host only.  net, B and max_activity are
+ * used for the REMOTE rule only (net may be NULL otherwise). */
+snn_status snn_suggest_ckpt(const snn_net* net, int32_t T, int32_t B, int32_t strategy, size_t device_budget_bytes,
+                            float max_activity, snn_ckpt* out);
 
 /* Bytes of device and pinned-host workspace a train step of T steps and batch B needs.
  * max_activity in (0, 1]: upper bound on the mean fraction of active neurons per layer
@@ -198,7 +214,8 @@ const char* snn_last_error(const snn_net* net); /* owned by net; valid until the
  * (t-t0) % keep_every == 0, also to local slot keep_slot + (t-t0)/keep_every - 1.
  * FWD generates and stores the events; REFWD* replays the stored events.
  * BWD back-propagates t = t1 .. t0+1 with V_t in local slot buf_slot + (t-t0-1).
- * D2H copies local slot in_slot to remote slot remote_slot; H2D the reverse into keep_slot.
+ * D2H copies local slot in_slot to remote slot remote_slot; H2D the reverse into keep_slot; both move
+ * max(buf_len, 1) consecutive slots in one transfer.
  * ZERO clears local slot keep_slot (the initial state). */
 typedef enum { SNN_OP_FWD = 0, SNN_OP_REFWD1 = 1, SNN_OP_REFWD2 = 2, SNN_OP_BWD = 3,
                SNN_OP_D2H = 4, SNN_OP_H2D = 5, SNN_OP_ZERO = 6 } snn_op_kind;

@@ -18,7 +18,7 @@ import numpy as np
 
 from .oracle import NetSpec, Oracle
 
-STANDARD, CHUNK, REMOTE, DOUBLE = 0, 1, 2, 3
+STANDARD, CHUNK, REMOTE, DOUBLE, HIERARCHICAL = 0, 1, 2, 3, 4
 
 
 class _Tier:
@@ -103,7 +103,7 @@ class _Run:
 
 
 def bptt_checkpointed(orc: Oracle, spec: NetSpec, inp, targets, W_ff, W_rec, W_out, strategy: int,
-                      chunk_size: int = 0, remote_chunk_size: int = 0):
+                      chunk_size: int = 0, remote_chunk_size: int = 0, nb_local: int = 0):
     run = _Run(orc, spec, inp, targets, W_ff, W_rec, W_out)
     T = run.T
     local, remote = _Tier(), _Tier()
@@ -123,6 +123,8 @@ def bptt_checkpointed(orc: Oracle, spec: NetSpec, inp, targets, W_ff, W_rec, W_o
         return run.result(local, remote, 0)
 
     assert K >= 1
+    if strategy == HIERARCHICAL:
+        return _hierarchical(run, local, remote, K, nb_local)
     if strategy == DOUBLE:
         assert R >= K and R % K == 0
     # ---- forward pass: keep checkpoints only ------------------------------------------------
@@ -178,3 +180,59 @@ def bptt_checkpointed(orc: Oracle, spec: NetSpec, inp, targets, W_ff, W_rec, W_o
                 chunk_peak = max(chunk_peak, chunk_backward(t0, min(r1, t0 + K), local.get(t0)))
                 local.drop(t0)
     return run.result(local, remote, chunk_peak)
+
+
+def _hierarchical(run: _Run, local: _Tier, remote: _Tier, K: int, P: int):
+    """Section "Hierarchical Checkpointing": checkpoints every K steps live in remote memory and are
+    moved nb_local = P at a time, one communication per batch; the last batch of checkpoints is
+    stored locally and never moved.  Local memory: chunk_size + nb_local states (Eq. 9).  The paper's
+    Eq. 10 counts the communications as 2 (nb_checkpoints / nb_local - nb_local); the text explains
+    the subtracted term as the last batch that stays local, so it is read here as
+    2 (number of batches - 1), each communication moving one batch."""
+    assert P >= 1
+    T = run.T
+    n_ck = -(-T // K)
+    n_b = -(-n_ck // P)
+    comms = 0
+    V = run.zero_state()
+    batch = {}
+
+    def add_checkpoint(t, v):
+        nonlocal batch, comms
+        j = (t // K) // P
+        batch[t] = v
+        run.ckpts.append(("remote" if j < n_b - 1 else "local", t))
+        if len(batch) == P and j < n_b - 1:   # a complete batch that is not the last one leaves at once
+            for tt, vv in batch.items():
+                remote.put(tt, vv)
+            comms += 1
+            batch = {}
+
+    add_checkpoint(0, V)
+    for t in range(1, T + 1):
+        V = run.step(V, t, True); run.fwd_steps += 1
+        if t % K == 0 and t < T:
+            add_checkpoint(t, V)
+    run.trace.append(("forward", 0, T))
+    run.readout()
+    chunk_peak, local_peak = 0, len(batch)
+    for j in range(n_b - 1, -1, -1):
+        if j < n_b - 1:
+            batch = {c * K: remote.get(c * K) for c in range(j * P, (j + 1) * P)}
+            comms += 1
+        local_peak = max(local_peak, len(batch))
+        for c in range(min(n_ck, (j + 1) * P) - 1, j * P - 1, -1):
+            t0, t1 = c * K, min(T, c * K + K)
+            buf, Vt = {}, batch[t0]
+            for t in range(t0 + 1, t1 + 1):
+                Vt = run.step(Vt, t, False); run.refwd_steps[0] += 1
+                buf[t] = Vt
+            run.trace.append(("reforward1", t0, t1))
+            for t in range(t1, t0, -1):
+                run.backward(buf[t], t)
+            run.trace.append(("backward", t1, t0))
+            chunk_peak = max(chunk_peak, len(buf))
+    res = run.result(local, remote, chunk_peak)
+    res["stats"]["local_states_peak"] = local_peak + chunk_peak
+    res["stats"]["transfers"] = comms
+    return res

@@ -15,18 +15,19 @@ LIB_PATH = os.path.join(HERE, "libsnnckpt.so")
 
 SNN_OK, SNN_ERR_INVALID_ARG, SNN_ERR_WORKSPACE_TOO_SMALL, SNN_ERR_EVENT_OVERFLOW = 0, 1, 2, 3
 SNN_ERR_DEVICE_TIMEOUT, SNN_ERR_CUDA, SNN_ERR_UNSUPPORTED = 4, 5, 6
-SNN_STANDARD, SNN_CHUNK, SNN_REMOTE, SNN_DOUBLE = 0, 1, 2, 3
+SNN_STANDARD, SNN_CHUNK, SNN_REMOTE, SNN_DOUBLE, SNN_HIERARCHICAL, SNN_DOUBLE_LOCAL = 0, 1, 2, 3, 4, 5
 SNN_CELL_LIF, SNN_CELL_GRADED = 0, 1
 SNN_SURR_FAST_SIGMOID, SNN_SURR_SIGMOID = 0, 1
 SNN_INPUT_BITS, SNN_INPUT_DENSE = 0, 1
 SNN_FLAG_INPUT_ON_HOST, SNN_FLAG_FORWARD_ONLY, SNN_FLAG_TIME_PHASES = 1, 2, 4
 PHASE_NAMES = ["fwd", "refwd1", "refwd2", "bwd", "dw", "readout", "d2h", "h2d"]
 SNN_OP_FWD, SNN_OP_REFWD1, SNN_OP_REFWD2, SNN_OP_BWD, SNN_OP_D2H, SNN_OP_H2D, SNN_OP_ZERO = range(7)
-STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "remote", SNN_DOUBLE: "double"}
+STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "remote", SNN_DOUBLE: "double",
+                  SNN_HIERARCHICAL: "hierarchical", SNN_DOUBLE_LOCAL: "double_local"}
 
 EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_train_step", "snn_peak_memory",
            "snn_memory_stats_get", "snn_last_error", "snn_plan", "snn_compact_spikes", "snn_get_event_layout",
-           "snn_phase_times_get", "snn_train_step_static"]
+           "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt"]
 SNN_STATIC_WORKSPACE_BYTES = 32 << 20
 
 
@@ -37,7 +38,8 @@ class snn_config(C.Structure):
 
 
 class snn_ckpt(C.Structure):
-    _fields_ = [("strategy", C.c_int32), ("chunk_size", C.c_int32), ("remote_chunk_size", C.c_int32)]
+    _fields_ = [("strategy", C.c_int32), ("chunk_size", C.c_int32), ("remote_chunk_size", C.c_int32),
+                ("nb_local", C.c_int32)]
 
 
 class snn_step_args(C.Structure):
@@ -93,6 +95,8 @@ def _load() -> C.CDLL:
     lib.snn_compact_spikes.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
     lib.snn_phase_times_get.argtypes = [C.c_void_p, C.POINTER(snn_phase_times)]
+    lib.snn_suggest_ckpt.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_size_t, C.c_float,
+                                     C.POINTER(snn_ckpt)]
     lib.snn_get_event_layout.argtypes = [C.c_void_p, C.c_int32, C.POINTER(snn_event_layout)]
     return lib
 
@@ -179,6 +183,15 @@ def snn_plan(T: int, ckpt: snn_ckpt):
     ops = (snn_op * n.value)()
     _check(lib.snn_plan(T, C.byref(ckpt), ops, n.value, C.byref(n), C.byref(nl), C.byref(nr)))
     return list(ops), nl.value, nr.value
+
+
+def snn_suggest_ckpt(net, T: int, B: int, strategy: int, device_budget_bytes: int = 0,
+                     max_activity: float = 0.25) -> snn_ckpt:
+    """Checkpoint intervals by the paper's rules of thumb (host only; net may be None except for REMOTE
+    with a budget)."""
+    c = snn_ckpt()
+    _check(lib.snn_suggest_ckpt(net, T, B, strategy, device_budget_bytes, max_activity, C.byref(c)), net)
+    return c
 
 
 def snn_compact_spikes(masks_ptr: int, n_rows: int, n_words: int, idx_out_ptr: int, capacity: int,

@@ -24,7 +24,8 @@ struct snn_net {
   snn_memory_stats stats{};
   // layout of the last step, for inspection
   std::vector<snn_event_layout> ev_layout;
-  cudaEvent_t ev_main = nullptr, ev_slot[2] = {nullptr, nullptr};
+  cudaEvent_t ev_main = nullptr;
+  std::vector<cudaEvent_t> copy_events;    // one per checkpoint copy in flight, grown on demand
   std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
   snn_phase_times phases{};
 };
@@ -54,7 +55,9 @@ struct Layout {
   int words[MAXL + 1];
   size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
   size_t event_bytes, total;
+  size_t tier2;          // DOUBLE_LOCAL: the second checkpoint tier, in device memory
   int n_local, n_remote;
+  bool tier2_on_device;
 };
 
 bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float max_activity, Layout& lo,
@@ -99,6 +102,8 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   }
   lo.event_bytes = cur - ev0;
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
+  lo.tier2_on_device = ck->strategy == SNN_DOUBLE_LOCAL;
+  lo.tier2 = lo.tier2_on_device ? take((size_t)lo.n_remote * lo.state_bytes) : 0;
   lo.total = cur;
   return true;
 }
@@ -137,8 +142,7 @@ extern "C" snn_status snn_create(const snn_config* cfg, snn_net** out) {
 extern "C" void snn_destroy(snn_net* net) {
   if (!net) return;
   if (net->ev_main) cudaEventDestroy(net->ev_main);
-  for (auto& e : net->ev_slot)
-    if (e) cudaEventDestroy(e);
+  for (auto& e : net->copy_events) cudaEventDestroy(e);
   for (auto& e : net->timing_events) cudaEventDestroy(e);
   delete net;
 }
@@ -155,7 +159,7 @@ extern "C" snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t
   if (!compute_layout(net, T, B, ckpt, max_activity, lo, why))
     return fail(const_cast<snn_net*>(net), SNN_ERR_INVALID_ARG, "%s", why.c_str());
   if (device_bytes) *device_bytes = lo.total;
-  if (pinned_bytes) *pinned_bytes = (size_t)lo.n_remote * lo.state_bytes;
+  if (pinned_bytes) *pinned_bytes = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
   return SNN_OK;
 }
 
@@ -206,7 +210,8 @@ struct Exec {
   int L, B, T;
   int launches = 0, d2h = 0, h2d = 0;
   int carry_cur = 0;
-  bool slot_pending[2] = {false, false};
+  std::vector<int> slot_event;   // per local slot: index of the copy event it waits on, or -1
+  int copies_in_flight = 0;
   bool remote_tier;
   bool timed = false;
   struct Span { int phase, ev0, ev1, launches; };
@@ -262,11 +267,13 @@ struct Exec {
   uint32_t* off(int l, int t) const { return at<uint32_t>(lo.off[l]) + (size_t)t * B; }
   uint32_t* pool(int l) const { return at<uint32_t>(lo.pool[l]); }
 
+  // The main stream waits for the checkpoint copy that last touched local slot s, if one is pending.
   snn_status wait_slot(int s) {
-    if (remote_tier && s >= 0 && s < 2 && slot_pending[s]) {
-      CUDA_TRY(cudaStreamWaitEvent(main, net->ev_slot[s], 0));
-      slot_pending[s] = false;
-    }
+    if (!remote_tier || s < 0 || s >= (int)slot_event.size() || slot_event[s] < 0) return SNN_OK;
+    const int e = slot_event[s];
+    CUDA_TRY(cudaStreamWaitEvent(main, net->copy_events[e], 0));
+    for (int& x : slot_event)
+      if (x == e) x = -1;
     return SNN_OK;
   }
 
@@ -484,19 +491,39 @@ struct Exec {
   }
 
   snn_status run_copy(const snn_op& op) {
-    char* remote = static_cast<char*>(a->pinned_ws) + (size_t)op.remote_slot * lo.state_bytes;
-    const bool to_host = op.kind == SNN_OP_D2H;
-    const int s = to_host ? op.in_slot : op.keep_slot;
+    const int count = std::max(1, op.buf_len);
+    const size_t bytes = (size_t)count * lo.state_bytes;
+    char* remote = (lo.tier2_on_device ? ws + lo.tier2 : static_cast<char*>(a->pinned_ws)) +
+                   (size_t)op.remote_slot * lo.state_bytes;
+    const bool out = op.kind == SNN_OP_D2H;
+    const int s = out ? op.in_slot : op.keep_slot;
     char* local = ws + lo.slots + (size_t)s * lo.state_bytes;
+    // a slot that an earlier copy still uses: order the two copies through the main stream
+    for (int k = 0; k < count; ++k)
+      if (wait_slot(s + k) != SNN_OK) return SNN_ERR_CUDA;
     // the copy starts after everything issued so far on the main stream
     CUDA_TRY(cudaEventRecord(net->ev_main, main));
     CUDA_TRY(cudaStreamWaitEvent(side, net->ev_main, 0));
-    const int span = begin_span(to_host ? SNN_PHASE_D2H : SNN_PHASE_H2D, side);
-    if (to_host) { CUDA_TRY(cudaMemcpyAsync(remote, local, lo.state_bytes, cudaMemcpyDeviceToHost, side)); ++d2h; }
-    else { CUDA_TRY(cudaMemcpyAsync(local, remote, lo.state_bytes, cudaMemcpyHostToDevice, side)); ++h2d; }
+    const int span = begin_span(out ? SNN_PHASE_D2H : SNN_PHASE_H2D, side);
+    const cudaMemcpyKind kind = lo.tier2_on_device ? cudaMemcpyDeviceToDevice
+                                                    : (out ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice);
+    if (out) { CUDA_TRY(cudaMemcpyAsync(remote, local, bytes, kind, side)); ++d2h; }
+    else { CUDA_TRY(cudaMemcpyAsync(local, remote, bytes, kind, side)); ++h2d; }
     end_span(span, side);
-    CUDA_TRY(cudaEventRecord(net->ev_slot[s], side));
-    slot_pending[s] = true;
+    // one event per copy in flight; events are reused once every slot that waited on them was released
+    int e = 0;
+    for (;; ++e) {
+      bool used = false;
+      for (int x : slot_event) used |= x == e;
+      if (!used) break;
+    }
+    while ((int)net->copy_events.size() <= e) {
+      cudaEvent_t ev;
+      CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+      net->copy_events.push_back(ev);
+    }
+    CUDA_TRY(cudaEventRecord(net->copy_events[e], side));
+    for (int k = 0; k < count; ++k) slot_event[s + k] = e;
     return SNN_OK;
   }
 };
@@ -537,7 +564,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   if (!compute_layout(net, T, B, &a->ckpt, a->max_activity, ex.lo, why))
     return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
   const Layout& lo = ex.lo;
-  const size_t pinned_need = (size_t)lo.n_remote * lo.state_bytes;
+  const size_t pinned_need = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
   if (a->device_ws_bytes < lo.total)
     return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL, "device workspace %zu < %zu bytes", a->device_ws_bytes, lo.total);
   if (pinned_need > 0 && (!a->pinned_ws || a->pinned_ws_bytes < pinned_need))
@@ -553,11 +580,10 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   ex.main = (cudaStream_t)a->main_stream;
   ex.side = a->side_stream ? (cudaStream_t)a->side_stream : ex.main;
   ex.remote_tier = lo.n_remote > 0;
+  ex.slot_event.assign(lo.n_local, -1);
   ex.timed = (a->flags & SNN_FLAG_TIME_PHASES) != 0;
   if (!net->ev_main) {
     CUDA_TRY(cudaEventCreateWithFlags(&net->ev_main, cudaEventDisableTiming));
-    CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[0], cudaEventDisableTiming));
-    CUDA_TRY(cudaEventCreateWithFlags(&net->ev_slot[1], cudaEventDisableTiming));
   }
   {
     static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory

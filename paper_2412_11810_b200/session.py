@@ -65,8 +65,8 @@ class Session:
         self.dW_rec = [torch.empty_like(w) for w in self.W_rec]
         self.dW_out = torch.empty_like(self.W_out)
 
-    def ckpt(self, strategy: int, chunk_size: int = 0, remote_chunk_size: int = 0) -> sb.snn_ckpt:
-        return sb.snn_ckpt(strategy, chunk_size, remote_chunk_size)
+    def ckpt(self, strategy: int, chunk_size: int = 0, remote_chunk_size: int = 0, nb_local: int = 0) -> sb.snn_ckpt:
+        return sb.snn_ckpt(strategy, chunk_size, remote_chunk_size, nb_local)
 
     def ensure_workspace(self, T: int, B: int, ck: sb.snn_ckpt, max_activity: float):
         d, p = sb.snn_workspace_query(self.net, T, B, ck, max_activity)
@@ -81,7 +81,7 @@ class Session:
     # ---- the training step -----------------------------------------------------------------
     def train_step(self, input_bits, targets, strategy: int = sb.SNN_STANDARD, chunk_size: int = 0,
                    remote_chunk_size: int = 0, max_activity: float = 0.25, forward_only: bool = False,
-                   keep_V: bool = False, time_phases: bool = False) -> float:
+                   keep_V: bool = False, time_phases: bool = False, nb_local: int = 0) -> float:
         """input_bits: uint32 [T][B][ceil(N_0/32)] spike words (LIF cell; int32 storage) or float32
         [T][B][N_0] dense values (graded cell), as a CUDA tensor or as a pinned host tensor / numpy
         array (then it is copied to the device inside the call); targets alike."""
@@ -94,7 +94,7 @@ class Session:
             if not isinstance(targets, torch.Tensor):
                 targets = torch.from_numpy(np.ascontiguousarray(targets, np.int32)).pin_memory()
         T, B = int(input_bits.shape[0]), int(input_bits.shape[1])
-        ck = self.ckpt(strategy, chunk_size, remote_chunk_size)
+        ck = self.ckpt(strategy, chunk_size, remote_chunk_size, nb_local)
         self.ensure_workspace(T, B, ck, max_activity)
         flags = (sb.SNN_FLAG_INPUT_ON_HOST if on_host else 0) | (sb.SNN_FLAG_FORWARD_ONLY if forward_only else 0) \
             | (sb.SNN_FLAG_TIME_PHASES if time_phases else 0)

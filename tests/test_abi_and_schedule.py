@@ -45,8 +45,11 @@ def test_workspace_query_and_bad_intervals():
     assert p0 == 0 and p1 == 0 and p2 == 10 * ms
     # same event storage, different number of dense states: T+1, K + T/K, K + 2 (256-byte rounding aside)
     assert abs((d0 - d1) - ms * (101 - 20)) < 512 and abs((d1 - d2) - ms * (20 - 12)) < 512
+    d3, p3 = sb.snn_workspace_query(net, 100, 2, sb.snn_ckpt(sb.SNN_DOUBLE, 5, 20), 0.25)
+    d4, p4 = sb.snn_workspace_query(net, 100, 2, sb.snn_ckpt(sb.SNN_DOUBLE_LOCAL, 5, 20), 0.25)
+    assert p3 == 5 * ms and p4 == 0 and abs((d4 - d3) - 5 * ms) < 512      # the second tier moves on device
     for ck in (sb.snn_ckpt(sb.SNN_CHUNK, 0, 0), sb.snn_ckpt(sb.SNN_DOUBLE, 4, 6), sb.snn_ckpt(sb.SNN_DOUBLE, 8, 4),
-               sb.snn_ckpt(7, 1, 1)):
+               sb.snn_ckpt(sb.SNN_HIERARCHICAL, 4, 0, 0), sb.snn_ckpt(7, 1, 1)):
         with pytest.raises(sb.SnnError):
             sb.snn_workspace_query(net, 100, 2, ck, 0.25)
     with pytest.raises(sb.SnnError):
@@ -68,7 +71,14 @@ def test_train_step_rejects_bad_arguments_without_a_gpu():
 CASES = [(sb.SNN_STANDARD, 0, 0), (sb.SNN_CHUNK, 4, 0), (sb.SNN_CHUNK, 1, 0), (sb.SNN_CHUNK, 13, 0),
          (sb.SNN_CHUNK, 40, 0), (sb.SNN_REMOTE, 4, 0), (sb.SNN_REMOTE, 1, 0), (sb.SNN_REMOTE, 13, 0),
          (sb.SNN_DOUBLE, 2, 6), (sb.SNN_DOUBLE, 3, 3), (sb.SNN_DOUBLE, 1, 4), (sb.SNN_DOUBLE, 2, 26),
-         (sb.SNN_DOUBLE, 13, 13)]
+         (sb.SNN_DOUBLE, 13, 13), (sb.SNN_DOUBLE_LOCAL, 2, 6), (sb.SNN_DOUBLE_LOCAL, 3, 3),
+         (sb.SNN_HIERARCHICAL, 2, 2), (sb.SNN_HIERARCHICAL, 2, 3), (sb.SNN_HIERARCHICAL, 3, 1),
+         (sb.SNN_HIERARCHICAL, 1, 4), (sb.SNN_HIERARCHICAL, 4, 9), (sb.SNN_HIERARCHICAL, 13, 2)]
+# the third number is remote_chunk_size, except for HIERARCHICAL where it is nb_local
+
+
+def _ckpt(strategy, K, R):
+    return sb.snn_ckpt(strategy, K, 0, R) if strategy == sb.SNN_HIERARCHICAL else sb.snn_ckpt(strategy, K, R, 0)
 
 
 def _execute_plan(orc, spec, d, T, ops, n_local, n_remote):
@@ -90,9 +100,13 @@ def _execute_plan(orc, spec, d, T, ops, n_local, n_remote):
         if k == sb.SNN_OP_ZERO:
             local[op.keep_slot] = (0, [np.zeros((B, sizes[l + 1]), orc.real) for l in range(L)])
         elif k == sb.SNN_OP_D2H:
-            remote[op.remote_slot] = local[op.in_slot]; count["d2h"] += 1
+            for i in range(max(1, op.buf_len)):
+                remote[op.remote_slot + i] = local[op.in_slot + i]
+            count["d2h"] += 1
         elif k == sb.SNN_OP_H2D:
-            local[op.keep_slot] = remote[op.remote_slot]; count["h2d"] += 1
+            for i in range(max(1, op.buf_len)):
+                local[op.keep_slot + i] = remote[op.remote_slot + i]
+            count["h2d"] += 1
         elif k in (sb.SNN_OP_FWD, sb.SNN_OP_REFWD1, sb.SNN_OP_REFWD2):
             tcur, V = local[op.in_slot]
             assert tcur == op.t0, "the input slot must hold the state of step t0"
@@ -138,7 +152,7 @@ def test_plan_reproduces_full_storage_bptt(orc32, strategy, K, R):
     T = w.T
     spec = NetSpec(w.sizes, leak_from_tau(w.tau_mem), w.theta, w.beta, w.scale())
     full = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
-    ops, n_local, n_remote = sb.snn_plan(T, sb.snn_ckpt(strategy, K, R))
+    ops, n_local, n_remote = sb.snn_plan(T, _ckpt(strategy, K, R))
     r = _execute_plan(orc32, spec, d, T, ops, n_local, n_remote)
     assert r["loss"] == full["loss"]
     for a, b in zip(r["dW_ff"] + r["dW_rec"] + [r["dW_out"]], full["dW_ff"] + full["dW_rec"] + [full["dW_out"]]):
@@ -157,6 +171,13 @@ def test_plan_reproduces_full_storage_bptt(orc32, strategy, K, R):
         assert n_local == Kc + 2 and n_remote == math.ceil(T / K)                                   # Eq. 6 (+1 staging)
         assert c["d2h"] + c["h2d"] == 2 * math.ceil(T / K)                                          # Eq. 7
         assert np.all(c["re1"][1:] == 1)
+    elif strategy == sb.SNN_HIERARCHICAL:
+        n_ck = math.ceil(T / K)
+        P = min(R, n_ck)
+        n_b = math.ceil(n_ck / P)
+        assert n_local == Kc + P                                                                    # Eq. 9
+        assert n_remote == (n_b - 1) * P and c["d2h"] == c["h2d"] == n_b - 1                        # Eq. 10 as read
+        assert np.all(c["re1"][1:] == 1) and c["re2"].sum() == 0
     else:
         assert n_local == Kc + math.ceil(min(R, T) / K) + 1 <= K + R // K + 1                       # Eq. 11 (+1 staging)
         assert n_remote == math.ceil(T / R) and c["d2h"] + c["h2d"] == 2 * math.ceil(T / R)         # Eq. 13
@@ -204,3 +225,27 @@ def test_long_sequence_plans_stay_small_and_valid():
         assert np.all(covered[1:] == 1)
         if ck.strategy == sb.SNN_DOUBLE:
             assert n_local == ck.chunk_size + ck.remote_chunk_size // ck.chunk_size + 1
+
+
+def test_suggested_intervals_follow_the_papers_rules():
+    """Hyperparameter Study: chunk_size = sqrt(T) (64 at T = 4096); Double: remote_chunk_size within
+    64 .. 256 at T = 4096 and chunk_size = sqrt(remote_chunk_size); Remote: the largest chunk that fits."""
+    c = sb.snn_suggest_ckpt(None, 4096, 1, sb.SNN_CHUNK)
+    assert (c.strategy, c.chunk_size) == (sb.SNN_CHUNK, 64)
+    c = sb.snn_suggest_ckpt(None, 4096, 1, sb.SNN_DOUBLE)
+    assert 64 <= c.remote_chunk_size <= 256 and c.chunk_size ** 2 == c.remote_chunk_size
+    for T in (7, 100, 1000, 5000):
+        c = sb.snn_suggest_ckpt(None, T, 1, sb.SNN_DOUBLE)
+        assert c.remote_chunk_size % c.chunk_size == 0 and c.chunk_size >= 1
+        sb.snn_plan(T, c)
+        h = sb.snn_suggest_ckpt(None, T, 1, sb.SNN_HIERARCHICAL)
+        assert h.chunk_size >= 1 and h.nb_local >= 1
+        sb.snn_plan(T, h)
+    net = sb.snn_create([8, 16, 4], 20.0, 1.0)
+    budget, _ = sb.snn_workspace_query(net, 1000, 2, sb.snn_ckpt(sb.SNN_REMOTE, 37, 0), 0.25)
+    c = sb.snn_suggest_ckpt(net, 1000, 2, sb.SNN_REMOTE, budget, 0.25)
+    fits = lambda K: sb.snn_workspace_query(net, 1000, 2, sb.snn_ckpt(sb.SNN_REMOTE, K, 0), 0.25)[0] <= budget
+    assert c.chunk_size >= 37 and fits(c.chunk_size) and not fits(c.chunk_size + 1)
+    with pytest.raises(sb.SnnError):
+        sb.snn_suggest_ckpt(net, 1000, 2, sb.SNN_REMOTE, 1024, 0.25)
+    sb.snn_destroy(net)

@@ -104,7 +104,8 @@ def test_forward_c1_bit_exact(orc32):
 
 # ---------------------------------------------------------------- gradients and strategies
 STRATS = [(1, 4, 0), (1, 1, 0), (1, 13, 0), (1, 40, 0), (2, 4, 0), (2, 1, 0), (2, 5, 0), (3, 2, 6), (3, 3, 3),
-          (3, 1, 4), (3, 2, 26), (3, 13, 13)]
+          (3, 1, 4), (3, 2, 26), (3, 13, 13), (5, 2, 6), (5, 1, 4), (4, 2, 2), (4, 2, 3), (4, 3, 1), (4, 1, 4),
+          (4, 4, 9)]   # (strategy, chunk_size, remote_chunk_size or, for strategy 4, nb_local)
 
 
 def _bits(t):
@@ -124,7 +125,8 @@ def test_gradients_and_all_strategies_tiny(orc32):
     for strat, K, R in STRATS:
         for g in s.dW_ff + s.dW_rec + [s.dW_out]:
             g.fill_(float("nan"))
-        loss2 = s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0)
+        loss2 = s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=0 if strat == 4 else R,
+                             nb_local=R if strat == 4 else 0, max_activity=1.0)
         assert loss2 == loss
         for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
             assert np.array_equal(a, b), f"strategy {strat} K={K} R={R} differs from STANDARD"
@@ -135,11 +137,16 @@ def test_gradients_and_all_strategies_tiny(orc32):
         elif strat == 2:
             assert st.local_state_slots == Kc + 2
             assert st.d2h_copies == st.h2d_copies == math.ceil(w.T / K)
+        elif strat == 4:
+            n_ck = math.ceil(w.T / K)
+            P = min(R, n_ck)
+            assert st.local_state_slots == Kc + P
+            assert st.d2h_copies == st.h2d_copies == math.ceil(n_ck / P) - 1
         else:
             assert st.local_state_slots == Kc + math.ceil(min(R, w.T) / K) + 1
             assert st.d2h_copies == st.h2d_copies == math.ceil(w.T / R)
         dev, pin = s.peak_memory()
-        assert pin == st.remote_state_slots * st.state_bytes
+        assert pin == (0 if strat == 5 else st.remote_state_slots * st.state_bytes)
     s.close()
 
 

@@ -295,7 +295,8 @@ def test_weight_gradient_sparsity_identities(orc32):
 # ---------------------------------------------------------------- checkpointing: exactness, traces, cost models
 CASES = [(ck.STANDARD, 0, 0), (ck.CHUNK, 4, 0), (ck.CHUNK, 1, 0), (ck.CHUNK, 13, 0), (ck.CHUNK, 50, 0),
          (ck.REMOTE, 4, 0), (ck.REMOTE, 5, 0), (ck.DOUBLE, 2, 6), (ck.DOUBLE, 3, 3), (ck.DOUBLE, 1, 4),
-         (ck.DOUBLE, 2, 26)]
+         (ck.DOUBLE, 2, 26), (ck.HIERARCHICAL, 2, 2), (ck.HIERARCHICAL, 2, 3), (ck.HIERARCHICAL, 3, 1),
+         (ck.HIERARCHICAL, 4, 9)]   # third number: remote_chunk_size, or nb_local for HIERARCHICAL
 
 
 @pytest.mark.parametrize("strategy,K,R", CASES)
@@ -306,7 +307,7 @@ def test_every_strategy_equals_full_storage_bit_for_bit(orc32, strategy, K, R):
     spec = spec_of(w)
     full = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
     c = ck.bptt_checkpointed(orc32, spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"],
-                             strategy, K, R)
+                             strategy, K, 0 if strategy == ck.HIERARCHICAL else R, R)
     assert c["loss"] == full["loss"]
     for a, b in zip(c["dW_ff"] + c["dW_rec"] + [c["dW_out"]], full["dW_ff"] + full["dW_rec"] + [full["dW_out"]]):
         assert np.array_equal(a, b)
@@ -325,6 +326,12 @@ def test_every_strategy_equals_full_storage_bit_for_bit(orc32, strategy, K, R):
         assert st["refwd1_steps"] == T and st["refwd2_steps"] == 0
     elif strategy == ck.REMOTE:
         assert st["local_states_peak"] == Kc + 1 and st["transfers"] == 2 * math.ceil(T / K)
+        assert st["refwd1_steps"] == T
+    elif strategy == ck.HIERARCHICAL:
+        n_ck = math.ceil(T / K)
+        P = min(R, n_ck)
+        # Eq. 9: chunk_size + nb_local states; Eq. 10 read as two communications per batch but the last
+        assert st["local_states_peak"] == Kc + P and st["transfers"] == 2 * (math.ceil(n_ck / P) - 1)
         assert st["refwd1_steps"] == T
     else:
         assert st["local_states_peak"] == Kc + math.ceil(min(R, T) / K) <= K + R // K
