@@ -27,7 +27,7 @@ import snn_workloads as wl  # noqa: E402
 
 METRIC = "sample_timesteps_per_s"
 UNIT = "sample-timesteps/s"
-STRATEGY_NAME = {0: "standard", 1: "chunk", 2: "remote", 3: "double"}
+STRATEGY_NAME = {0: "standard", 1: "chunk", 2: "remote", 3: "double", 4: "hierarchical", 5: "double_local"}
 ORACLE_SAMPLE_T = 100   # steps per oracle "step" in --impl reference
 
 
@@ -241,9 +241,11 @@ def run_ours(args, rank, world):
         T = w.T
         K0 = w.chunk_size if w.strategy in (1, 2) else max(1, int(round(T ** 0.5)))
         Kd, Rd = (w.chunk_size, w.remote_chunk_size) if w.strategy == 3 else (16, 256)
-        alt = {0: (0, 0), 1: (K0, 0), 2: (K0, 0), 3: (Kd, Rd)}
+        P0 = max(1, int(round((-(-T // K0)) ** 0.5)))          # nb_local = sqrt(number of checkpoints)
+        alt = {0: (0, 0), 1: (K0, 0), 2: (K0, 0), 3: (Kd, Rd), 4: (K0, P0), 5: (Kd, Rd)}
         for strat, (K, R) in ([] if args.no_strategies else alt.items()):
-            kws = dict(strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=args.max_activity)
+            kws = dict(strategy=strat, chunk_size=K, remote_chunk_size=0 if strat == 4 else R,
+                       nb_local=R if strat == 4 else 0, max_activity=args.max_activity)
             s.train_step(bits, targets, **kws)
             tms = []
             for _ in range(3):
@@ -256,7 +258,8 @@ def run_ours(args, rank, world):
             st = s.stats()
             dp, pp = s.peak_memory()
             per_strategy[STRATEGY_NAME[strat]] = {
-                "chunk_size": K, "remote_chunk_size": R, "value": w.B * T / (float(np.median(tms)) / 1e3),
+                "chunk_size": K, "remote_chunk_size": 0 if strat == 4 else R, "nb_local": R if strat == 4 else 0,
+                "d2h_copies": st.d2h_copies, "h2d_copies": st.h2d_copies, "value": w.B * T / (float(np.median(tms)) / 1e3),
                 "ms_per_step": float(np.median(tms)), "device_peak_bytes": dp, "pinned_peak_bytes": pp,
                 "local_state_slots": st.local_state_slots, "state_bytes": st.state_bytes,
                 "kernel_launches": st.kernel_launches}
