@@ -125,6 +125,19 @@ def run_reference(args, rank):
     }))
 
 
+def aggregate_replicas(per_rank_ms, units_per_rank, world, dist=None, device=None):
+    """Whole-job throughput of independent replicas: every rank processed units_per_rank units; the job
+    took as long as its slowest rank (max over ranks of each entry of per_rank_ms).  Returns
+    (list of max times in ms, list of units per second)."""
+    times = [float(x) for x in per_rank_ms]
+    if dist is not None and world > 1:
+        import torch
+        t = torch.tensor(times, dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        times = [float(x) for x in t]
+    return times, [units_per_rank * world / (ms / 1e3) for ms in times]
+
+
 def algorithmic_bytes(w, activity, B):
     """Bytes the method must move per launch of each step kernel (one wavefront launch = one step of
     every layer), from the per-layer figures: forward gathers the active weight rows and writes V and
@@ -206,13 +219,8 @@ def run_ours(args, rank, world):
     timed_steps(1, bits_host, tg_host)
     e2e_ms, _ = timed_steps(max(3, args.steps // 4), bits_host, tg_host)
     e2e_total = float(sum(e2e_ms)) / len(e2e_ms) * args.steps
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_total], device=s.device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total = float(t[0]), float(t[1])
-    units = w.B * w.T * args.steps * world
-    value = units / (total_ms / 1e3)
-    e2e_value = units / (e2e_total / 1e3)
+    (total_ms, e2e_total), (value, e2e_value) = aggregate_replicas(
+        [total_ms, e2e_total], w.B * w.T * args.steps, world, dist, s.device)
 
     out = None
     if rank == 0:

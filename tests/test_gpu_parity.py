@@ -359,3 +359,21 @@ def test_cell_and_input_format_must_match():
         s.train_step(a_bits, targets)
     assert e.value.status == b.SNN_ERR_UNSUPPORTED
     s.close()
+
+
+@pytest.mark.parametrize("B", [1, 40])
+def test_batch_sizes_outside_the_backward_tiles(orc32, B):
+    """One sample, and more samples than one pass of the backward kernel covers (32); layers of
+    different widths so that some layers have fewer row tiles than the widest one."""
+    w = wl.small(sizes=(40, 260, 516, 6), T=9, B=B, p_in=0.15, g_ff=(2.5, 1.6), seed=31)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    assert all(0.01 < float(x[1:].mean()) < 0.6 for x in ref["S"])
+    s, bits, targets = make_session(w, d)
+    s.train_step(bits, targets, strategy=0, max_activity=1.0)
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    s.train_step(bits, targets, strategy=3, chunk_size=2, remote_chunk_size=4, max_activity=1.0)
+    for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+        assert np.array_equal(a, b)
+    s.close()
