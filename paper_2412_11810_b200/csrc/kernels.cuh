@@ -523,7 +523,7 @@ __device__ __forceinline__ void warp_transpose_reduce(float (&v)[NV], int lane) 
   }
 }
 
-constexpr int BWD_STAGES = 4;   // weight-row groups (4 rows x 512 B per warp) in flight per warp
+constexpr int BWD_STAGES = 4;   // chunks of the W and delta tiles in flight per CTA
 
 __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer& L, int i, int b, float sum) {
   if (i >= L.N || b >= p.B) return;
@@ -537,12 +537,38 @@ __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer&
   if (L.carry_out) L.carry_out[k] = dl;
 }
 
-// BT samples per thread (8 or 16), WB sample groups per CTA; launched with cluster size CS along x:
-// blockIdx.x = row_tile * CS + rank.
-template <int BT, int WB>
-__global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
-  constexpr int NT = 32 * BWD_WR * WB, NV = BWD_RT * BT, VPL = NV / 32, NWARP = BWD_WR * WB, BP = BT * WB;
-  constexpr int STAGE_F4 = (BWD_TM + BP) * 32;      // float4 per stage: 32 weight rows + BP delta rows, 128 k each
+// The contraction itself runs on the tensor cores as a 3-pass TF32 product: every fp32 operand is
+// split into hi = tf32(x) and lo = tf32(x - hi), and D += A_lo B_hi + A_hi B_lo + A_hi B_hi with fp32
+// accumulation, which keeps the result at fp32 accuracy (the dropped lo*lo term is ~2^-22 relative).
+constexpr int BWD_LD = 132;   // padded row length (floats) of the staged tiles: fragment loads hit 32 banks
+
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+  hi = to_tf32(x);
+  lo = to_tf32(x - __uint_as_float(hi));
+}
+// D(16x8) += A(16x8, row) * B(8x8, col); lane = 4 g + t holds A[g][t], A[g+8][t], A[g][t+4], A[g+8][t+4],
+// B[t][g], B[t+4][g] and D[g][2t], D[g][2t+1], D[g+8][2t], D[g+8][2t+1].
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// NTN = sample tiles of 8 per pass (BP = 8 NTN samples), NWARP warps per CTA; launched with cluster
+// size CS along x: blockIdx.x = row_tile * CS + rank.  A CTA owns 32 rows x BP samples.  Chunks of
+// 128 k of W [32][128] and delta [BP][128] stream through a BWD_STAGES-deep cp.async pipeline; within
+// a chunk warp w multiplies the k-steps w, w + NWARP, ... (8 k each) for the whole tile, so every warp
+// ends with a partial 32 x BP tile: the partials are summed in warp order through shared memory, then
+// across the cluster in rank order.
+template <int NTN, int NWARP>
+__global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * BWD_LD, TILE = BWD_TM * BP;
   pdl_launch_dependents();
   cg::cluster_group cluster = cg::this_cluster();
   const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
@@ -550,18 +576,15 @@ __global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_ke
   if (L.mode == 0) return;                          // same for the whole cluster
   const int tile_row0 = (blockIdx.x / CS) * BWD_TM;
   if (tile_row0 >= L.N) return;                     // same for the whole cluster
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int wr = warp % BWD_WR, wb = warp / BWD_WR;
-  const int row0 = tile_row0 + wr * BWD_RT;
-  __shared__ float s_part[NWARP * NV];
-  extern __shared__ float4 s_tiles[];               // [BWD_STAGES][BWD_TM + BP][32]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  __shared__ float s_part[TILE];
+  extern __shared__ float4 s_dyn[];
+  float* const s_tiles = reinterpret_cast<float*>(s_dyn);   // [BWD_STAGES][ROWS][BWD_LD]; later [NWARP][32][BP]
   // this rank's slice of each contraction range, in units of 4 floats
   const int q_rec = L.N / 4, q_ff = L.W_ffa ? L.N_post / 4 : 0;
   const int lo_rec = (int)((long long)q_rec * rank / CS) * 4, hi_rec = (int)((long long)q_rec * (rank + 1) / CS) * 4;
   const int lo_ff = (int)((long long)q_ff * rank / CS) * 4, hi_ff = (int)((long long)q_ff * (rank + 1) / CS) * 4;
-  // One chunk = 128 consecutive k of one matrix: a [32 rows][128] tile of W and a [BP][128] tile of
-  // delta.  Chunks run over this rank's slice of W_ff(l+1) first, then of W_rec, k ascending.  The
-  // tiles of the next BWD_STAGES-1 chunks are in flight (cp.async) while one chunk is multiplied.
+  // chunks run over this rank's slice of W_ff(l+1) first, then of W_rec, k ascending
   const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
   const int rlast = L.N - 1, blast = p.B - 1;
   auto locate = [&](int it, const float*& W, const float*& d, int& ld, int& k0, int& hi) {
@@ -575,70 +598,102 @@ __global__ void __launch_bounds__(32 * BWD_WR * WB, WB == 1 ? 2 : 1) bwd_step_ke
       if (it < it_all) {
         const float* W; const float* d; int ld, k0, hi;
         locate(it, W, d, ld, k0, hi);
-        float4* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F4;
-        for (int q = tid; q < STAGE_F4; q += NT) {
-          const int rr = q >> 5, k = k0 + 4 * (q & 31);
+        float* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
+        for (int q = tid; q < ROWS * 32; q += NT) {
+          const int rr = q >> 5, c4 = q & 31, k = k0 + 4 * c4;
+          float* dst = st + rr * BWD_LD + 4 * c4;
           if (k < hi) {
             // rows and samples past the end are clamped to the last valid one; their sums are never used
             const float* src = rr < BWD_TM
                                    ? W + (size_t)(tile_row0 + rr < rlast ? tile_row0 + rr : rlast) * ld + k
                                    : d + (size_t)(bp0 + rr - BWD_TM < blast ? bp0 + rr - BWD_TM : blast) * ld + k;
-            cp_async16(st + q, src);
+            cp_async16(dst, src);
+          } else {
+            *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);   // past the slice: contributes 0
           }
         }
       }
       cp_async_commit();
     };
-    float acc[NV];
+    float acc[2][NTN][4];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) acc[i] = 0.f;
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
     for (int it = 0; it < BWD_STAGES - 1; ++it) issue(it);
     for (int it = 0; it < it_all; ++it) {
       cp_async_wait<BWD_STAGES - 2>();   // this thread's copies of chunk `it` have landed
       __syncthreads();                   // ... everybody's have, and chunk it-1 has been consumed
       issue(it + BWD_STAGES - 1);        // refills the stage chunk it-1 used
-      const float* W; const float* d; int ld, k0, hi;
-      locate(it, W, d, ld, k0, hi);
-      if (k0 + 4 * lane < hi) {
-        const float4* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F4 + lane;
-        float4 w[BWD_RT];
+      const float* Ws = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
+      const float* Ds = Ws + BWD_TM * BWD_LD;
+#pragma unroll 1
+      for (int ks = warp; ks < 16; ks += NWARP) {
+        const int kk = ks * 8 + t;
+        uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
 #pragma unroll
-        for (int r = 0; r < BWD_RT; ++r) w[r] = st[(wr * BWD_RT + r) * 32];
-#pragma unroll
-        for (int bb = 0; bb < BT; ++bb) {
-          const float4 dv = st[(BWD_TM + wb * BT + bb) * 32];
-#pragma unroll
-          for (int r = 0; r < BWD_RT; ++r) {
-            float a = acc[r * BT + bb];
-            a = fmaf(w[r].x, dv.x, a); a = fmaf(w[r].y, dv.y, a);
-            a = fmaf(w[r].z, dv.z, a); a = fmaf(w[r].w, dv.w, a);
-            acc[r * BT + bb] = a;
-          }
+        for (int mt = 0; mt < 2; ++mt) {
+          const float* r0 = Ws + (mt * 16 + g) * BWD_LD + kk;
+          split_tf32(r0[0], a_hi[mt][0], a_lo[mt][0]);
+          split_tf32(r0[8 * BWD_LD], a_hi[mt][1], a_lo[mt][1]);
+          split_tf32(r0[4], a_hi[mt][2], a_lo[mt][2]);
+          split_tf32(r0[8 * BWD_LD + 4], a_hi[mt][3], a_lo[mt][3]);
         }
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) {
+          const float* r0 = Ds + (nt * 8 + g) * BWD_LD + kk;
+          split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
+          split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) {
+            mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
+            mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
+            mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
+          }
       }
     }
     cp_async_wait<0>();
-    __syncthreads();   // the stages are free again for the next pass over the samples
-    const int b0 = bp0 + wb * BT;
-    warp_transpose_reduce<NV>(acc, lane);
+    __syncthreads();   // the stages are free: they now hold the warps' partial tiles [NWARP][32][BP]
+    {
+      float* mine = s_tiles + (size_t)warp * TILE;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) {
+          const int r = mt * 16 + g, c = nt * 8 + 2 * t;
+          mine[r * BP + c] = acc[mt][nt][0];       mine[r * BP + c + 1] = acc[mt][nt][1];
+          mine[(r + 8) * BP + c] = acc[mt][nt][2]; mine[(r + 8) * BP + c + 1] = acc[mt][nt][3];
+        }
+    }
+    __syncthreads();
     if (CS == 1) {
+      for (int e = tid; e < TILE; e += NT) {
+        float sum = 0.f;
 #pragma unroll
-      for (int j = 0; j < VPL; ++j) {
-        const int idx = lane * VPL + j;
-        bwd_epilogue(p, L, row0 + idx / BT, b0 + idx % BT, acc[j]);
+        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILE + e];
+        bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum);
       }
+      __syncthreads();   // before the next pass refills the stages
     } else {
+      for (int e = tid; e < TILE; e += NT) {
+        float sum = 0.f;
 #pragma unroll
-      for (int j = 0; j < VPL; ++j) s_part[warp * NV + lane * VPL + j] = acc[j];
+        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILE + e];
+        s_part[e] = sum;
+      }
       cluster.sync();
       // every rank finishes a share of the tile: totals summed over the ranks in rank order
-      for (int e = rank + CS * tid; e < NWARP * NV; e += CS * NT) {
+      for (int e = rank + CS * tid; e < TILE; e += CS * NT) {
         float sum = 0.f;
         for (int r = 0; r < CS; ++r) sum += cluster.map_shared_rank(s_part, r)[e];
-        const int w = e / NV, idx = e % NV;
-        bwd_epilogue(p, L, tile_row0 + (w % BWD_WR) * BWD_RT + idx / BT, bp0 + (w / BWD_WR) * BT + idx % BT, sum);
+        bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum);
       }
-      cluster.sync();  // nobody leaves or overwrites s_part while another rank still reads it
+      cluster.sync();  // nobody leaves or overwrites s_part / the stages while another rank still reads
     }
   }
 }

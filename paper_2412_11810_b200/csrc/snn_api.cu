@@ -406,9 +406,11 @@ struct Exec {
     else launch_pdl(dw_kernel<U, false>, grid, dim3(32 * DW_ROWS), dw_smem_bytes<U, false>(d.window), d);
     ++launches;
   }
-  template <int BT, int WB> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
-    return launch_pdl(bwd_step_kernel<BT, WB>, dim3(tiles * CS, 1, L), dim3(32 * BWD_WR * WB),
-                      (size_t)BWD_STAGES * (BWD_TM + BT * WB) * 32 * sizeof(float4), p, CS);
+  // dynamic shared memory of bwd_step_kernel for BP samples per pass: the staged tiles
+  static size_t bwd_smem_bytes(int bp) { return (size_t)BWD_STAGES * (BWD_TM + bp) * BWD_LD * sizeof(float); }
+  template <int NTN, int NWARP> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
+    return launch_pdl(bwd_step_kernel<NTN, NWARP>, dim3(tiles * CS, 1, L), dim3(32 * NWARP),
+                      bwd_smem_bytes(8 * NTN), p, CS);
   }
 
   // BWD: layer wavefront, layer l runs L-l steps behind the last layer; then the weight
@@ -448,9 +450,9 @@ struct Exec {
         f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
       }
       cudaError_t le;
-      if (B <= 8) le = launch_bwd<8, 1>(p, tiles, CS);
-      else if (B <= 16) le = launch_bwd<16, 1>(p, tiles, CS);
-      else le = launch_bwd<16, 2>(p, tiles, CS);
+      if (B <= 8) le = launch_bwd<1, 8>(p, tiles, CS);
+      else if (B <= 16) le = launch_bwd<2, 8>(p, tiles, CS);
+      else le = launch_bwd<4, 16>(p, tiles, CS);
       if (le != cudaSuccess) return fail(net, SNN_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(le));
       ++launches;
     }
@@ -588,14 +590,14 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   {
     static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
     if (!smem_opt_in) {
-      auto bwd_smem = [](int bp) { return (int)(BWD_STAGES * (BWD_TM + bp) * 32 * sizeof(float4)); };
+
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(8)));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(16)));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bwd_smem(32)));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8)));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(16)));
+      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(32)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, true>(DW_WINDOW)));
