@@ -587,30 +587,41 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
   // chunks run over this rank's slice of W_ff(l+1) first, then of W_rec, k ascending
   const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
   const int rlast = L.N - 1, blast = p.B - 1;
-  auto locate = [&](int it, const float*& W, const float*& d, int& ld, int& k0, int& hi) {
-    if (it < it_ff) { W = L.W_ffa; d = L.d_above; ld = L.N_post; k0 = lo_ff + it * 128; hi = hi_ff; }
-    else { W = L.W_rec; d = L.d_next; ld = L.N; k0 = lo_rec + (it - it_ff) * 128; hi = hi_rec; }
-  };
-
+  // Every thread copies the same ITER (row, 16-byte column) positions of each chunk; their global
+  // addresses at k = 0 are worked out once per pass over the samples, so that issuing a chunk costs an
+  // add, a compare and the copy per position.
+  constexpr int ITER = ROWS * 32 / NT;
+  static_assert(ROWS * 32 % NT == 0, "the staged tile divides evenly among the threads");
   pdl_wait();
   for (int bp0 = 0; bp0 < p.B; bp0 += BP) {
+    const float* src_rec[ITER];
+    const float* src_ff[ITER];
+    int dst_off[ITER], kcol[ITER];
+#pragma unroll
+    for (int j = 0; j < ITER; ++j) {
+      const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
+      kcol[j] = 4 * c4;
+      dst_off[j] = rr * BWD_LD + 4 * c4;
+      if (rr < BWD_TM) {   // rows and samples past the end are clamped to the last valid one; never used
+        const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;
+        src_rec[j] = L.W_rec + row * L.N + 4 * c4;
+        src_ff[j] = L.W_ffa ? L.W_ffa + row * L.N_post + 4 * c4 : nullptr;
+      } else {
+        const size_t b = bp0 + rr - BWD_TM < blast ? bp0 + rr - BWD_TM : blast;
+        src_rec[j] = L.d_next + b * L.N + 4 * c4;
+        src_ff[j] = L.d_above ? L.d_above + b * L.N_post + 4 * c4 : nullptr;
+      }
+    }
     auto issue = [&](int it) {
       if (it < it_all) {
-        const float* W; const float* d; int ld, k0, hi;
-        locate(it, W, d, ld, k0, hi);
+        const bool ff = it < it_ff;
+        const int k0 = ff ? lo_ff + it * 128 : lo_rec + (it - it_ff) * 128;
+        const int hi = ff ? hi_ff : hi_rec;
         float* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
-        for (int q = tid; q < ROWS * 32; q += NT) {
-          const int rr = q >> 5, c4 = q & 31, k = k0 + 4 * c4;
-          float* dst = st + rr * BWD_LD + 4 * c4;
-          if (k < hi) {
-            // rows and samples past the end are clamped to the last valid one; their sums are never used
-            const float* src = rr < BWD_TM
-                                   ? W + (size_t)(tile_row0 + rr < rlast ? tile_row0 + rr : rlast) * ld + k
-                                   : d + (size_t)(bp0 + rr - BWD_TM < blast ? bp0 + rr - BWD_TM : blast) * ld + k;
-            cp_async16(dst, src);
-          } else {
-            *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);   // past the slice: contributes 0
-          }
+#pragma unroll
+        for (int j = 0; j < ITER; ++j) {
+          if (k0 + kcol[j] < hi) cp_async16(st + dst_off[j], (ff ? src_ff[j] : src_rec[j]) + k0);
+          else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);   // past the slice
         }
       }
       cp_async_commit();
@@ -647,14 +658,19 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
           split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
           split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
         }
+        // small terms first; consecutive instructions go to different accumulators
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) {
-            mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
-            mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
-            mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
-          }
+          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
       }
     }
     cp_async_wait<0>();
