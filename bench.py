@@ -152,6 +152,18 @@ def algorithmic_bytes(w, activity, B):
     return fwd, bwd
 
 
+def dw_bytes(w, activity, B, n_steps):
+    """Bytes one weight-gradient launch (a segment of n_steps steps, all matrices) must move: every touched
+    dW row read and written once, and one delta row read per event."""
+    sz = w.sizes
+    total = 0.0
+    for l in range(1, w.L + 1):
+        for n_pre, p in ((sz[l - 1], activity[l - 1]), (sz[l], activity[l])):
+            touched = n_pre * (1.0 - (1.0 - min(p, 1.0)) ** (n_steps * B))
+            total += 8.0 * sz[l] * touched + 4.0 * sz[l] * n_steps * B * p * n_pre
+    return total
+
+
 def run_ours(args, rank, world):
     import torch
     from paper_2412_11810_b200 import Session, binding as sb
@@ -233,13 +245,16 @@ def run_ours(args, rank, world):
         ph = {k: (sum(p[k][0] for p in phases) / len(phases), phases[0][k][1]) for k in phases[0]}
         peak, peak_kind = read_peaks()
         dominant = max(("fwd", "refwd1", "refwd2", "bwd", "dw"), key=lambda k: ph[k][0])
-        per_launch_bytes = {"fwd": fwd_b, "refwd1": fwd_b, "refwd2": fwd_b, "bwd": bwd_b}.get(dominant)
+        seg = {0: w.T, 1: w.chunk_size, 2: w.chunk_size, 3: w.chunk_size, 4: w.chunk_size, 5: w.chunk_size}[w.strategy]
+        per_launch_bytes = {"fwd": fwd_b, "refwd1": fwd_b, "refwd2": fwd_b, "bwd": bwd_b,
+                            "dw": dw_bytes(w, activity, w.B, min(seg, w.T))}.get(dominant)
         roof = None
         if per_launch_bytes and ph[dominant][1] > 0:
             avg_s = ph[dominant][0] / 1e3 / ph[dominant][1]
             ach = per_launch_bytes / avg_s / 1e9
             roof = {"bound": "hbm", "kernel": {"fwd": "fwd_step_kernel<true>", "refwd1": "fwd_step_kernel<false>",
-                                               "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel"}[dominant],
+                                               "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel",
+                                               "dw": "dw_kernel"}[dominant],
                     "phase": dominant,
                     "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak,
                     "traffic": None, "algorithmic_bytes_per_launch": per_launch_bytes,
