@@ -744,17 +744,19 @@ struct DwParams {
 
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
 constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
-constexpr int DW_GROUP = 4;       // delta rows per copy group
+// delta rows per copy group: 4, or 2 for the widest column tile (keeps the ring at 64 KB per CTA)
+template <int U> __host__ __device__ constexpr int dw_group() { return U >= 4 ? 2 : 4; }
 constexpr int DW_STAGES = 2;      // copy groups in flight per warp
 
 // shared memory of dw_kernel in bytes for a window of `window` pairs
 template <int U, bool GRADED> constexpr size_t dw_smem_bytes(int window) {
-  return (size_t)DW_ROWS * DW_STAGES * DW_GROUP * U * 32 * sizeof(float4) +
+  return (size_t)DW_ROWS * DW_STAGES * dw_group<U>() * U * 32 * sizeof(float4) +
          (size_t)window * sizeof(uint32_t) * (2 + DW_ROWS + (GRADED ? 1 + DW_ROWS : 0));
 }
 
 template <int U, bool GRADED>
 __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const __grid_constant__ DwParams p) {
+  constexpr int DW_GROUP = dw_group<U>();
   pdl_launch_dependents();
   const DwArgs& a = p.m[blockIdx.z];
   if ((int)blockIdx.y * DW_ROWS >= a.N_pre || (int)blockIdx.x * 128 * U >= a.N) return;
