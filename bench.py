@@ -244,6 +244,9 @@ def run_ours(args, rank, world):
         fwd_b, bwd_b = algorithmic_bytes(w, activity, w.B)
         ph = {k: (sum(p[k][0] for p in phases) / len(phases), phases[0][k][1]) for k in phases[0]}
         peak, peak_kind = read_peaks()
+        if ph["ffgemm"][1] > 0:
+            # layer-by-layer backward order: a backward launch is one step of ONE layer and streams W_rec only
+            bwd_b = sum(4.0 * n * n + 16.0 * w.B * n for n in w.sizes[1:-1]) / w.L
         dominant = max(("fwd", "refwd1", "refwd2", "bwd", "dw"), key=lambda k: ph[k][0])
         seg = {0: w.T, 1: w.chunk_size, 2: w.chunk_size, 3: w.chunk_size, 4: w.chunk_size, 5: w.chunk_size}[w.strategy]
         per_launch_bytes = {"fwd": fwd_b, "refwd1": fwd_b, "refwd2": fwd_b, "bwd": bwd_b,

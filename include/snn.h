@@ -121,6 +121,13 @@ snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const s
 #define SNN_FLAG_INPUT_ON_HOST 1u /* input and targets are pinned host pointers; copied in the call */
 #define SNN_FLAG_FORWARD_ONLY 2u  /* forward pass, readout and loss only                            */
 #define SNN_FLAG_TIME_PHASES 4u   /* bracket every pass with CUDA events (see snn_phase_times_get)  */
+/* The backward pass has two launch orders.  Wavefront: one launch per step covers all layers and also
+ * multiplies by W_ff of the layer above.  Layer by layer: runs of 32 steps, the feed-forward term of a
+ * whole run computed as one product so that W_ff is streamed once per run.  By default the second is
+ * used when the weights exceed 96 MB (they then do not stay in L2); these flags force one or the other.
+ * Gradients are bit-identical across strategies for a given order, not between the two orders. */
+#define SNN_FLAG_BACKWARD_LAYER_BY_LAYER 8u
+#define SNN_FLAG_BACKWARD_WAVEFRONT 16u
 
 typedef struct {
   int32_t T, B;
@@ -195,10 +202,11 @@ snn_status snn_memory_stats_get(const snn_net* net, snn_memory_stats* out);
 /* Device time of the last step per pass of Fig. 1, measured with CUDA events on the main stream
  * when the step ran with SNN_FLAG_TIME_PHASES, and the kernels launched in each.  BWD is the
  * surrogate-gradient step kernel, DW the sparse outer-product weight-gradient kernel; D2H and H2D are the
- * checkpoint copies, timed on the side stream (their `launches` count copies; they overlap the passes). */
+ * checkpoint copies, timed on the side stream (their `launches` count copies; they overlap the passes);
+ * FFGEMM is the time-batched feed-forward product of the layer-by-layer backward order. */
 typedef enum { SNN_PHASE_FWD = 0, SNN_PHASE_REFWD1 = 1, SNN_PHASE_REFWD2 = 2, SNN_PHASE_BWD = 3,
                SNN_PHASE_DW = 4, SNN_PHASE_READOUT = 5, SNN_PHASE_D2H = 6, SNN_PHASE_H2D = 7,
-               SNN_N_PHASES = 8 } snn_phase;
+               SNN_PHASE_FFGEMM = 8, SNN_N_PHASES = 9 } snn_phase;
 typedef struct {
   float ms[SNN_N_PHASES];
   int32_t launches[SNN_N_PHASES];

@@ -475,6 +475,7 @@ struct BwdLayer {
   const float* d_next;    // [B][N]      delta^l_{t+1}
   const float* d_above;   // [B][N_post] delta^{l+1}_t or null
   const float* g_out;     // [B][N] or null
+  const float* g_ff;      // [B][N] or null: W_ff^{l+1} delta^{l+1}_t computed ahead for a run of steps
   float* carry_out;       // optional second copy of delta_t
   int N, N_post;
   int mode;               // 0 idle, 1 step
@@ -530,6 +531,7 @@ __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer&
   const size_t k = (size_t)b * L.N + i;
   const float dn = L.d_next[k];
   float g = sum + (L.g_out ? L.g_out[k] : 0.f);
+  if (L.g_ff) g += L.g_ff[k];
   if (p.cell == 0) g = fmaf(-p.theta, dn, g);
   const float sp = surrogate_grad(L.V_delta[k], p.theta, p.beta, p.surrogate, p.cell);
   const float dl = fmaf(g, sp, p.alpha * dn);
@@ -711,6 +713,132 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
       }
       cluster.sync();  // nobody leaves or overwrites s_part / the stages while another rank still reads
     }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Time-batched feed-forward part of the backward pass: for a run of steps the deltas of the layer
+// above are all known before the layer below starts, so W_ff^{l+1} delta^{l+1}_t is one product
+// with M = steps x B columns instead of one per step:
+//   out[(ts, b)][i] = sum_k W[i][k] * delta_{t0+1+ts}[b][k]
+// W is then streamed once per 64 (step, sample) pairs instead of once per step.  Same machinery as
+// bwd_step_kernel: 32 rows of W per CTA, 128-wide chunks of k through a cp.async pipeline, 3-pass
+// TF32 tensor-core product, warp partials summed in warp order; per output the order of additions
+// depends on k only, not on which pairs share a tile.
+struct FfGemmParams {
+  const float* W;        // [N][K]   W_ff of the layer above (row = neuron of this layer)
+  const float* delta0;   // delta of the layer above at the first step of the run: row (ts, b) at
+                         //   delta0 + ts * slot_stride + b * K
+  float* out;            // [n_steps * B][N]
+  size_t slot_stride;    // floats between consecutive steps
+  int N, K, B, n_steps;
+};
+
+constexpr int FFG_NTN = 8, FFG_NWARP = 16;   // 64 (step, sample) pairs per pass, 16 warps
+
+__global__ void __launch_bounds__(32 * FFG_NWARP, 1) ff_gemm_kernel(const __grid_constant__ FfGemmParams p) {
+  constexpr int NTN = FFG_NTN, NWARP = FFG_NWARP, NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP;
+  constexpr int STAGE_F = ROWS * BWD_LD, TILE = BWD_TM * BP, ITER = ROWS * 32 / NT;
+  constexpr int BPP = BP + 1, TILEP = BWD_TM * BPP;   // partial tiles padded: conflict-free column reads
+  static_assert(ROWS * 32 % NT == 0, "the staged tile divides evenly among the threads");
+  pdl_launch_dependents();
+  const int tile_row0 = blockIdx.x * BWD_TM;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  extern __shared__ float4 s_dyn[];
+  float* const s_tiles = reinterpret_cast<float*>(s_dyn);   // [BWD_STAGES][ROWS][BWD_LD]; later [NWARP][32][BP]
+  const int M = p.n_steps * p.B, it_all = (p.K + 127) / 128;
+  const int rlast = p.N - 1;
+  pdl_wait();
+  for (int bp0 = 0; bp0 < M; bp0 += BP) {
+    const float* src[ITER];
+    int dst_off[ITER], kcol[ITER];
+#pragma unroll
+    for (int j = 0; j < ITER; ++j) {
+      const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
+      kcol[j] = 4 * c4;
+      dst_off[j] = rr * BWD_LD + 4 * c4;
+      if (rr < BWD_TM) {   // rows and pairs past the end are clamped to the last valid one; never stored
+        const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;
+        src[j] = p.W + row * p.K + 4 * c4;
+      } else {
+        const int m = bp0 + rr - BWD_TM < M - 1 ? bp0 + rr - BWD_TM : M - 1;
+        src[j] = p.delta0 + (size_t)(m / p.B) * p.slot_stride + (size_t)(m % p.B) * p.K + 4 * c4;
+      }
+    }
+    auto issue = [&](int it) {
+      if (it < it_all) {
+        const int k0 = it * 128;
+        float* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
+#pragma unroll
+        for (int j = 0; j < ITER; ++j) {
+          if (k0 + kcol[j] < p.K) cp_async16(st + dst_off[j], src[j] + k0);
+          else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+      cp_async_commit();
+    };
+    float acc[2][NTN][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+    for (int it = 0; it < BWD_STAGES - 1; ++it) issue(it);
+    for (int it = 0; it < it_all; ++it) {
+      cp_async_wait<BWD_STAGES - 2>();
+      __syncthreads();
+      issue(it + BWD_STAGES - 1);
+      const float* Ws = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
+      const float* Ds = Ws + BWD_TM * BWD_LD;
+#pragma unroll 1
+      for (int ks = warp; ks < 16; ks += NWARP) {
+        const int kk = ks * 8 + t;
+        uint32_t a_hi[2][4], a_lo[2][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const float* r0 = Ws + (mt * 16 + g) * BWD_LD + kk;
+          split_tf32(r0[0], a_hi[mt][0], a_lo[mt][0]);
+          split_tf32(r0[8 * BWD_LD], a_hi[mt][1], a_lo[mt][1]);
+          split_tf32(r0[4], a_hi[mt][2], a_lo[mt][2]);
+          split_tf32(r0[8 * BWD_LD + 4], a_hi[mt][3], a_lo[mt][3]);
+        }
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) {
+          uint32_t b_hi[2], b_lo[2];
+          const float* r0 = Ds + (nt * 8 + g) * BWD_LD + kk;
+          split_tf32(r0[0], b_hi[0], b_lo[0]);
+          split_tf32(r0[4], b_hi[1], b_lo[1]);
+          mma_tf32(acc[0][nt], a_lo[0], b_hi); mma_tf32(acc[1][nt], a_lo[1], b_hi);
+          mma_tf32(acc[0][nt], a_hi[0], b_lo); mma_tf32(acc[1][nt], a_hi[1], b_lo);
+          mma_tf32(acc[0][nt], a_hi[0], b_hi); mma_tf32(acc[1][nt], a_hi[1], b_hi);
+        }
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();   // the stages are free: they now hold the warps' partial tiles [NWARP][32][BP]
+    {
+      float* mine = s_tiles + (size_t)warp * TILEP;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) {
+          const int r = mt * 16 + g, c = nt * 8 + 2 * t;
+          mine[r * BPP + c] = acc[mt][nt][0];       mine[r * BPP + c + 1] = acc[mt][nt][1];
+          mine[(r + 8) * BPP + c] = acc[mt][nt][2]; mine[(r + 8) * BPP + c + 1] = acc[mt][nt][3];
+        }
+    }
+    __syncthreads();
+    // out[m][i]: consecutive threads take consecutive rows i of one pair m (coalesced stores)
+    for (int e = tid; e < TILE; e += NT) {
+      const int r = e % BWD_TM, c = e / BWD_TM;
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILEP + r * BPP + c];
+      const int i = tile_row0 + r, m = bp0 + c;
+      if (i < p.N && m < M) p.out[(size_t)m * p.N + i] = sum;
+    }
+    __syncthreads();   // before the next pass refills the stages
   }
 }
 

@@ -45,6 +45,7 @@ snn_status fail(snn_net* net, snn_status st, const char* fmt, ...) {
 }
 
 constexpr size_t ALIGN = 256;
+constexpr int BWD_RUN = 32;   // steps per run of the layer-by-layer backward pass
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
@@ -55,6 +56,8 @@ struct Layout {
   int words[MAXL + 1];
   size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
   size_t event_bytes, total;
+  size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets)
+  bool layer_major;      // backward goes layer by layer over runs of steps, with that product batched over time
   size_t tier2;          // DOUBLE_LOCAL: the second checkpoint tier, in device memory
   int n_local, n_remote;
   bool tier2_on_device;
@@ -101,6 +104,15 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     lo.act[l] = (graded && l > 0) ? take(4 * (size_t)2 * B * sz[l]) : 0;
   }
   lo.event_bytes = cur - ev0;
+  {
+    // Networks whose weights do not stay in L2: streaming W_ff once per run of steps instead of once per
+    // step pays for giving up the layer wavefront in the backward pass.  A function of the sizes only.
+    size_t wbytes = 0;
+    int maxN = 0;
+    for (int l = 1; l <= L; ++l) { wbytes += 4 * ((size_t)sz[l - 1] * sz[l] + (size_t)sz[l] * sz[l]); maxN = std::max(maxN, sz[l]); }
+    lo.layer_major = L > 1 && wbytes > ((size_t)96 << 20);
+    lo.gff = L > 1 ? take(4 * (size_t)BWD_RUN * B * maxN) : 0;
+  }
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
   lo.tier2_on_device = ck->strategy == SNN_DOUBLE_LOCAL;
   lo.tier2 = lo.tier2_on_device ? take((size_t)lo.n_remote * lo.state_bytes) : 0;
@@ -408,8 +420,8 @@ struct Exec {
   }
   // dynamic shared memory of bwd_step_kernel for BP samples per pass: the staged tiles
   static size_t bwd_smem_bytes(int bp) { return (size_t)BWD_STAGES * (BWD_TM + bp) * BWD_LD * sizeof(float); }
-  template <int NTN, int NWARP> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS) {
-    return launch_pdl(bwd_step_kernel<NTN, NWARP>, dim3(tiles * CS, 1, L), dim3(32 * NWARP),
+  template <int NTN, int NWARP> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS, int n_layers = 0) {
+    return launch_pdl(bwd_step_kernel<NTN, NWARP>, dim3(tiles * CS, 1, n_layers ? n_layers : L), dim3(32 * NWARP),
                       bwd_smem_bytes(8 * NTN), p, CS);
   }
 
@@ -434,6 +446,53 @@ struct Exec {
     int CS = 1;
     while (CS < 8 && tiles * L * CS * 2 <= wave && minN / (4 * CS * 2) >= 32) CS *= 2;
     int span = begin_span(SNN_PHASE_BWD);
+    const bool layer_major = L > 1 && ((a->flags & SNN_FLAG_BACKWARD_LAYER_BY_LAYER) ||
+                                       (lo.layer_major && !(a->flags & SNN_FLAG_BACKWARD_WAVEFRONT)));
+    if (layer_major) {
+      // Runs of at most BWD_RUN steps, latest first; within a run the layers go from the last to the first:
+      // the feed-forward term of layer l for the whole run is one product (ff_gemm_kernel), then the steps
+      // of layer l follow one launch each.
+      for (int hi = n; hi > 0; hi -= BWD_RUN) {
+        const int lo_s = std::max(0, hi - BWD_RUN);     // steps t0+lo_s+1 .. t0+hi
+        for (int l = L; l >= 1; --l) {
+          if (l < L) {
+            FfGemmParams gp;
+            gp.W = a->W_ff[l]; gp.N = sz[l]; gp.K = sz[l + 1]; gp.B = B; gp.n_steps = hi - lo_s;
+            gp.delta0 = slot(op.buf_slot + lo_s, l + 1); gp.slot_stride = lo.state_bytes / 4;
+            gp.out = at<float>(lo.gff);
+            end_span(span);
+            span = begin_span(SNN_PHASE_FFGEMM);
+            CUDA_TRY(launch_pdl(ff_gemm_kernel, dim3((sz[l] + BWD_TM - 1) / BWD_TM), dim3(32 * FFG_NWARP),
+                                bwd_smem_bytes(8 * FFG_NTN), gp));
+            ++launches;
+            end_span(span);
+            span = begin_span(SNN_PHASE_BWD);
+          }
+          const int tiles_l = (sz[l] + BWD_TM - 1) / BWD_TM;
+          int CS_l = 1;
+          while (CS_l < 8 && tiles_l * CS_l * 2 <= wave && sz[l] / (4 * CS_l * 2) >= 32) CS_l *= 2;
+          for (int ts = hi - 1; ts >= lo_s; --ts) {
+            const int t = op.t0 + ts + 1;
+            std::memset(&p.lay[0], 0, sizeof p.lay[0]);
+            BwdLayer& f = p.lay[0];
+            f.mode = 1;
+            f.N = sz[l]; f.N_post = 0;
+            f.W_rec = a->W_rec[l - 1];
+            f.V_delta = slot(op.buf_slot + ts, l);
+            f.d_next = t == op.t1 ? carry(carry_cur, l) : slot(op.buf_slot + ts + 1, l);
+            f.g_out = l == L ? at<float>(lo.g_out) : nullptr;
+            f.g_ff = l < L ? at<float>(lo.gff) + (size_t)(ts - lo_s) * B * sz[l] : nullptr;
+            f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
+            cudaError_t le;
+            if (B <= 8) le = launch_bwd<1, 8>(p, tiles_l, CS_l, 1);
+            else if (B <= 16) le = launch_bwd<2, 8>(p, tiles_l, CS_l, 1);
+            else le = launch_bwd<4, 16>(p, tiles_l, CS_l, 1);
+            if (le != cudaSuccess) return fail(net, SNN_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(le));
+            ++launches;
+          }
+        }
+      }
+    } else
     for (int s = 0; s <= n + L - 2; ++s) {
       for (int l = L; l >= 1; --l) {
         BwdLayer& f = p.lay[l - 1];
@@ -597,6 +656,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(16)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(32)));

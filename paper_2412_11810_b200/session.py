@@ -81,7 +81,8 @@ class Session:
     # ---- the training step -----------------------------------------------------------------
     def train_step(self, input_bits, targets, strategy: int = sb.SNN_STANDARD, chunk_size: int = 0,
                    remote_chunk_size: int = 0, max_activity: float = 0.25, forward_only: bool = False,
-                   keep_V: bool = False, time_phases: bool = False, nb_local: int = 0) -> float:
+                   keep_V: bool = False, time_phases: bool = False, nb_local: int = 0,
+                   extra_flags: int = 0) -> float:
         """input_bits: uint32 [T][B][ceil(N_0/32)] spike words (LIF cell; int32 storage) or float32
         [T][B][N_0] dense values (graded cell), as a CUDA tensor or as a pinned host tensor / numpy
         array (then it is copied to the device inside the call); targets alike."""
@@ -97,7 +98,7 @@ class Session:
         ck = self.ckpt(strategy, chunk_size, remote_chunk_size, nb_local)
         self.ensure_workspace(T, B, ck, max_activity)
         flags = (sb.SNN_FLAG_INPUT_ON_HOST if on_host else 0) | (sb.SNN_FLAG_FORWARD_ONLY if forward_only else 0) \
-            | (sb.SNN_FLAG_TIME_PHASES if time_phases else 0)
+            | (sb.SNN_FLAG_TIME_PHASES if time_phases else 0) | extra_flags
         dbg = None
         if keep_V:
             self.debug_V = [torch.zeros((T + 1, B, self.sizes[l + 1]), dtype=torch.float32, device=self.device)

@@ -377,3 +377,27 @@ def test_batch_sizes_outside_the_backward_tiles(orc32, B):
     for a, b in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
         assert np.array_equal(a, b)
     s.close()
+
+
+def test_layer_by_layer_backward_order(orc32):
+    """The launch order used for large networks (feed-forward term of a run of steps as one product),
+    forced here on a small one: same gradients within tolerance, and all strategies bit-identical to
+    STANDARD under that order; runs longer and shorter than 32 steps."""
+    b = sb()
+    w = wl.small(sizes=(96, 640, 516, 260, 12), T=71, B=11, p_in=0.06, g_ff=(2.5, 1.5, 1.5), g_rec=(1.0, 1.0, 1.0), seed=41)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    assert all(0.005 < float(x[1:].mean()) < 0.5 for x in ref["S"])
+    s, bits, targets = make_session(w, d)
+    f = b.SNN_FLAG_BACKWARD_LAYER_BY_LAYER
+    s.train_step(bits, targets, strategy=0, extra_flags=f)
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 9, 0), (1, 40, 0), (2, 33, 0), (3, 4, 16), (3, 1, 3)]:
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, extra_flags=f)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R)
+    # the wavefront order agrees within tolerance (different summation, not bit-identical)
+    s.train_step(bits, targets, strategy=1, chunk_size=9, extra_flags=b.SNN_FLAG_BACKWARD_WAVEFRONT)
+    assert_grads_close(s.gradients(), ref)
+    s.close()
