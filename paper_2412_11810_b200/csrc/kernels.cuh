@@ -749,7 +749,8 @@ __global__ void __launch_bounds__(32 * FFG_NWARP, 1) ff_gemm_kernel(const __grid
   const int M = p.n_steps * p.B, it_all = (p.K + 127) / 128;
   const int rlast = p.N - 1;
   pdl_wait();
-  for (int bp0 = 0; bp0 < M; bp0 += BP) {
+  {   // one pass of 64 (step, sample) pairs per CTA: blockIdx.y selects it
+    const int bp0 = blockIdx.y * BP;
     const float* src[ITER];
     int dst_off[ITER], kcol[ITER];
 #pragma unroll
@@ -838,7 +839,6 @@ __global__ void __launch_bounds__(32 * FFG_NWARP, 1) ff_gemm_kernel(const __grid
       const int i = tile_row0 + r, m = bp0 + c;
       if (i < p.N && m < M) p.out[(size_t)m * p.N + i] = sum;
     }
-    __syncthreads();   // before the next pass refills the stages
   }
 }
 
