@@ -128,6 +128,16 @@ snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const s
  * Gradients are bit-identical across strategies for a given order, not between the two orders. */
 #define SNN_FLAG_BACKWARD_LAYER_BY_LAYER 8u
 #define SNN_FLAG_BACKWARD_WAVEFRONT 16u
+/* The recomputation passes run as one launch per segment while the weights fit in L2 (each CTA walks
+ * through the segment's steps from the stored events); this flag forces one launch per step, the
+ * order used for larger networks.  Results are bit-identical either way. */
+#define SNN_FLAG_REFORWARD_PER_STEP 32u
+/* The forward pass of a spiking (LIF) network whose weights fit in L2 runs as one cooperative launch per
+ * forward operation of the plan when the device can hold all its thread blocks at once: blocks wait for
+ * each other's spike words sample by sample instead of once per launch.  This flag forces one launch per
+ * step.  Results are bit-identical either way.  A wait that does not end within a few seconds makes the
+ * step return SNN_ERR_DEVICE_TIMEOUT. */
+#define SNN_FLAG_FORWARD_PER_STEP 64u
 
 typedef struct {
   int32_t T, B;

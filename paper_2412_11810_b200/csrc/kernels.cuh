@@ -459,6 +459,395 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
 }
 
 // ------------------------------------------------------------------------------------------
+// Re-forward of a whole segment of steps in one launch (the recomputation passes of Sec. 3).
+//
+// Once the forward pass has stored the events of every step, V_t of a neuron depends on nothing
+// but its own V_{t-1} and those lists: no CTA needs another CTA's result.  A CTA therefore keeps
+// the state of its 512 neurons of one sample in registers and walks through all steps of the
+// segment: the lists of consecutive steps are laid end to end in shared memory (each padded to a
+// whole number of copy groups; a padding entry is a zero-filled copy, and adding +0 leaves an
+// fp32 sum unchanged), so the ring of row copies never drains at a step boundary.  Per step the
+// arithmetic is that of fwd_step_kernel, operation for operation.
+struct SegLayer {
+  const float* W_ff;          // [N_pre][N]
+  const float* W_rec;         // [N][N]
+  const uint32_t* ff_pool;    // event pool of the layer below [B][ff_cap]
+  const uint32_t* ff_off;     // its offsets, row 0: list (t, b) = [off[t * B + b], off[(t + 1) * B + b])
+  const uint32_t* rec_pool;   // own event pool [B][rec_cap]
+  const uint32_t* rec_off;    // own offsets, row 0
+  const float* ff_vals;       // graded cell: values that go with ff_pool
+  const float* rec_vals;      // graded cell: values that go with rec_pool
+  const uint32_t* mask0;      // [B][W] own spike words at the segment's first state (step t0)
+  size_t state_off;           // offset of this layer inside a state slot, in floats
+  uint32_t ff_cap, rec_cap;
+  int N, W;
+};
+
+struct SegParams {
+  SegLayer lay[MAXL];
+  float* slots;               // state slot s starts at slots + s * slot_stride
+  size_t slot_stride;         // floats
+  int B, t0, t1;              // steps t0+1 .. t1 are computed from the state of step t0
+  int in_slot, buf_slot, buf_len, keep_every, keep_slot;   // as in snn_op
+  float alpha, theta;
+};
+
+constexpr int SEG_STEPS = 32;                          // steps whose list bounds are staged at a time
+constexpr int SEG_GROUPS = LIST_CHUNK / GATHER_ROWS;   // copy groups per window of the merged list
+
+__device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* gmem_src, bool real) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gmem_src), "r"(real ? 16u : 0u) : "memory");
+}
+
+template <bool GRADED>
+__global__ void __launch_bounds__(FWD_THREADS) refwd_segment_kernel(const __grid_constant__ SegParams p) {
+  pdl_launch_dependents();
+  const SegLayer& L = p.lay[blockIdx.z];
+  const int col0 = blockIdx.x * FWD_COLS;
+  if (col0 >= L.N) return;
+  const int b = blockIdx.y, B = p.B, tid = threadIdx.x;
+  __shared__ const float* s_row[LIST_CHUNK];   // listed weight rows at this CTA's first column, null = padding
+  __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
+  __shared__ uint32_t s_offF[SEG_STEPS + 1], s_offR[SEG_STEPS + 1];
+  __shared__ int s_gstart[SEG_STEPS + 1];      // first copy group of each step of the window
+  __shared__ int s_plan[2];                    // steps in the window (0: part of one long step), groups
+  __shared__ uint8_t s_glast[SEG_GROUPS];      // group ends a step
+  extern __shared__ float4 s_stage[];          // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
+  const int col = col0 + tid * 4;
+  const bool active = col < L.N;
+  const float* const Wff_tile = L.W_ff + col0;
+  const float* const Wrec_tile = L.W_rec + col0;
+  const uint32_t* const ff_pool = L.ff_pool + (size_t)b * L.ff_cap;
+  const uint32_t* const rec_pool = L.rec_pool + (size_t)b * L.rec_cap;
+  float* const state = p.slots + L.state_off + (size_t)b * L.N + col;
+
+  pdl_wait();
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  uint32_t sp = 0;   // spikes of the four neurons at the previous step
+  if (active) {
+    v = *reinterpret_cast<const float4*>(state + (size_t)p.in_slot * p.slot_stride);
+    if (!GRADED) sp = (L.mask0[(size_t)b * L.W + (col >> 5)] >> (col & 31)) & 15u;
+  }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  int t = p.t0 + 1;        // first step of the next window
+  int t_cur = t;           // step whose events this thread is adding
+  uint32_t e_skip = 0;     // events of step t that earlier windows already took
+
+  while (t <= p.t1) {
+    const int ns_try = min(SEG_STEPS, p.t1 - t + 1);
+    __syncthreads();
+    if (tid <= ns_try) {
+      s_offF[tid] = L.ff_off[(size_t)(t + tid) * B + b];
+      s_offR[tid] = L.rec_off[(size_t)(t - 1 + tid) * B + b];
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int ns = 0, g_tot = 0;
+      for (int j = 0; j < ns_try; ++j) {
+        uint32_t n_j = (s_offF[j + 1] - s_offF[j]) + (s_offR[j + 1] - s_offR[j]);
+        if (j == 0) n_j -= e_skip;
+        const int g_j = n_j == 0 ? 1 : (int)((n_j + GATHER_ROWS - 1) / GATHER_ROWS);
+        if (g_tot + g_j > SEG_GROUPS) break;
+        s_gstart[j] = g_tot;
+        g_tot += g_j;
+        ns = j + 1;
+      }
+      if (ns == 0) { s_gstart[0] = 0; g_tot = SEG_GROUPS; }   // one step longer than a window: take a part
+      s_gstart[ns == 0 ? 1 : ns] = g_tot;
+      s_plan[0] = ns; s_plan[1] = g_tot;
+    }
+    __syncthreads();
+    const int ns = s_plan[0], g_tot = s_plan[1];
+    {
+      int j = 0;
+      for (int i = tid; i < g_tot * GATHER_ROWS; i += FWD_THREADS) {
+        const int g = i / GATHER_ROWS;
+        while (j + 1 < ns && s_gstart[j + 1] <= g) ++j;
+        const uint32_t e = (uint32_t)(g - s_gstart[j]) * GATHER_ROWS + (i % GATHER_ROWS) + (j == 0 ? e_skip : 0u);
+        const uint32_t n_ff = s_offF[j + 1] - s_offF[j], n_all = n_ff + (s_offR[j + 1] - s_offR[j]);
+        const float* row = nullptr;
+        float val = 0.f;
+        if (e < n_ff) {
+          const uint32_t q = s_offF[j] + e;
+          row = Wff_tile + (size_t)ff_pool[q] * L.N;
+          if (GRADED) val = L.ff_vals[(size_t)b * L.ff_cap + q];
+        } else if (e < n_all) {
+          const uint32_t q = s_offR[j] + (e - n_ff);
+          row = Wrec_tile + (size_t)rec_pool[q] * L.N;
+          if (GRADED) val = L.rec_vals[(size_t)b * L.rec_cap + q];
+        }
+        s_row[i] = row;
+        if (GRADED) s_val[i] = val;
+        if (i % GATHER_ROWS == 0) s_glast[g] = (ns > 0 && g + 1 == s_gstart[j + 1]) ? 1 : 0;
+      }
+    }
+    __syncthreads();
+    if (active) {
+      float4* const ring = s_stage + tid;
+      const int lane_col = tid * 4;
+      auto issue = [&](int g) {
+        if (g < g_tot) {
+          float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+          const float* const* rows = s_row + g * GATHER_ROWS;
+#pragma unroll
+          for (int u = 0; u < GATHER_ROWS; ++u) {
+            const float* r = rows[u];
+            cp_async16_or_zero(dst + u * FWD_THREADS, r ? r + lane_col : Wff_tile, r != nullptr);
+          }
+        }
+        cp_async_commit();
+      };
+      for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
+      for (int g = 0; g < g_tot; ++g) {
+        issue(g + GATHER_STAGES - 1);
+        cp_async_wait<GATHER_STAGES - 1>();
+        const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+#pragma unroll
+        for (int u = 0; u < GATHER_ROWS; ++u) {
+          const float4 w = src[u * FWD_THREADS];
+          if (GRADED) {
+            const float sv = s_val[g * GATHER_ROWS + u];
+            acc.x = __fmaf_rn(sv, w.x, acc.x); acc.y = __fmaf_rn(sv, w.y, acc.y);
+            acc.z = __fmaf_rn(sv, w.z, acc.z); acc.w = __fmaf_rn(sv, w.w, acc.w);
+          } else {
+            acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+            acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+          }
+        }
+        if (s_glast[g]) {   // the step's lists are through: leak, reset, store
+          if (GRADED) {
+            v.x = __fmaf_rn(p.alpha, v.x, acc.x); v.y = __fmaf_rn(p.alpha, v.y, acc.y);
+            v.z = __fmaf_rn(p.alpha, v.z, acc.z); v.w = __fmaf_rn(p.alpha, v.w, acc.w);
+          } else {
+            v.x = __fsub_rn(__fmaf_rn(p.alpha, v.x, acc.x), __fmul_rn(p.theta, (float)(sp & 1u)));
+            v.y = __fsub_rn(__fmaf_rn(p.alpha, v.y, acc.y), __fmul_rn(p.theta, (float)((sp >> 1) & 1u)));
+            v.z = __fsub_rn(__fmaf_rn(p.alpha, v.z, acc.z), __fmul_rn(p.theta, (float)((sp >> 2) & 1u)));
+            v.w = __fsub_rn(__fmaf_rn(p.alpha, v.w, acc.w), __fmul_rn(p.theta, (float)((sp >> 3) & 1u)));
+            sp = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) |
+                 (v.w > p.theta ? 8u : 0u);
+          }
+          const int d = t_cur - p.t0;
+          *reinterpret_cast<float4*>(state + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = v;
+          if (p.keep_every > 0 && d % p.keep_every == 0)
+            *reinterpret_cast<float4*>(state + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = v;
+          acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          ++t_cur;
+        }
+      }
+      cp_async_wait<0>();
+    }
+    if (ns == 0) e_skip += SEG_GROUPS * GATHER_ROWS;
+    else { e_skip = 0; t += ns; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Forward pass over a whole segment of steps in one cooperative launch (LIF cell).
+//
+// Unlike the recomputation above the spikes are not known yet, so a CTA (column tile, sample b,
+// layer l) can start step t only when the spike words of (l, t-1, b) and (l-1, t, b) are complete.
+// These are the only dependences: samples never wait for one another and a lower layer may run
+// ahead of a higher one.  Each (layer, sample) has a counter of finished (tile, step) pairs; a
+// producer publishes its words with a fence and an atomic add, a consumer polls the counter with
+// acquire loads and then reads the words past L1.  Every buffer a step writes is indexed by the
+// step or owned by the writing thread, so running ahead overwrites nothing that is still needed.
+// All CTAs must be resident together (cooperative launch); a wait that does not end within
+// SYNC_POLL_LIMIT polls raises STATUS_SYNC_TIMEOUT and the CTA returns.
+constexpr uint32_t STATUS_SYNC_TIMEOUT = 2u;
+constexpr uint32_t SYNC_POLL_LIMIT = 1u << 22;   // a few seconds
+constexpr int SEG_WORDS = 1024;                  // spike words of both sources of a layer, staged per step
+
+struct FwdSegLayer {
+  const float* W_ff;          // [N_pre][N]
+  const float* W_rec;         // [N][N]
+  const uint32_t* ff_words;   // spike words of the layer below; row of step t at (t - ff_row0) * B * W_pre
+  uint32_t* words;            // own spike words [T+1][B][W]
+  uint32_t* ff_pool;          // event pool of the layer below [B][ff_cap] (written here if write_ff_list)
+  uint32_t* ff_off;           // its offsets, row 0
+  uint32_t* rec_pool;         // own event pool [B][rec_cap]
+  uint32_t* rec_off;          // own offsets, row 0
+  uint32_t* counts;           // [B][N] spike counts (last layer) or null
+  float* V_dbg;               // [T+1][B][N] copy of every state, or null
+  size_t state_off;           // offset of this layer inside a state slot, in floats
+  uint32_t ff_cap, rec_cap;
+  int N_pre, N, W_pre, W;
+  int ff_row0;                // 1 for the input (its rows start at step 1), 0 for hidden layers
+  int write_ff_list;          // the layer below is the input: this layer stores its lists
+  int tiles;                  // column tiles (CTAs per sample) of this layer
+};
+
+struct FwdSegParams {
+  FwdSegLayer lay[MAXL];
+  float* slots;
+  size_t slot_stride;         // floats
+  uint32_t* status;
+  uint32_t* progress;         // [L][B] finished (tile, step) pairs, zero at launch
+  int B, t0, t1;
+  int in_slot, buf_slot, buf_len, keep_every, keep_slot;
+  float alpha, theta;
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ bool wait_progress(const uint32_t* counter, uint32_t target) {
+  for (uint32_t i = 0; i < SYNC_POLL_LIMIT; ++i) {
+    if (ld_acquire_gpu(counter) >= target) return true;
+    if (i > 32) __nanosleep(64);
+  }
+  return false;
+}
+
+__global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_constant__ FwdSegParams p) {
+  const int l = blockIdx.z;
+  const FwdSegLayer& L = p.lay[l];
+  const int col0 = blockIdx.x * FWD_COLS;
+  if (col0 >= L.N) return;
+  const int b = blockIdx.y, B = p.B, tid = threadIdx.x;
+  const bool tile0 = blockIdx.x == 0;
+  __shared__ const float* s_row[LIST_CHUNK];
+  __shared__ uint32_t s_words[SEG_WORDS];
+  __shared__ uint32_t s_pref[SEG_WORDS + 1];
+  __shared__ uint32_t s_warp[FWD_THREADS / 32];
+  __shared__ int s_ok;
+  extern __shared__ float4 s_stage[];   // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
+  const int col = col0 + tid * 4;
+  const bool active = col < L.N;
+  const float* const Wff_tile = L.W_ff + col0;
+  const float* const Wrec_tile = L.W_rec + col0;
+  uint32_t* const ff_pool = L.ff_pool + (size_t)b * L.ff_cap;
+  uint32_t* const rec_pool = L.rec_pool + (size_t)b * L.rec_cap;
+  float* const state = p.slots + L.state_off + (size_t)b * L.N + col;
+  uint32_t* const my_progress = p.progress + (size_t)l * B + b;
+  const uint32_t* const below_progress = l > 0 ? p.progress + (size_t)(l - 1) * B + b : nullptr;
+  const uint32_t below_tiles = l > 0 ? (uint32_t)p.lay[l - 1].tiles : 0u;
+
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (active) v = *reinterpret_cast<const float4*>(state + (size_t)p.in_slot * p.slot_stride);
+  // where the next lists go in the pools (this CTA is the only writer of its sample's pools)
+  uint32_t rec_end = 0, ff_end = 0;
+  if (tile0) {
+    rec_end = L.rec_off[(size_t)p.t0 * B + b];
+    if (L.write_ff_list) ff_end = L.ff_off[(size_t)(p.t0 + 1) * B + b];
+  }
+
+  for (int t = p.t0 + 1; t <= p.t1; ++t) {
+    const uint32_t d = (uint32_t)(t - p.t0);
+    if (tid == 0) {
+      bool ok = wait_progress(my_progress, (uint32_t)L.tiles * (d - 1));
+      if (ok && l > 0) ok = wait_progress(below_progress, below_tiles * d);
+      if (!ok) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+      s_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_ok) return;
+    {
+      const uint32_t* ffw = L.ff_words + ((size_t)(t - L.ff_row0) * B + b) * L.W_pre;
+      const uint32_t* recw = L.words + ((size_t)(t - 1) * B + b) * L.W;
+      for (int w = tid; w < L.W_pre + L.W; w += FWD_THREADS)
+        s_words[w] = __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre));
+    }
+    __syncthreads();
+    const WordPair wp{s_words, L.W_pre, s_words + L.W_pre, L.W};
+    const uint32_t total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
+    const uint32_t n_ff = s_pref[L.W_pre];
+    const uint32_t pw = active ? s_words[L.W_pre + (col >> 5)] >> (col & 31) : 0u;
+    if (tile0) {   // append the two lists to the event pools
+      const bool wr_ff = L.write_ff_list != 0;
+      const uint32_t room_ff = wr_ff ? L.ff_cap - ff_end : 0u, room_rec = L.rec_cap - rec_end;
+      write_lists_from_words<FWD_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + ff_end : nullptr, room_ff,
+                                                 rec_pool + rec_end, room_rec);
+      const uint32_t n_rec = total - n_ff;
+      rec_end += n_rec < room_rec ? n_rec : room_rec;
+      if (wr_ff) ff_end += n_ff < room_ff ? n_ff : room_ff;
+      if (tid == 0) {
+        L.rec_off[(size_t)t * B + b] = rec_end;
+        if (wr_ff) L.ff_off[(size_t)(t + 1) * B + b] = ff_end;
+        if (n_rec > room_rec || (wr_ff && n_ff > room_ff)) atomicOr(p.status, STATUS_EVENT_OVERFLOW);
+      }
+    }
+
+    // gather-accumulate in list order: feed-forward events, then recurrent events
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
+      const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
+      fill_rows_from_words<FWD_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
+      __syncthreads();
+      if (active) {
+        float4* const ring = s_stage + tid;
+        const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
+        const int lane_col = tid * 4;
+        auto issue = [&](int g) {
+          if (g < n_groups) {
+            float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+            const float* const* rows = s_row + g * GATHER_ROWS;
+#pragma unroll
+            for (int u = 0; u < GATHER_ROWS; ++u) {
+              const bool real = g * GATHER_ROWS + u < n;
+              cp_async16_or_zero(dst + u * FWD_THREADS, real ? rows[u] + lane_col : Wff_tile, real);
+            }
+          }
+          cp_async_commit();
+        };
+        for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
+        for (int g = 0; g < n_groups; ++g) {
+          issue(g + GATHER_STAGES - 1);
+          cp_async_wait<GATHER_STAGES - 1>();
+          const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+#pragma unroll
+          for (int u = 0; u < GATHER_ROWS; ++u) {   // rows past the list's end were zero-filled: +0 changes nothing
+            const float4 w = src[u * FWD_THREADS];
+            acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+            acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+          }
+        }
+        cp_async_wait<0>();
+      }
+      __syncthreads();
+    }
+
+    // leak, reset by subtraction of the previous step's own spike, threshold
+    uint32_t nib = 0;
+    if (active) {
+      v.x = __fsub_rn(__fmaf_rn(p.alpha, v.x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
+      v.y = __fsub_rn(__fmaf_rn(p.alpha, v.y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
+      v.z = __fsub_rn(__fmaf_rn(p.alpha, v.z, acc.z), __fmul_rn(p.theta, (float)((pw >> 2) & 1u)));
+      v.w = __fsub_rn(__fmaf_rn(p.alpha, v.w, acc.w), __fmul_rn(p.theta, (float)((pw >> 3) & 1u)));
+      *reinterpret_cast<float4*>(state + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = v;
+      if (p.keep_every > 0 && d % p.keep_every == 0)
+        *reinterpret_cast<float4*>(state + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = v;
+      if (L.V_dbg) *reinterpret_cast<float4*>(L.V_dbg + ((size_t)t * B + b) * L.N + col) = v;
+      nib = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) |
+            (v.w > p.theta ? 8u : 0u);
+      if (L.counts && nib) {
+        uint4* c = reinterpret_cast<uint4*>(L.counts + (size_t)b * L.N + col);
+        uint4 cv = *c;
+        cv.x += nib & 1u; cv.y += (nib >> 1) & 1u; cv.z += (nib >> 2) & 1u; cv.w += (nib >> 3) & 1u;
+        *c = cv;
+      }
+    }
+    {   // eight neighbouring lanes hold the 32 bits of one spike word
+      const int lane = tid & 31;
+      uint32_t word = nib << (4 * (lane & 7));
+      word |= __shfl_xor_sync(0xffffffffu, word, 1);
+      word |= __shfl_xor_sync(0xffffffffu, word, 2);
+      word |= __shfl_xor_sync(0xffffffffu, word, 4);
+      const int widx = col >> 5;
+      if ((lane & 7) == 0 && widx < L.W) L.words[((size_t)t * B + b) * L.W + widx] = word;
+    }
+    __syncthreads();
+    if (tid == 0) {   // publish: this tile's words of step t are complete
+      __threadfence();
+      atomicAdd(my_progress, 1u);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Backward step: delta^l_t = g_S sigma'(V^l_t - theta) + alpha delta^l_{t+1}, with
 // g_S = g_out + W_ff^{l+1} delta^{l+1}_t + W_rec^l delta^l_{t+1} - theta delta^l_{t+1}.
 //

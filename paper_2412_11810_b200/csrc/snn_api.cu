@@ -28,6 +28,7 @@ struct snn_net {
   std::vector<cudaEvent_t> copy_events;    // one per checkpoint copy in flight, grown on demand
   std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
   snn_phase_times phases{};
+  int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
 };
 
 namespace {
@@ -49,7 +50,7 @@ constexpr int BWD_RUN = 32;   // steps per run of the layer-by-layer backward pa
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-  size_t status, logits, dlogits, g_out, counts, carry[2], in_stage, tg_stage;
+  size_t status, progress, logits, dlogits, g_out, counts, carry[2], in_stage, tg_stage;
   size_t off[MAXL + 1], pool[MAXL + 1], mask[MAXL + 1];
   size_t vals[MAXL + 1], pref[MAXL + 1], act[MAXL + 1], in_words;   // graded cell only
   uint32_t cap[MAXL + 1];
@@ -58,6 +59,7 @@ struct Layout {
   size_t event_bytes, total;
   size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets)
   bool layer_major;      // backward goes layer by layer over runs of steps, with that product batched over time
+  bool weights_resident; // all weight matrices together stay in L2
   size_t tier2;          // DOUBLE_LOCAL: the second checkpoint tier, in device memory
   int n_local, n_remote;
   bool tier2_on_device;
@@ -79,6 +81,7 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   for (int l = 1; l <= L; ++l) { lo.layer_off[l] = (size_t)B * sumN; sumN += sz[l]; }
   lo.state_bytes = 4 * (size_t)B * sumN;
   lo.status = take(256);
+  lo.progress = take(4 * (size_t)MAXL * B);   // per (layer, sample): finished (tile, step) pairs of a forward launch
   lo.logits = take(4 * (size_t)B * N_out);
   lo.dlogits = take(4 * (size_t)B * N_out);
   lo.g_out = take(4 * (size_t)B * N_L);
@@ -110,7 +113,8 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     size_t wbytes = 0;
     int maxN = 0;
     for (int l = 1; l <= L; ++l) { wbytes += 4 * ((size_t)sz[l - 1] * sz[l] + (size_t)sz[l] * sz[l]); maxN = std::max(maxN, sz[l]); }
-    lo.layer_major = L > 1 && wbytes > ((size_t)96 << 20);
+    lo.weights_resident = wbytes <= ((size_t)96 << 20);
+    lo.layer_major = L > 1 && !lo.weights_resident;
     lo.gff = L > 1 ? take(4 * (size_t)BWD_RUN * B * maxN) : 0;
   }
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
@@ -352,12 +356,108 @@ struct Exec {
     return SNN_OK;
   }
 
+  // REFWD1 / REFWD2 as one launch: the stored events make every (sample, column tile, layer) independent,
+  // so each CTA walks through the segment's steps on its own.  Used while the weights stay in L2; beyond
+  // that the per-step launches keep the samples in step, and the rows they share are read from HBM once.
+  snn_status run_reforward_segment(const snn_op& op) {
+    SegParams p;
+    std::memset(&p, 0, sizeof p);
+    p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
+    p.B = B; p.t0 = op.t0; p.t1 = op.t1;
+    p.in_slot = op.in_slot; p.buf_slot = op.buf_slot; p.buf_len = op.buf_len;
+    p.keep_every = op.keep_every; p.keep_slot = op.keep_slot;
+    p.alpha = net->alpha; p.theta = net->theta;
+    for (int l = 1; l <= L; ++l) {
+      SegLayer& s = p.lay[l - 1];
+      s.W_ff = a->W_ff[l - 1]; s.W_rec = a->W_rec[l - 1];
+      s.ff_pool = pool(l - 1); s.ff_off = off(l - 1, 0); s.ff_cap = lo.cap[l - 1];
+      s.rec_pool = pool(l); s.rec_off = off(l, 0); s.rec_cap = lo.cap[l];
+      if (graded()) { s.ff_vals = vals(l - 1); s.rec_vals = vals(l); }
+      s.mask0 = mask(l, op.t0);
+      s.state_off = lo.layer_off[l];
+      s.N = net->sizes[l]; s.W = lo.words[l];
+    }
+    void (*k)(SegParams) = graded() ? refwd_segment_kernel<true> : refwd_segment_kernel<false>;
+    CUDA_TRY(launch_pdl(k, fwd_grid(), dim3(FWD_THREADS), FWD_DYN_SMEM, p));
+    ++launches;
+    CUDA_TRY(cudaGetLastError());
+    return SNN_OK;
+  }
+
+  // FWD as one cooperative launch per op: CTAs wait for the spike words they need, sample by sample
+  // (fwd_segment_kernel).  Possible when all CTAs of the grid are resident together.
+  bool forward_segment_possible() {
+    if (graded() || !lo.weights_resident || (a->flags & SNN_FLAG_FORWARD_PER_STEP)) return false;
+    for (int l = 1; l <= L; ++l)
+      if (lo.words[l - 1] + lo.words[l] > SEG_WORDS) return false;
+    if (net->fwd_segment_capacity < 0) {
+      int dev = 0, sms = 0, per_sm = 0, coop = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fwd_segment_kernel, FWD_THREADS, FWD_DYN_SMEM) != cudaSuccess) {
+        cudaGetLastError();
+        net->fwd_segment_capacity = 0;
+      } else {
+        net->fwd_segment_capacity = coop ? sms * per_sm : 0;
+      }
+    }
+    const dim3 g = fwd_grid();
+    return (long long)g.x * g.y * g.z <= net->fwd_segment_capacity;
+  }
+
+  snn_status run_forward_segment(const snn_op& op) {
+    FwdSegParams p;
+    std::memset(&p, 0, sizeof p);
+    p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
+    p.status = at<uint32_t>(lo.status); p.progress = at<uint32_t>(lo.progress);
+    p.B = B; p.t0 = op.t0; p.t1 = op.t1;
+    p.in_slot = op.in_slot; p.buf_slot = op.buf_slot; p.buf_len = op.buf_len;
+    p.keep_every = op.keep_every; p.keep_slot = op.keep_slot;
+    p.alpha = net->alpha; p.theta = net->theta;
+    for (int l = 1; l <= L; ++l) {
+      FwdSegLayer& s = p.lay[l - 1];
+      s.W_ff = a->W_ff[l - 1]; s.W_rec = a->W_rec[l - 1];
+      s.ff_words = l == 1 ? in_mask(1) : mask(l - 1, 0);
+      s.ff_row0 = l == 1 ? 1 : 0;
+      s.words = mask(l, 0);
+      s.ff_pool = pool(l - 1); s.ff_off = off(l - 1, 0); s.ff_cap = lo.cap[l - 1];
+      s.rec_pool = pool(l); s.rec_off = off(l, 0); s.rec_cap = lo.cap[l];
+      s.counts = l == L ? at<uint32_t>(lo.counts) : nullptr;
+      s.V_dbg = (a->debug_V && a->debug_V[l - 1]) ? a->debug_V[l - 1] : nullptr;
+      s.state_off = lo.layer_off[l];
+      s.N_pre = net->sizes[l - 1]; s.N = net->sizes[l]; s.W_pre = lo.words[l - 1]; s.W = lo.words[l];
+      s.write_ff_list = l == 1;
+      s.tiles = (net->sizes[l] + FWD_COLS - 1) / FWD_COLS;
+    }
+    CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L * B, main));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = fwd_grid(); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = FWD_DYN_SMEM; cfg.stream = main;
+    cudaLaunchAttribute at1[1];
+    at1[0].id = cudaLaunchAttributeCooperative;
+    at1[0].val.cooperative = 1;
+    cfg.attrs = at1; cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, fwd_segment_kernel, p));
+    ++launches;
+    return SNN_OK;
+  }
+
   // FWD / REFWD1 / REFWD2: layer wavefront, layer l runs l-1 steps behind layer 1.
   snn_status run_forward(const snn_op& op, bool gen) {
     if (wait_slot(op.in_slot) != SNN_OK || wait_slot(op.keep_slot) != SNN_OK) return SNN_ERR_CUDA;
     const int n = op.t1 - op.t0;
     const int span = begin_span(op.kind == SNN_OP_FWD ? SNN_PHASE_FWD
                                 : op.kind == SNN_OP_REFWD1 ? SNN_PHASE_REFWD1 : SNN_PHASE_REFWD2);
+    if (!gen && lo.weights_resident && !(a->flags & SNN_FLAG_REFORWARD_PER_STEP)) {
+      const snn_status st = run_reforward_segment(op);
+      end_span(span);
+      return st;
+    }
+    if (gen && forward_segment_possible()) {
+      const snn_status st = run_forward_segment(op);
+      end_span(span);
+      return st;
+    }
     FwdParams p;
     std::memset(&p, 0, sizeof p);
     p.B = B; p.alpha = net->alpha; p.theta = net->theta; p.status = at<uint32_t>(lo.status);
@@ -657,6 +757,9 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(refwd_segment_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(refwd_segment_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(16)));
@@ -763,6 +866,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = lo.vals[l]; e.pool_capacity = lo.cap[l];
     e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];
   }
+  if (host_status[0] & STATUS_SYNC_TIMEOUT)
+    return fail(net, SNN_ERR_DEVICE_TIMEOUT, "a thread block gave up waiting for the spikes of another one");
   if (host_status[0] & STATUS_EVENT_OVERFLOW)
     return fail(net, SNN_ERR_EVENT_OVERFLOW, "more events than max_activity=%g allows", (double)a->max_activity);
   return SNN_OK;

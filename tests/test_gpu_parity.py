@@ -59,10 +59,10 @@ def test_compaction_capacity_clamps(orc32):
 
 
 # ---------------------------------------------------------------- forward: membranes, spikes, events
-def _check_forward(orc32, w, d):
+def _check_forward(orc32, w, d, extra_flags=0):
     ref = run_oracle(orc32, w, d, do_backward=False)
     s, bits, targets = make_session(w, d)
-    loss = s.train_step(bits, targets, forward_only=True, keep_V=True, max_activity=1.0)
+    loss = s.train_step(bits, targets, forward_only=True, keep_V=True, max_activity=1.0, extra_flags=extra_flags)
     assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
     for l in range(w.L):
         V = s.debug_V[l].cpu().numpy()
@@ -94,6 +94,19 @@ def test_forward_ragged_sizes_bit_exact(orc32):
     w = wl.small(sizes=(70, 3000, 36, 7), T=9, B=2, p_in=0.5, g_ff=(3.0, 6.0), g_rec=(1.0, 1.0), seed=3)
     ref = _check_forward(orc32, w, wl.make(w))
     assert ref["S"][0][1:].mean() > 0.1
+
+
+def test_forward_one_launch_per_step_bit_exact(orc32):
+    """Small spiking networks run the forward pass as one cooperative launch per forward operation; the
+    launch-per-step kernel (the one large networks use) must give the same bits."""
+    f = sb().SNN_FLAG_FORWARD_PER_STEP
+    w = wl.small()
+    _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    w = wl.small(sizes=(70, 3000, 36, 7), T=9, B=2, p_in=0.5, g_ff=(3.0, 6.0), g_rec=(1.0, 1.0), seed=3)
+    _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    w = wl.small(sizes=(33, 520, 1100, 600, 9), T=37, B=6, p_in=0.1, g_ff=(2.5, 1.5, 1.5), g_rec=(1.0, 1.0, 1.0), seed=5)
+    _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    _check_forward(orc32, w, wl.make(w))
 
 
 def test_forward_c1_bit_exact(orc32):
@@ -400,4 +413,54 @@ def test_layer_by_layer_backward_order(orc32):
     # the wavefront order agrees within tolerance (different summation, not bit-identical)
     s.train_step(bits, targets, strategy=1, chunk_size=9, extra_flags=b.SNN_FLAG_BACKWARD_WAVEFRONT)
     assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
+def test_reforward_as_one_launch_per_segment(orc32):
+    """The recomputation passes walk through a whole segment inside one launch (small networks: the
+    default).  Gradients must be bit-identical to STANDARD, which recomputes nothing, and to the same
+    strategy with one launch per step; sizes that are no multiple of the column tile, segments longer
+    than the 32 steps staged at a time, steps with no events at all and steps with more events than
+    one window of the merged list (1024) holds."""
+    b = sb()
+    cases = [
+        wl.small(sizes=(70, 700, 1300, 7), T=83, B=5, p_in=0.05, g_ff=(2.5, 1.4), g_rec=(1.0, 1.0), seed=51),
+        wl.small(sizes=(40, 4000, 6), T=12, B=2, p_in=0.5, g_ff=(6.0,), g_rec=(3.0,), seed=52),     # > 1024 events per step
+        wl.small(sizes=(64, 96, 5), T=90, B=3, p_in=0.01, g_ff=(1.5,), g_rec=(0.5,), seed=53),      # mostly silent steps
+    ]
+    for w in cases:
+        d = wl.make(w)
+        ref = run_oracle(orc32, w, d)
+        s, bits, targets = make_session(w, d)
+        s.train_step(bits, targets, strategy=0, max_activity=1.0)
+        assert_grads_close(s.gradients(), ref)
+        base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+        for strat, K, R, P in [(1, 40, 0, 0), (1, 7, 0, 0), (2, 11, 0, 0), (3, 4, 16, 0), (3, 3, 9, 0), (4, 5, 0, 3), (5, 2, 8, 0)]:
+            for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_REFORWARD_PER_STEP | b.SNN_FLAG_FORWARD_PER_STEP):
+                for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+                    g.fill_(float("nan"))
+                s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, nb_local=P,
+                             max_activity=1.0, extra_flags=flags)
+                for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+                    assert np.array_equal(x, y), (w.sizes, strat, K, R, P, flags)
+        s.close()
+    # the widest case really has steps beyond one window
+    S = run_oracle(orc32, cases[1], wl.make(cases[1]))["S"]
+    assert S[0][1:].sum(axis=-1).max() > 1024
+
+
+def test_graded_reforward_as_one_launch_per_segment(orc32):
+    b = sb()
+    w = _graded(sizes=(48, 600, 532, 9), T=45, B=4, seed=54)
+    d = wl.make(w)
+    s, bits, targets = make_session(w, d)
+    s.train_step(bits, targets, strategy=0, max_activity=1.0)
+    assert_grads_close(s.gradients(), run_oracle(orc32, w, d))
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 6, 0), (3, 4, 12), (2, 40, 0)]:
+        for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP):
+            s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0,
+                         extra_flags=flags)
+            for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+                assert np.array_equal(x, y), (strat, K, R, flags)
     s.close()
