@@ -128,9 +128,9 @@ snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const s
  * Gradients are bit-identical across strategies for a given order, not between the two orders. */
 #define SNN_FLAG_BACKWARD_LAYER_BY_LAYER 8u
 #define SNN_FLAG_BACKWARD_WAVEFRONT 16u
-/* The recomputation passes run as one launch per segment while the weights fit in L2 (each CTA walks
- * through the segment's steps from the stored events); this flag forces one launch per step, the
- * order used for larger networks.  Results are bit-identical either way. */
+/* While the weights fit in L2 the recomputation passes take two launches per run of steps (the input
+ * currents of all its steps from the stored events at once, then the leak/reset recurrence); this flag
+ * forces one launch per step, the order used for larger networks.  Results are bit-identical either way. */
 #define SNN_FLAG_REFORWARD_PER_STEP 32u
 /* The forward pass of a spiking (LIF) network whose weights fit in L2 runs as one cooperative launch per
  * forward operation of the plan when the device can hold all its thread blocks at once: blocks wait for

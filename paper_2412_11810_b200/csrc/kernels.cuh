@@ -458,16 +458,22 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   }
 }
 
+// 16-byte asynchronous copy, or 16 zero bytes when `real` is false (nothing is read then).
+__device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* gmem_src, bool real) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gmem_src), "r"(real ? 16u : 0u) : "memory");
+}
+
 // ------------------------------------------------------------------------------------------
-// Re-forward of a whole segment of steps in one launch (the recomputation passes of Sec. 3).
+// Re-forward of a run of steps in two launches (the recomputation passes of Sec. 3).
 //
-// Once the forward pass has stored the events of every step, V_t of a neuron depends on nothing
-// but its own V_{t-1} and those lists: no CTA needs another CTA's result.  A CTA therefore keeps
-// the state of its 512 neurons of one sample in registers and walks through all steps of the
-// segment: the lists of consecutive steps are laid end to end in shared memory (each padded to a
-// whole number of copy groups; a padding entry is a zero-filled copy, and adding +0 leaves an
-// fp32 sum unchanged), so the ring of row copies never drains at a step boundary.  Per step the
-// arithmetic is that of fwd_step_kernel, operation for operation.
+// Once the forward pass has stored the events of every step, the input current
+// I_t = S^{l-1}_t W_ff + S^l_{t-1} W_rec of any step can be computed without the steps before it:
+// only the leak/reset recurrence V_t = alpha V_{t-1} + I_t - theta S_{t-1} is sequential, and it is
+// elementwise.  refwd_gather_kernel computes I_t for all steps of the run at once (one CTA per
+// step, sample, layer and column tile: enough warps per SM to keep the L2 gather busy) and leaves
+// it where V_t will go; refwd_scan_kernel then walks through the steps and replaces I_t by V_t.
+// Per neuron the arithmetic is that of fwd_step_kernel, operation for operation.
 struct SegLayer {
   const float* W_ff;          // [N_pre][N]
   const float* W_rec;         // [N][N]
@@ -477,137 +483,85 @@ struct SegLayer {
   const uint32_t* rec_off;    // own offsets, row 0
   const float* ff_vals;       // graded cell: values that go with ff_pool
   const float* rec_vals;      // graded cell: values that go with rec_pool
-  const uint32_t* mask0;      // [B][W] own spike words at the segment's first state (step t0)
   size_t state_off;           // offset of this layer inside a state slot, in floats
   uint32_t ff_cap, rec_cap;
-  int N, W;
+  int N;
 };
 
 struct SegParams {
   SegLayer lay[MAXL];
   float* slots;               // state slot s starts at slots + s * slot_stride
   size_t slot_stride;         // floats
-  int B, t0, t1;              // steps t0+1 .. t1 are computed from the state of step t0
-  int in_slot, buf_slot, buf_len, keep_every, keep_slot;   // as in snn_op
-  float alpha, theta;
+  int B;
+  int t0;                     // the operation computes steps t0+1 .. from the state of step t0
+  int d0, n;                  // this run: steps t0+d0+1 .. t0+d0+n
+  int buf_slot, buf_len;      // step t0+d goes to slot buf_slot + (d-1) % buf_len (as in snn_op)
 };
 
-constexpr int SEG_STEPS = 32;                          // steps whose list bounds are staged at a time
-constexpr int SEG_GROUPS = LIST_CHUNK / GATHER_ROWS;   // copy groups per window of the merged list
-
-__device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* gmem_src, bool real) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-               "l"(gmem_src), "r"(real ? 16u : 0u) : "memory");
-}
+constexpr int RG_ROWS = 4;     // weight rows per copy group
+constexpr int RG_STAGES = 5;   // copy groups in flight per thread (20 rows, 40 KB per CTA: four CTAs per SM)
+constexpr size_t REFWD_DYN_SMEM = (size_t)RG_STAGES * RG_ROWS * FWD_THREADS * sizeof(float4);
 
 template <bool GRADED>
-__global__ void __launch_bounds__(FWD_THREADS) refwd_segment_kernel(const __grid_constant__ SegParams p) {
+__global__ void __launch_bounds__(FWD_THREADS, 4) refwd_gather_kernel(const __grid_constant__ SegParams p) {
   pdl_launch_dependents();
-  const SegLayer& L = p.lay[blockIdx.z];
+  const int l = blockIdx.z / p.n, d = p.d0 + 1 + blockIdx.z % p.n;
+  const SegLayer& L = p.lay[l];
   const int col0 = blockIdx.x * FWD_COLS;
   if (col0 >= L.N) return;
-  const int b = blockIdx.y, B = p.B, tid = threadIdx.x;
-  __shared__ const float* s_row[LIST_CHUNK];   // listed weight rows at this CTA's first column, null = padding
+  const int b = blockIdx.y, B = p.B, tid = threadIdx.x, t = p.t0 + d;
+  __shared__ const float* s_row[LIST_CHUNK];
   __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
-  __shared__ uint32_t s_offF[SEG_STEPS + 1], s_offR[SEG_STEPS + 1];
-  __shared__ int s_gstart[SEG_STEPS + 1];      // first copy group of each step of the window
-  __shared__ int s_plan[2];                    // steps in the window (0: part of one long step), groups
-  __shared__ uint8_t s_glast[SEG_GROUPS];      // group ends a step
-  extern __shared__ float4 s_stage[];          // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
+  extern __shared__ float4 s_stage[];   // [RG_STAGES][RG_ROWS][FWD_THREADS]
   const int col = col0 + tid * 4;
   const bool active = col < L.N;
   const float* const Wff_tile = L.W_ff + col0;
   const float* const Wrec_tile = L.W_rec + col0;
   const uint32_t* const ff_pool = L.ff_pool + (size_t)b * L.ff_cap;
   const uint32_t* const rec_pool = L.rec_pool + (size_t)b * L.rec_cap;
-  float* const state = p.slots + L.state_off + (size_t)b * L.N + col;
 
   pdl_wait();
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  uint32_t sp = 0;   // spikes of the four neurons at the previous step
-  if (active) {
-    v = *reinterpret_cast<const float4*>(state + (size_t)p.in_slot * p.slot_stride);
-    if (!GRADED) sp = (L.mask0[(size_t)b * L.W + (col >> 5)] >> (col & 31)) & 15u;
-  }
+  const uint32_t s_ff = L.ff_off[(size_t)t * B + b], n_ff = L.ff_off[(size_t)(t + 1) * B + b] - s_ff;
+  const uint32_t s_rec = L.rec_off[(size_t)(t - 1) * B + b], total = n_ff + (L.rec_off[(size_t)t * B + b] - s_rec);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  int t = p.t0 + 1;        // first step of the next window
-  int t_cur = t;           // step whose events this thread is adding
-  uint32_t e_skip = 0;     // events of step t that earlier windows already took
-
-  while (t <= p.t1) {
-    const int ns_try = min(SEG_STEPS, p.t1 - t + 1);
-    __syncthreads();
-    if (tid <= ns_try) {
-      s_offF[tid] = L.ff_off[(size_t)(t + tid) * B + b];
-      s_offR[tid] = L.rec_off[(size_t)(t - 1 + tid) * B + b];
-    }
-    __syncthreads();
-    if (tid == 0) {
-      int ns = 0, g_tot = 0;
-      for (int j = 0; j < ns_try; ++j) {
-        uint32_t n_j = (s_offF[j + 1] - s_offF[j]) + (s_offR[j + 1] - s_offR[j]);
-        if (j == 0) n_j -= e_skip;
-        const int g_j = n_j == 0 ? 1 : (int)((n_j + GATHER_ROWS - 1) / GATHER_ROWS);
-        if (g_tot + g_j > SEG_GROUPS) break;
-        s_gstart[j] = g_tot;
-        g_tot += g_j;
-        ns = j + 1;
-      }
-      if (ns == 0) { s_gstart[0] = 0; g_tot = SEG_GROUPS; }   // one step longer than a window: take a part
-      s_gstart[ns == 0 ? 1 : ns] = g_tot;
-      s_plan[0] = ns; s_plan[1] = g_tot;
-    }
-    __syncthreads();
-    const int ns = s_plan[0], g_tot = s_plan[1];
-    {
-      int j = 0;
-      for (int i = tid; i < g_tot * GATHER_ROWS; i += FWD_THREADS) {
-        const int g = i / GATHER_ROWS;
-        while (j + 1 < ns && s_gstart[j + 1] <= g) ++j;
-        const uint32_t e = (uint32_t)(g - s_gstart[j]) * GATHER_ROWS + (i % GATHER_ROWS) + (j == 0 ? e_skip : 0u);
-        const uint32_t n_ff = s_offF[j + 1] - s_offF[j], n_all = n_ff + (s_offR[j + 1] - s_offR[j]);
-        const float* row = nullptr;
-        float val = 0.f;
-        if (e < n_ff) {
-          const uint32_t q = s_offF[j] + e;
-          row = Wff_tile + (size_t)ff_pool[q] * L.N;
-          if (GRADED) val = L.ff_vals[(size_t)b * L.ff_cap + q];
-        } else if (e < n_all) {
-          const uint32_t q = s_offR[j] + (e - n_ff);
-          row = Wrec_tile + (size_t)rec_pool[q] * L.N;
-          if (GRADED) val = L.rec_vals[(size_t)b * L.rec_cap + q];
-        }
-        s_row[i] = row;
-        if (GRADED) s_val[i] = val;
-        if (i % GATHER_ROWS == 0) s_glast[g] = (ns > 0 && g + 1 == s_gstart[j + 1]) ? 1 : 0;
-      }
+  for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
+    const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
+    for (int i = tid; i < n; i += FWD_THREADS) {
+      const uint32_t q = c0 + i;
+      s_row[i] = q < n_ff ? Wff_tile + (size_t)ff_pool[s_ff + q] * L.N
+                          : Wrec_tile + (size_t)rec_pool[s_rec + (q - n_ff)] * L.N;
+      if (GRADED)
+        s_val[i] = q < n_ff ? L.ff_vals[(size_t)b * L.ff_cap + s_ff + q]
+                            : L.rec_vals[(size_t)b * L.rec_cap + s_rec + (q - n_ff)];
     }
     __syncthreads();
     if (active) {
       float4* const ring = s_stage + tid;
+      const int n_groups = (n + RG_ROWS - 1) / RG_ROWS;
       const int lane_col = tid * 4;
       auto issue = [&](int g) {
-        if (g < g_tot) {
-          float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
-          const float* const* rows = s_row + g * GATHER_ROWS;
+        if (g < n_groups) {
+          float4* dst = ring + (size_t)(g % RG_STAGES) * RG_ROWS * FWD_THREADS;
+          const float* const* rows = s_row + g * RG_ROWS;
 #pragma unroll
-          for (int u = 0; u < GATHER_ROWS; ++u) {
-            const float* r = rows[u];
-            cp_async16_or_zero(dst + u * FWD_THREADS, r ? r + lane_col : Wff_tile, r != nullptr);
+          for (int u = 0; u < RG_ROWS; ++u) {   // past the list's end: a zero-filled copy (+0 leaves the sum unchanged)
+            const bool real = g * RG_ROWS + u < n;
+            cp_async16_or_zero(dst + u * FWD_THREADS, real ? rows[u] + lane_col : Wff_tile, real);
           }
         }
         cp_async_commit();
       };
-      for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
-      for (int g = 0; g < g_tot; ++g) {
-        issue(g + GATHER_STAGES - 1);
-        cp_async_wait<GATHER_STAGES - 1>();
-        const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
+      for (int g = 0; g < RG_STAGES - 1; ++g) issue(g);
+      for (int g = 0; g < n_groups; ++g) {
+        issue(g + RG_STAGES - 1);
+        cp_async_wait<RG_STAGES - 1>();
+        const float4* src = ring + (size_t)(g % RG_STAGES) * RG_ROWS * FWD_THREADS;
 #pragma unroll
-        for (int u = 0; u < GATHER_ROWS; ++u) {
+        for (int u = 0; u < RG_ROWS; ++u) {
           const float4 w = src[u * FWD_THREADS];
           if (GRADED) {
-            const float sv = s_val[g * GATHER_ROWS + u];
+            const int i = g * RG_ROWS + u;
+            const float sv = i < n ? s_val[i] : 0.f;
             acc.x = __fmaf_rn(sv, w.x, acc.x); acc.y = __fmaf_rn(sv, w.y, acc.y);
             acc.z = __fmaf_rn(sv, w.z, acc.z); acc.w = __fmaf_rn(sv, w.w, acc.w);
           } else {
@@ -615,31 +569,73 @@ __global__ void __launch_bounds__(FWD_THREADS) refwd_segment_kernel(const __grid
             acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
           }
         }
-        if (s_glast[g]) {   // the step's lists are through: leak, reset, store
-          if (GRADED) {
-            v.x = __fmaf_rn(p.alpha, v.x, acc.x); v.y = __fmaf_rn(p.alpha, v.y, acc.y);
-            v.z = __fmaf_rn(p.alpha, v.z, acc.z); v.w = __fmaf_rn(p.alpha, v.w, acc.w);
-          } else {
-            v.x = __fsub_rn(__fmaf_rn(p.alpha, v.x, acc.x), __fmul_rn(p.theta, (float)(sp & 1u)));
-            v.y = __fsub_rn(__fmaf_rn(p.alpha, v.y, acc.y), __fmul_rn(p.theta, (float)((sp >> 1) & 1u)));
-            v.z = __fsub_rn(__fmaf_rn(p.alpha, v.z, acc.z), __fmul_rn(p.theta, (float)((sp >> 2) & 1u)));
-            v.w = __fsub_rn(__fmaf_rn(p.alpha, v.w, acc.w), __fmul_rn(p.theta, (float)((sp >> 3) & 1u)));
-            sp = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) |
-                 (v.w > p.theta ? 8u : 0u);
-          }
-          const int d = t_cur - p.t0;
-          *reinterpret_cast<float4*>(state + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = v;
-          if (p.keep_every > 0 && d % p.keep_every == 0)
-            *reinterpret_cast<float4*>(state + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = v;
-          acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          ++t_cur;
-        }
       }
       cp_async_wait<0>();
     }
-    if (ns == 0) e_skip += SEG_GROUPS * GATHER_ROWS;
-    else { e_skip = 0; t += ns; }
+    __syncthreads();
   }
+  if (active)
+    *reinterpret_cast<float4*>(p.slots + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride + L.state_off +
+                               (size_t)b * L.N + col) = acc;
+}
+
+// The recurrence over the steps of a run.  A state slot is one flat array (all layers, [B][N_l] each) and
+// the update is elementwise, so a thread owns four adjacent floats of it and needs no layer arithmetic.
+struct ScanParams {
+  float* slots;
+  size_t slot_stride;         // floats
+  size_t n_quads;             // float4 per state
+  const float* v_start;       // state of step t0+d0 (a slot, or `carry` of the previous run)
+  float* carry;               // receives the state of the run's last step
+  int t0, d0, n;
+  int buf_slot, buf_len, keep_every, keep_slot;
+  float alpha, theta;
+};
+
+constexpr int SCAN_BATCH = 8;   // steps whose loads are in flight together
+
+template <bool GRADED>
+__global__ void __launch_bounds__(128) refwd_scan_kernel(const __grid_constant__ ScanParams p) {
+  pdl_launch_dependents();
+  const size_t q = (size_t)blockIdx.x * 128 + threadIdx.x;
+  if (q >= p.n_quads) return;
+  pdl_wait();
+  float4 v = reinterpret_cast<const float4*>(p.v_start)[q];
+  // spikes of the previous step: S_0 = 0, later S_t = [V_t > theta]
+  uint32_t sp = 0;
+  if (!GRADED && p.t0 + p.d0 > 0)
+    sp = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) | (v.w > p.theta ? 8u : 0u);
+  for (int i0 = 0; i0 < p.n; i0 += SCAN_BATCH) {
+    float4 I[SCAN_BATCH];
+    float4* where[SCAN_BATCH];
+#pragma unroll
+    for (int u = 0; u < SCAN_BATCH; ++u) {
+      const int d = p.d0 + i0 + u + 1;
+      where[u] = reinterpret_cast<float4*>(p.slots + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) + q;
+      I[u] = i0 + u < p.n ? *where[u] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < SCAN_BATCH; ++u) {
+      if (i0 + u < p.n) {
+        if (GRADED) {
+          v.x = __fmaf_rn(p.alpha, v.x, I[u].x); v.y = __fmaf_rn(p.alpha, v.y, I[u].y);
+          v.z = __fmaf_rn(p.alpha, v.z, I[u].z); v.w = __fmaf_rn(p.alpha, v.w, I[u].w);
+        } else {
+          v.x = __fsub_rn(__fmaf_rn(p.alpha, v.x, I[u].x), __fmul_rn(p.theta, (float)(sp & 1u)));
+          v.y = __fsub_rn(__fmaf_rn(p.alpha, v.y, I[u].y), __fmul_rn(p.theta, (float)((sp >> 1) & 1u)));
+          v.z = __fsub_rn(__fmaf_rn(p.alpha, v.z, I[u].z), __fmul_rn(p.theta, (float)((sp >> 2) & 1u)));
+          v.w = __fsub_rn(__fmaf_rn(p.alpha, v.w, I[u].w), __fmul_rn(p.theta, (float)((sp >> 3) & 1u)));
+          sp = (v.x > p.theta ? 1u : 0u) | (v.y > p.theta ? 2u : 0u) | (v.z > p.theta ? 4u : 0u) |
+               (v.w > p.theta ? 8u : 0u);
+        }
+        *where[u] = v;
+        const int d = p.d0 + i0 + u + 1;
+        if (p.keep_every > 0 && d % p.keep_every == 0)
+          reinterpret_cast<float4*>(p.slots + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride)[q] = v;
+      }
+    }
+  }
+  reinterpret_cast<float4*>(p.carry)[q] = v;
 }
 
 // ------------------------------------------------------------------------------------------

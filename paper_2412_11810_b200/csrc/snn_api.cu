@@ -50,7 +50,7 @@ constexpr int BWD_RUN = 32;   // steps per run of the layer-by-layer backward pa
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-  size_t status, progress, logits, dlogits, g_out, counts, carry[2], in_stage, tg_stage;
+  size_t status, progress, logits, dlogits, g_out, counts, carry[2], vcarry, in_stage, tg_stage;
   size_t off[MAXL + 1], pool[MAXL + 1], mask[MAXL + 1];
   size_t vals[MAXL + 1], pref[MAXL + 1], act[MAXL + 1], in_words;   // graded cell only
   uint32_t cap[MAXL + 1];
@@ -88,6 +88,7 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.counts = take(4 * (size_t)B * N_L);
   lo.carry[0] = take(lo.state_bytes);
   lo.carry[1] = take(lo.state_bytes);
+  lo.vcarry = take(lo.state_bytes);   // last state of a re-forward run, start of the next
   lo.words[0] = (sz[0] + 31) / 32;
   const bool graded = net->cell == SNN_CELL_GRADED;
   lo.in_stage = take(4 * (size_t)T * B * (graded ? sz[0] : lo.words[0]));
@@ -356,30 +357,49 @@ struct Exec {
     return SNN_OK;
   }
 
-  // REFWD1 / REFWD2 as one launch: the stored events make every (sample, column tile, layer) independent,
-  // so each CTA walks through the segment's steps on its own.  Used while the weights stay in L2; beyond
-  // that the per-step launches keep the samples in step, and the rows they share are read from HBM once.
-  snn_status run_reforward_segment(const snn_op& op) {
-    SegParams p;
-    std::memset(&p, 0, sizeof p);
-    p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
-    p.B = B; p.t0 = op.t0; p.t1 = op.t1;
-    p.in_slot = op.in_slot; p.buf_slot = op.buf_slot; p.buf_len = op.buf_len;
-    p.keep_every = op.keep_every; p.keep_slot = op.keep_slot;
-    p.alpha = net->alpha; p.theta = net->theta;
+  // REFWD1 / REFWD2 without one launch per step: the stored events make the input current of every step
+  // independent of the steps before it, so a run of steps is two launches, all currents at once and then
+  // the leak/reset recurrence (refwd_gather_kernel, refwd_scan_kernel).  A run is as long as the ring of
+  // state slots the operation writes to.  Used while the weights stay in L2; beyond that the per-step
+  // launches keep the samples in step, and the rows they share are read from HBM once.
+  bool reforward_runs_possible(const snn_op& op) const {
+    if (!lo.weights_resident || (a->flags & SNN_FLAG_REFORWARD_PER_STEP)) return false;
+    return (long long)L * std::min(op.buf_len, op.t1 - op.t0) <= 65535;
+  }
+
+  snn_status run_reforward_runs(const snn_op& op) {
+    SegParams g;
+    std::memset(&g, 0, sizeof g);
+    g.slots = at<float>(lo.slots); g.slot_stride = lo.state_bytes / 4;
+    g.B = B; g.t0 = op.t0; g.buf_slot = op.buf_slot; g.buf_len = op.buf_len;
     for (int l = 1; l <= L; ++l) {
-      SegLayer& s = p.lay[l - 1];
+      SegLayer& s = g.lay[l - 1];
       s.W_ff = a->W_ff[l - 1]; s.W_rec = a->W_rec[l - 1];
       s.ff_pool = pool(l - 1); s.ff_off = off(l - 1, 0); s.ff_cap = lo.cap[l - 1];
       s.rec_pool = pool(l); s.rec_off = off(l, 0); s.rec_cap = lo.cap[l];
       if (graded()) { s.ff_vals = vals(l - 1); s.rec_vals = vals(l); }
-      s.mask0 = mask(l, op.t0);
       s.state_off = lo.layer_off[l];
-      s.N = net->sizes[l]; s.W = lo.words[l];
+      s.N = net->sizes[l];
     }
-    void (*k)(SegParams) = graded() ? refwd_segment_kernel<true> : refwd_segment_kernel<false>;
-    CUDA_TRY(launch_pdl(k, fwd_grid(), dim3(FWD_THREADS), FWD_DYN_SMEM, p));
-    ++launches;
+    ScanParams c;
+    std::memset(&c, 0, sizeof c);
+    c.slots = g.slots; c.slot_stride = g.slot_stride; c.n_quads = lo.state_bytes / 16;
+    c.carry = at<float>(lo.vcarry);
+    c.t0 = op.t0; c.buf_slot = op.buf_slot; c.buf_len = op.buf_len;
+    c.keep_every = op.keep_every; c.keep_slot = op.keep_slot;
+    c.alpha = net->alpha; c.theta = net->theta;
+    void (*kg)(SegParams) = graded() ? refwd_gather_kernel<true> : refwd_gather_kernel<false>;
+    void (*kc)(ScanParams) = graded() ? refwd_scan_kernel<true> : refwd_scan_kernel<false>;
+    const int n_all = op.t1 - op.t0;
+    const dim3 fg = fwd_grid();
+    for (int d0 = 0; d0 < n_all; d0 += op.buf_len) {
+      const int n = std::min(op.buf_len, n_all - d0);
+      g.d0 = c.d0 = d0; g.n = c.n = n;
+      c.v_start = d0 == 0 ? at<float>(lo.slots) + (size_t)op.in_slot * g.slot_stride : c.carry;
+      CUDA_TRY(launch_pdl(kg, dim3(fg.x, fg.y, (unsigned)(L * n)), dim3(FWD_THREADS), REFWD_DYN_SMEM, g));
+      CUDA_TRY(launch_pdl(kc, dim3((unsigned)((c.n_quads + 127) / 128)), dim3(128), 0, c));
+      launches += 2;
+    }
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
   }
@@ -448,8 +468,8 @@ struct Exec {
     const int n = op.t1 - op.t0;
     const int span = begin_span(op.kind == SNN_OP_FWD ? SNN_PHASE_FWD
                                 : op.kind == SNN_OP_REFWD1 ? SNN_PHASE_REFWD1 : SNN_PHASE_REFWD2);
-    if (!gen && lo.weights_resident && !(a->flags & SNN_FLAG_REFORWARD_PER_STEP)) {
-      const snn_status st = run_reforward_segment(op);
+    if (!gen && reforward_runs_possible(op)) {
+      const snn_status st = run_reforward_runs(op);
       end_span(span);
       return st;
     }
@@ -758,8 +778,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(refwd_segment_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(refwd_segment_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFWD_DYN_SMEM));
+      CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFWD_DYN_SMEM));
       CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8)));
       CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(16)));
