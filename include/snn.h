@@ -138,6 +138,10 @@ snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const s
  * step.  Results are bit-identical either way.  A wait that does not end within a few seconds makes the
  * step return SNN_ERR_DEVICE_TIMEOUT. */
 #define SNN_FLAG_FORWARD_PER_STEP 64u
+/* Small spiking networks (batch up to 64; the columns of W_ff and W_rec that 16 neurons need within
+ * 200 KB; at most one thread block of 16 neurons per SM over all layers) keep their weights in shared
+ * memory during a forward launch.  This flag makes them stream the weights from L2 like larger ones. */
+#define SNN_FLAG_FORWARD_STREAM_WEIGHTS 128u
 
 typedef struct {
   int32_t T, B;

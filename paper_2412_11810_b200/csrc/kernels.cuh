@@ -844,6 +844,321 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
 }
 
 // ------------------------------------------------------------------------------------------
+// Forward pass with the weights resident in shared memory (LIF cell, networks of a few thousand
+// neurons: all weight matrices together must fit the shared memory of the whole device).
+//
+// A CTA owns RS_COLS columns of one layer and keeps those columns of W_ff and W_rec (every row) in
+// shared memory for all steps of the launch, so an event costs a shared-memory read instead of an
+// L2 gather.  Per step a half-warp turns the spike words of one sample into the list of weight rows
+// in canonical order (feed-forward events, then recurrent ones, ascending); then the first four
+// warps add the rows, one thread per sample and four columns, apply leak, reset and threshold, and
+// publish 16 spike bits per sample.  The event pools of a sample are appended to by one CTA of the
+// layer (sample index modulo the number of CTAs).  Every CTA of a layer needs the words of all
+// columns, so the layers synchronise through one counter each (finished (CTA, step) pairs), with
+// the publish / poll protocol of fwd_segment_kernel.  Cooperative launch; bounded waits.
+constexpr int RS_COLS = 16;        // columns of a layer per CTA
+constexpr int RS_THREADS = 512;    // 32 samples x RS_COLS columns
+constexpr int RS_LIST = 256;       // list entries per sample staged at a time
+constexpr int RS_MAX_GROUPS = 2;   // groups of 32 samples a thread can own: B <= 64
+
+struct ResLayer {
+  const float* W_ff;          // [N_pre][N]
+  const float* W_rec;         // [N][N]
+  const uint32_t* ff_words;   // spike words of the layer below; row of step t at (t - ff_row0) * B * W_pre
+  uint32_t* words;            // own spike words [T+1][B][W]
+  uint32_t* ff_pool;          // event pool of the layer below [B][ff_cap] (written here if write_ff_list)
+  uint32_t* ff_off;           // its offsets, row 0
+  uint32_t* rec_pool;         // own event pool [B][rec_cap]
+  uint32_t* rec_off;          // own offsets, row 0
+  uint32_t* counts;           // [B][N] spike counts (last layer) or null
+  float* V_dbg;               // [T+1][B][N] copy of every state, or null
+  size_t state_off;           // offset of this layer inside a state slot, in floats
+  uint32_t ff_cap, rec_cap;
+  int N_pre, N, W_pre, W;
+  int ff_row0;                // 1 for the input (its rows start at step 1), 0 for hidden layers
+  int write_ff_list;          // the layer below is the input: this layer stores its lists
+  int tiles;                  // CTAs of this layer
+  int cta0;                   // blockIdx.x of its first CTA
+};
+
+struct ResParams {
+  ResLayer lay[MAXL];
+  float* slots;
+  size_t slot_stride;         // floats
+  uint32_t* status;
+  uint32_t* progress;         // [L] finished (CTA, step) pairs per layer, zero at launch
+  int L, B, t0, t1;
+  int in_slot, buf_slot, buf_len, keep_every, keep_slot;
+  float alpha, theta;
+};
+
+__host__ __device__ inline size_t resident_words_bytes(int W_pre, int W, int B) {
+  return ((size_t)B * (W_pre + W) * 4 + 15) / 16 * 16;
+}
+__host__ __device__ inline size_t resident_smem_bytes(int N_pre, int N, int W_pre, int W, int B) {
+  return (size_t)(N_pre + N) * RS_COLS * 4 + resident_words_bytes(W_pre, W, B) + (size_t)32 * RS_LIST * 2;
+}
+
+__global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __grid_constant__ ResParams p) {
+  int l = 0;
+  while (l + 1 < p.L && (int)blockIdx.x >= p.lay[l + 1].cta0) ++l;
+  const ResLayer& L = p.lay[l];
+  const int tile = (int)blockIdx.x - L.cta0, col0 = tile * RS_COLS;
+  const int tid = threadIdx.x, B = p.B;
+  const int Wtot = L.W_pre + L.W, rows = L.N_pre + L.N;
+  const int groups = (B + 31) / 32;
+  extern __shared__ float4 s_dyn[];
+  float* const Ws = reinterpret_cast<float*>(s_dyn);                                     // [rows][RS_COLS]
+  uint32_t* const s_words = reinterpret_cast<uint32_t*>(Ws + (size_t)rows * RS_COLS);   // [B][Wtot]
+  uint16_t* const s_list = reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(s_words) +
+                                                       resident_words_bytes(L.W_pre, L.W, B));   // [32][RS_LIST]
+  __shared__ int s_ok;
+  __shared__ int s_n[32];   // list entries of each of the 32 samples in this chunk
+  __shared__ uint32_t s_ends[32][3];   // per sample: end of its recurrent and feed-forward pool lists, feed-forward events now
+
+  // Two roles.  Compaction: half-warp `bl` (16 lanes, lane index c) turns the words of sample 32 gi + bl into
+  // its list.  Accumulation: the first 128 threads; thread (sb, quad) owns columns 4 quad .. 4 quad + 3 of
+  // sample 32 gi + sb.
+  const int c = tid & (RS_COLS - 1), bl = tid >> 4;
+  const bool adder = tid < 128;
+  const int sb = tid >> 2, quad = tid & 3;
+  const int acol = col0 + quad * 4;            // first of this thread's four columns (accumulation role)
+  const bool acol_ok = adder && acol < L.N;    // N is a multiple of 4: all four or none
+
+  // ---- this CTA's columns of both matrices, every row, once per launch
+  for (int q = tid; q < rows * (RS_COLS / 4); q += RS_THREADS) {
+    const int r = q / (RS_COLS / 4), part = q % (RS_COLS / 4);
+    const int cc = col0 + part * 4;
+    const float* src = r < L.N_pre ? L.W_ff + (size_t)r * L.N + cc : L.W_rec + (size_t)(r - L.N_pre) * L.N + cc;
+    cp_async16_or_zero(Ws + (size_t)r * RS_COLS + part * 4, cc < L.N ? src : L.W_ff, cc < L.N);
+  }
+  cp_async_commit();
+
+  float4 v[RS_MAX_GROUPS];
+  uint32_t rec_end[RS_MAX_GROUPS], ff_end[RS_MAX_GROUPS];
+  bool owner[RS_MAX_GROUPS];   // this CTA appends the lists of the half-warp's sample to the event pools
+#pragma unroll
+  for (int gi = 0; gi < RS_MAX_GROUPS; ++gi) {
+    v[gi] = make_float4(0.f, 0.f, 0.f, 0.f); rec_end[gi] = 0; ff_end[gi] = 0; owner[gi] = false;
+    if (gi < groups) {
+      const int ba = gi * 32 + sb, bc = gi * 32 + bl;
+      if (acol_ok && ba < B)
+        v[gi] = *reinterpret_cast<const float4*>(p.slots + (size_t)p.in_slot * p.slot_stride + L.state_off +
+                                                 (size_t)ba * L.N + acol);
+      owner[gi] = bc < B && bc % L.tiles == tile;
+      if (owner[gi]) {
+        rec_end[gi] = L.rec_off[(size_t)p.t0 * B + bc];
+        if (L.write_ff_list) ff_end[gi] = L.ff_off[(size_t)(p.t0 + 1) * B + bc];
+      }
+    }
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+
+  uint32_t* const my_progress = p.progress + l;
+  const int wpl = (Wtot + RS_COLS - 1) / RS_COLS;   // words per lane of a half-warp
+  uint16_t* const lst = s_list + (size_t)bl * RS_LIST;
+
+  for (int t = p.t0 + 1; t <= p.t1; ++t) {
+    const uint32_t d = (uint32_t)(t - p.t0);
+    if (tid == 0) {
+      bool ok = wait_progress(my_progress, (uint32_t)L.tiles * (d - 1));
+      if (ok && l > 0) ok = wait_progress(p.progress + (l - 1), (uint32_t)p.lay[l - 1].tiles * d);
+      if (!ok) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+      s_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_ok) return;
+
+#pragma unroll
+    for (int gi = 0; gi < RS_MAX_GROUPS; ++gi) {
+      if (gi >= groups) break;                       // uniform
+      // ---- compaction role
+      const int b = gi * 32 + bl;
+      const bool b_ok = b < B;
+      uint32_t* const wrow = s_words + (size_t)(b_ok ? b : B - 1) * Wtot;
+      if (b_ok) {   // the sample's spike words, past L1 (other CTAs wrote them during this launch)
+        const uint32_t* ffw = L.ff_words + ((size_t)(t - L.ff_row0) * B + b) * L.W_pre;
+        const uint32_t* recw = L.words + ((size_t)(t - 1) * B + b) * L.W;
+        for (int w0 = c; w0 < Wtot; w0 += 4 * RS_COLS) {   // four loads in flight per lane
+          uint32_t r[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int w = w0 + j * RS_COLS;
+            r[j] = w < Wtot ? __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre)) : 0u;
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (w0 + j * RS_COLS < Wtot) wrow[w0 + j * RS_COLS] = r[j];
+        }
+      }
+      __syncwarp();
+      // events before this lane's words, in the sample's canonical order
+      const int w_lo = c * wpl, w_hi = min(Wtot, w_lo + wpl);
+      uint32_t cnt = 0, cnt_ff = 0;
+      for (int w = w_lo; w < w_hi; ++w) {
+        const uint32_t k = b_ok ? __popc(wrow[w]) : 0u;
+        cnt += k;
+        if (w < L.W_pre) cnt_ff += k;
+      }
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int s = 1; s < RS_COLS; s <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, s, RS_COLS);
+        if (c >= s) incl += y;
+      }
+      const uint32_t n_tot = __shfl_sync(0xffffffffu, incl, RS_COLS - 1, RS_COLS);
+      uint32_t n_ff = cnt_ff;
+#pragma unroll
+      for (int s = RS_COLS / 2; s >= 1; s >>= 1) n_ff += __shfl_xor_sync(0xffffffffu, n_ff, s, RS_COLS);
+      const uint32_t first = incl - cnt;
+      const bool pools = owner[gi];
+      const uint32_t room_rec = L.rec_cap - rec_end[gi], room_ff = L.write_ff_list ? L.ff_cap - ff_end[gi] : 0u;
+
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (uint32_t c0 = 0;; c0 += RS_LIST) {
+        // this lane's events that fall into [c0, c0 + RS_LIST): row of Ws into the list, index into the pools
+        uint32_t pos = first;
+        for (int w = w_lo; w < w_hi && pos < c0 + RS_LIST; ++w) {
+          uint32_t bits = b_ok ? wrow[w] : 0u;
+          const bool ff = w < L.W_pre;
+          const uint32_t idx0 = (uint32_t)(ff ? w : w - L.W_pre) * 32u;
+          if (pos + __popc(bits) <= c0) { pos += __popc(bits); continue; }
+          while (bits) {
+            const uint32_t idx = idx0 + (uint32_t)(__ffs(bits) - 1);
+            bits &= bits - 1;
+            if (pos >= c0 && pos < c0 + RS_LIST) {
+              lst[pos - c0] = (uint16_t)(ff ? idx : idx + (uint32_t)L.N_pre);
+            }
+            ++pos;
+          }
+        }
+        if (c == 0) {
+          s_n[bl] = (int)(n_tot > c0 ? (n_tot - c0 < (uint32_t)RS_LIST ? n_tot - c0 : (uint32_t)RS_LIST) : 0u);
+          if (pools) { s_ends[bl][0] = rec_end[gi]; s_ends[bl][1] = ff_end[gi]; s_ends[bl][2] = n_ff; }
+        }
+        const int more = __syncthreads_or(n_tot > c0 + RS_LIST);   // the lists of all 32 samples are in place
+        // ---- accumulation role: in list order, one accumulator per (sample, column)
+        if (adder) {
+          const int n = s_n[sb];
+          const uint16_t* const al = s_list + (size_t)sb * RS_LIST;
+          const float4* const Wq = reinterpret_cast<const float4*>(Ws) + quad;
+          auto add4 = [&](const float4 r) {
+            acc.x = __fadd_rn(acc.x, r.x); acc.y = __fadd_rn(acc.y, r.y);
+            acc.z = __fadd_rn(acc.z, r.z); acc.w = __fadd_rn(acc.w, r.w);
+          };
+          // eight rows at a time, the next eight already on their way while these are added
+          auto load8 = [&](int e, float4 (&w)[8]) {
+            const uint4 pk = *reinterpret_cast<const uint4*>(al + e);
+            w[0] = Wq[(pk.x & 0xffffu) * (RS_COLS / 4)]; w[1] = Wq[(pk.x >> 16) * (RS_COLS / 4)];
+            w[2] = Wq[(pk.y & 0xffffu) * (RS_COLS / 4)]; w[3] = Wq[(pk.y >> 16) * (RS_COLS / 4)];
+            w[4] = Wq[(pk.z & 0xffffu) * (RS_COLS / 4)]; w[5] = Wq[(pk.z >> 16) * (RS_COLS / 4)];
+            w[6] = Wq[(pk.w & 0xffffu) * (RS_COLS / 4)]; w[7] = Wq[(pk.w >> 16) * (RS_COLS / 4)];
+          };
+          auto add8 = [&](const float4 (&w)[8]) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) add4(w[j]);
+          };
+          const int n8 = n & ~7;
+          float4 wa[8], wb[8];
+          int e = 0;
+          if (n8 > 0) load8(0, wa);
+          while (e < n8) {
+            if (e + 8 < n8) load8(e + 8, wb);
+            add8(wa);
+            e += 8;
+            if (e >= n8) break;
+            if (e + 8 < n8) load8(e + 8, wa);
+            add8(wb);
+            e += 8;
+          }
+          for (; e < n; ++e) {
+            add4(Wq[(uint32_t)al[e] * (RS_COLS / 4)]);
+          }
+        } else {
+          // ---- meanwhile the other warps append the lists of the samples this CTA owns to the event pools
+          const int h = (tid - 128) >> 4, n_helpers = (RS_THREADS - 128) >> 4;
+          int bb = tile;
+          while (bb < 32 * gi) bb += L.tiles;
+          for (int k = 0; bb < B && bb < 32 * gi + 32; bb += L.tiles, ++k) {
+            if (k % n_helpers != h) continue;
+            const int sl = bb & 31;
+            const uint16_t* const pl = s_list + (size_t)sl * RS_LIST;
+            const uint32_t r_end = s_ends[sl][0], f_end = s_ends[sl][1], nf = s_ends[sl][2];
+            const uint32_t rm_rec = L.rec_cap - r_end, rm_ff = L.write_ff_list ? L.ff_cap - f_end : 0u;
+            const int n = s_n[sl];
+            for (int e = c; e < n; e += RS_COLS) {
+              const uint32_t r = pl[e], pos = c0 + (uint32_t)e;
+              if (pos < nf) { if (pos < rm_ff) L.ff_pool[(size_t)bb * L.ff_cap + f_end + pos] = r; }
+              else if (pos - nf < rm_rec) L.rec_pool[(size_t)bb * L.rec_cap + r_end + (pos - nf)] = r - (uint32_t)L.N_pre;
+            }
+          }
+        }
+        if (!more) break;
+        __syncthreads();   // before the lists are refilled
+      }
+
+      // ---- leak, reset by subtraction of the previous step's own spike, threshold (accumulation role)
+      const int ba = gi * 32 + sb;
+      uint32_t nib = 0;
+      if (acol_ok && ba < B) {
+        const uint32_t pw = s_words[(size_t)ba * Wtot + L.W_pre + (acol >> 5)] >> (acol & 31);
+        float4 vn;
+        vn.x = __fsub_rn(__fmaf_rn(p.alpha, v[gi].x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
+        vn.y = __fsub_rn(__fmaf_rn(p.alpha, v[gi].y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
+        vn.z = __fsub_rn(__fmaf_rn(p.alpha, v[gi].z, acc.z), __fmul_rn(p.theta, (float)((pw >> 2) & 1u)));
+        vn.w = __fsub_rn(__fmaf_rn(p.alpha, v[gi].w, acc.w), __fmul_rn(p.theta, (float)((pw >> 3) & 1u)));
+        v[gi] = vn;
+        float* const st = p.slots + L.state_off + (size_t)ba * L.N + acol;
+        *reinterpret_cast<float4*>(st + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = vn;
+        if (p.keep_every > 0 && d % p.keep_every == 0)
+          *reinterpret_cast<float4*>(st + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = vn;
+        if (L.V_dbg) *reinterpret_cast<float4*>(L.V_dbg + ((size_t)t * B + ba) * L.N + acol) = vn;
+        nib = (vn.x > p.theta ? 1u : 0u) | (vn.y > p.theta ? 2u : 0u) | (vn.z > p.theta ? 4u : 0u) |
+              (vn.w > p.theta ? 8u : 0u);
+        if (L.counts && nib) {
+          uint4* cp = reinterpret_cast<uint4*>(L.counts + (size_t)ba * L.N + acol);
+          uint4 cv = *cp;
+          cv.x += nib & 1u; cv.y += (nib >> 1) & 1u; cv.z += (nib >> 2) & 1u; cv.w += (nib >> 3) & 1u;
+          *cp = cv;
+        }
+      }
+      if (adder) {   // whole warps: four neighbouring lanes hold the 16 spike bits of one sample
+        uint32_t half = nib << (4 * quad);
+        half |= __shfl_xor_sync(0xffffffffu, half, 1);
+        half |= __shfl_xor_sync(0xffffffffu, half, 2);
+        if (quad == 0 && ba < B) {
+          uint16_t* const hrow = reinterpret_cast<uint16_t*>(L.words + ((size_t)t * B + ba) * L.W);
+          hrow[tile] = (uint16_t)half;
+          if (tile == L.tiles - 1 && (L.tiles & 1)) hrow[tile + 1] = 0;   // the unused half of the last word
+        }
+      }
+      // ---- compaction role again: where this sample's lists now end
+      if (pools && c == 0) {
+        const uint32_t n_rec = n_tot - n_ff;
+        rec_end[gi] += n_rec < room_rec ? n_rec : room_rec;
+        L.rec_off[(size_t)t * B + b] = rec_end[gi];
+        bool over = n_rec > room_rec;
+        if (L.write_ff_list) {
+          ff_end[gi] += n_ff < room_ff ? n_ff : room_ff;
+          L.ff_off[(size_t)(t + 1) * B + b] = ff_end[gi];
+          over = over || n_ff > room_ff;
+        }
+        if (over) atomicOr(p.status, STATUS_EVENT_OVERFLOW);
+      }
+      rec_end[gi] = __shfl_sync(0xffffffffu, rec_end[gi], 0, RS_COLS);   // the other lanes keep the same running ends
+      ff_end[gi] = __shfl_sync(0xffffffffu, ff_end[gi], 0, RS_COLS);
+      if (gi + 1 < groups) __syncthreads();   // s_list and s_n are reused by the next group of samples
+    }
+    __syncthreads();
+    if (tid == 0) {   // publish: this CTA's spike bits of step t are complete
+      __threadfence();
+      atomicAdd(my_progress, 1u);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Backward step: delta^l_t = g_S sigma'(V^l_t - theta) + alpha delta^l_{t+1}, with
 // g_S = g_out + W_ff^{l+1} delta^{l+1}_t + W_rec^l delta^l_{t+1} - theta delta^l_{t+1}.
 //

@@ -28,6 +28,8 @@ struct snn_net {
   std::vector<cudaEvent_t> copy_events;    // one per checkpoint copy in flight, grown on demand
   std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
   snn_phase_times phases{};
+  int coop_sms = -1;                       // SMs usable by a cooperative launch (-1: not asked yet)
+  size_t resident_smem_set = 0;            // dynamic shared memory fwd_resident_kernel is opted in for
   int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
 };
 
@@ -426,6 +428,81 @@ struct Exec {
     return (long long)g.x * g.y * g.z <= net->fwd_segment_capacity;
   }
 
+  // FWD with the weights held in shared memory for the whole launch (fwd_resident_kernel): small LIF networks.
+  size_t resident_smem_max() const {
+    size_t m = 0;
+    for (int l = 1; l <= L; ++l)
+      m = std::max(m, resident_smem_bytes(net->sizes[l - 1], net->sizes[l], lo.words[l - 1], lo.words[l], B));
+    return m;
+  }
+  bool forward_resident_possible() {
+    if (graded() || (a->flags & (SNN_FLAG_FORWARD_PER_STEP | SNN_FLAG_FORWARD_STREAM_WEIGHTS))) return false;
+    if (B > 32 * RS_MAX_GROUPS) return false;
+    long long ctas = 0;
+    for (int l = 1; l <= L; ++l) {
+      if (net->sizes[l - 1] + net->sizes[l] > 65535) return false;
+      ctas += (net->sizes[l] + RS_COLS - 1) / RS_COLS;
+    }
+    const size_t smem = resident_smem_max();
+    if (smem > (size_t)200 << 10) return false;
+    if (net->coop_sms < 0) {
+      int dev = 0, sms = 0, coop = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
+        cudaGetLastError();
+        net->coop_sms = 0;
+      } else {
+        net->coop_sms = coop ? sms : 0;
+      }
+    }
+    return ctas <= net->coop_sms;   // one CTA per SM (more than half of its shared memory each)
+  }
+
+  snn_status run_forward_resident(const snn_op& op) {
+    ResParams p;
+    std::memset(&p, 0, sizeof p);
+    p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
+    p.status = at<uint32_t>(lo.status); p.progress = at<uint32_t>(lo.progress);
+    p.L = L; p.B = B; p.t0 = op.t0; p.t1 = op.t1;
+    p.in_slot = op.in_slot; p.buf_slot = op.buf_slot; p.buf_len = op.buf_len;
+    p.keep_every = op.keep_every; p.keep_slot = op.keep_slot;
+    p.alpha = net->alpha; p.theta = net->theta;
+    int ctas = 0;
+    for (int l = 1; l <= L; ++l) {
+      ResLayer& s = p.lay[l - 1];
+      s.W_ff = a->W_ff[l - 1]; s.W_rec = a->W_rec[l - 1];
+      s.ff_words = l == 1 ? in_mask(1) : mask(l - 1, 0);
+      s.ff_row0 = l == 1 ? 1 : 0;
+      s.words = mask(l, 0);
+      s.ff_pool = pool(l - 1); s.ff_off = off(l - 1, 0); s.ff_cap = lo.cap[l - 1];
+      s.rec_pool = pool(l); s.rec_off = off(l, 0); s.rec_cap = lo.cap[l];
+      s.counts = l == L ? at<uint32_t>(lo.counts) : nullptr;
+      s.V_dbg = (a->debug_V && a->debug_V[l - 1]) ? a->debug_V[l - 1] : nullptr;
+      s.state_off = lo.layer_off[l];
+      s.N_pre = net->sizes[l - 1]; s.N = net->sizes[l]; s.W_pre = lo.words[l - 1]; s.W = lo.words[l];
+      s.write_ff_list = l == 1;
+      s.tiles = (net->sizes[l] + RS_COLS - 1) / RS_COLS;
+      s.cta0 = ctas;
+      ctas += s.tiles;
+    }
+    const size_t smem = resident_smem_max();
+    if (smem > net->resident_smem_set) {
+      CUDA_TRY(cudaFuncSetAttribute(fwd_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      net->resident_smem_set = smem;
+    }
+    CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L, main));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(RS_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cudaLaunchAttribute at1[1];
+    at1[0].id = cudaLaunchAttributeCooperative;
+    at1[0].val.cooperative = 1;
+    cfg.attrs = at1; cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, fwd_resident_kernel, p));
+    ++launches;
+    return SNN_OK;
+  }
+
   snn_status run_forward_segment(const snn_op& op) {
     FwdSegParams p;
     std::memset(&p, 0, sizeof p);
@@ -470,6 +547,11 @@ struct Exec {
                                 : op.kind == SNN_OP_REFWD1 ? SNN_PHASE_REFWD1 : SNN_PHASE_REFWD2);
     if (!gen && reforward_runs_possible(op)) {
       const snn_status st = run_reforward_runs(op);
+      end_span(span);
+      return st;
+    }
+    if (gen && forward_resident_possible()) {
+      const snn_status st = run_forward_resident(op);
       end_span(span);
       return st;
     }

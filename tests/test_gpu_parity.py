@@ -99,14 +99,22 @@ def test_forward_ragged_sizes_bit_exact(orc32):
 def test_forward_one_launch_per_step_bit_exact(orc32):
     """Small spiking networks run the forward pass as one cooperative launch per forward operation; the
     launch-per-step kernel (the one large networks use) must give the same bits."""
-    f = sb().SNN_FLAG_FORWARD_PER_STEP
+    f, g = sb().SNN_FLAG_FORWARD_PER_STEP, sb().SNN_FLAG_FORWARD_STREAM_WEIGHTS
     w = wl.small()
     _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    _check_forward(orc32, w, wl.make(w), extra_flags=g)
     w = wl.small(sizes=(70, 3000, 36, 7), T=9, B=2, p_in=0.5, g_ff=(3.0, 6.0), g_rec=(1.0, 1.0), seed=3)
     _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    # three layers, ragged tiles, 140 thread blocks of 16 neurons: weights in shared memory by default
     w = wl.small(sizes=(33, 520, 1100, 600, 9), T=37, B=6, p_in=0.1, g_ff=(2.5, 1.5, 1.5), g_rec=(1.0, 1.0, 1.0), seed=5)
     _check_forward(orc32, w, wl.make(w), extra_flags=f)
+    _check_forward(orc32, w, wl.make(w), extra_flags=g)
     _check_forward(orc32, w, wl.make(w))
+    # more than 32 samples (two samples groups per thread), more than 256 events per sample and step
+    w = wl.small(sizes=(100, 1000, 8), T=7, B=45, p_in=0.5, g_ff=(4.0,), g_rec=(2.0,), seed=6)
+    ref = _check_forward(orc32, w, wl.make(w))
+    assert ref["S"][0][1:].sum(axis=-1).max() > 256
+    _check_forward(orc32, w, wl.make(w), extra_flags=g)
 
 
 def test_forward_c1_bit_exact(orc32):
@@ -436,7 +444,8 @@ def test_reforward_as_one_launch_per_segment(orc32):
         assert_grads_close(s.gradients(), ref)
         base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
         for strat, K, R, P in [(1, 40, 0, 0), (1, 7, 0, 0), (2, 11, 0, 0), (3, 4, 16, 0), (3, 3, 9, 0), (4, 5, 0, 3), (5, 2, 8, 0)]:
-            for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_REFORWARD_PER_STEP | b.SNN_FLAG_FORWARD_PER_STEP):
+            for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_REFORWARD_PER_STEP | b.SNN_FLAG_FORWARD_PER_STEP,
+                          b.SNN_FLAG_FORWARD_STREAM_WEIGHTS):
                 for g in s.dW_ff + s.dW_rec + [s.dW_out]:
                     g.fill_(float("nan"))
                 s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, nb_local=P,
