@@ -1226,15 +1226,30 @@ __device__ __forceinline__ void warp_transpose_reduce(float (&v)[NV], int lane) 
 
 constexpr int BWD_STAGES = 4;   // chunks of the W and delta tiles in flight per CTA
 
-__device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer& L, int i, int b, float sum) {
+// What the epilogue of one output element needs from global memory; fetched before the contraction starts
+// so that the loads are long done when the sums arrive.
+struct BwdPre { float dn, go, gf, v; };
+
+__device__ __forceinline__ BwdPre bwd_prefetch(const BwdParams& p, const BwdLayer& L, int i, int b) {
+  BwdPre r{0.f, 0.f, 0.f, 0.f};
+  if (i >= L.N || b >= p.B) return r;
+  const size_t k = (size_t)b * L.N + i;
+  r.dn = L.d_next[k];
+  r.go = L.g_out ? L.g_out[k] : 0.f;
+  r.gf = L.g_ff ? L.g_ff[k] : 0.f;
+  r.v = L.V_delta[k];
+  return r;
+}
+
+__device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer& L, int i, int b, float sum,
+                                             const BwdPre& pre) {
   if (i >= L.N || b >= p.B) return;
   const size_t k = (size_t)b * L.N + i;
-  const float dn = L.d_next[k];
-  float g = sum + (L.g_out ? L.g_out[k] : 0.f);
-  if (L.g_ff) g += L.g_ff[k];
-  if (p.cell == 0) g = fmaf(-p.theta, dn, g);
-  const float sp = surrogate_grad(L.V_delta[k], p.theta, p.beta, p.surrogate, p.cell);
-  const float dl = fmaf(g, sp, p.alpha * dn);
+  float g = sum + pre.go;
+  if (L.g_ff) g += pre.gf;
+  if (p.cell == 0) g = fmaf(-p.theta, pre.dn, g);
+  const float sp = surrogate_grad(pre.v, p.theta, p.beta, p.surrogate, p.cell);
+  const float dl = fmaf(g, sp, p.alpha * pre.dn);
   L.V_delta[k] = dl;
   if (L.carry_out) L.carry_out[k] = dl;
 }
@@ -1244,10 +1259,11 @@ __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer&
 // accumulation, which keeps the result at fp32 accuracy (the dropped lo*lo term is ~2^-22 relative).
 constexpr int BWD_LD = 132;   // padded row length (floats) of the staged tiles: fragment loads hit 32 banks
 
+// fp32 -> tf32 (10 mantissa bits), round to nearest with ties away from zero: half an ulp added to the
+// magnitude, then the 13 low bits cleared.  Two integer operations at full rate instead of a conversion
+// instruction, which runs at an eighth of it and would cost as much as the tensor-core work it feeds.
 __device__ __forceinline__ uint32_t to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
+  return (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
 }
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
   hi = to_tf32(x);
@@ -1271,6 +1287,9 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
 template <int NTN, int NWARP>
 __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
   constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * BWD_LD, TILE = BWD_TM * BP;
+  constexpr int TS = BP + 8, TILEP = BWD_TM * TS;   // padded rows of the warps' partial tiles: 64-bit stores without bank conflicts
+  constexpr int EPI = TILE / NT;                    // output elements a thread finishes at most (cluster of one)
+  static_assert(TILE % NT == 0 && NWARP * TILEP <= BWD_STAGES * STAGE_F, "partial tiles fit the stages");
   pdl_launch_dependents();
   cg::cluster_group cluster = cg::this_cluster();
   const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
@@ -1296,6 +1315,12 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
   static_assert(ROWS * 32 % NT == 0, "the staged tile divides evenly among the threads");
   pdl_wait();
   for (int bp0 = 0; bp0 < p.B; bp0 += BP) {
+    BwdPre pre[EPI];
+#pragma unroll
+    for (int j = 0; j < EPI; ++j) {
+      const int q = tid + j * NT, e = CS == 1 ? q : rank + CS * q;
+      pre[j] = (e < TILE) ? bwd_prefetch(p, L, tile_row0 + e / BP, bp0 + e % BP) : BwdPre{0.f, 0.f, 0.f, 0.f};
+    }
     const float* src_rec[ITER];
     const float* src_ff[ITER];
     int dst_off[ITER], kcol[ITER];
@@ -1314,7 +1339,8 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
         src_ff[j] = L.d_above ? L.d_above + b * L.N_post + 4 * c4 : nullptr;
       }
     }
-    auto issue = [&](int it) {
+    // positions [j0, j1) of chunk `it`; the caller commits the group once all ITER positions are issued
+    auto issue_part = [&](int it, int j0, int j1) {
       if (it < it_all) {
         const bool ff = it < it_ff;
         const int k0 = ff ? lo_ff + it * 128 : lo_rec + (it - it_ff) * 128;
@@ -1322,10 +1348,14 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
         float* st = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
 #pragma unroll
         for (int j = 0; j < ITER; ++j) {
+          if (j < j0 || j >= j1) continue;
           if (k0 + kcol[j] < hi) cp_async16(st + dst_off[j], (ff ? src_ff[j] : src_rec[j]) + k0);
           else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);   // past the slice
         }
       }
+    };
+    auto issue = [&](int it) {
+      issue_part(it, 0, ITER);
       cp_async_commit();
     };
     float acc[2][NTN][4];
@@ -1339,7 +1369,11 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
     for (int it = 0; it < it_all; ++it) {
       cp_async_wait<BWD_STAGES - 2>();   // this thread's copies of chunk `it` have landed
       __syncthreads();                   // ... everybody's have, and chunk it-1 has been consumed
-      issue(it + BWD_STAGES - 1);        // refills the stage chunk it-1 used
+      // The copies that refill the stage chunk it-1 used are issued between the tensor-core passes of this
+      // warp's first k-step: copy instructions and mma instructions queue on different pipes, and in program
+      // order one after the other they would take turns instead of overlapping.
+      const int it_refill = it + BWD_STAGES - 1;
+      bool refill = true;
       const float* Ws = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
       const float* Ds = Ws + BWD_TM * BWD_LD;
 #pragma unroll 1
@@ -1365,53 +1399,72 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
           for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
+        if (refill) issue_part(it_refill, 0, ITER / 3);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
           for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
+        if (refill) issue_part(it_refill, ITER / 3, 2 * ITER / 3);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
           for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
+        if (refill) {
+          issue_part(it_refill, 2 * ITER / 3, ITER);
+          cp_async_commit();
+          refill = false;
+        }
       }
     }
     cp_async_wait<0>();
-    __syncthreads();   // the stages are free: they now hold the warps' partial tiles [NWARP][32][BP]
+    __syncthreads();   // the stages are free: they now hold the warps' partial tiles [NWARP][32][TS]
     {
-      float* mine = s_tiles + (size_t)warp * TILE;
+      float* mine = s_tiles + (size_t)warp * TILEP;
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NTN; ++nt) {
           const int r = mt * 16 + g, c = nt * 8 + 2 * t;
-          mine[r * BP + c] = acc[mt][nt][0];       mine[r * BP + c + 1] = acc[mt][nt][1];
-          mine[(r + 8) * BP + c] = acc[mt][nt][2]; mine[(r + 8) * BP + c + 1] = acc[mt][nt][3];
+          *reinterpret_cast<float2*>(mine + r * TS + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+          *reinterpret_cast<float2*>(mine + (r + 8) * TS + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
         }
     }
     __syncthreads();
     if (CS == 1) {
-      for (int e = tid; e < TILE; e += NT) {
+#pragma unroll
+      for (int j = 0; j < EPI; ++j) {
+        const int e = tid + j * NT;
         float sum = 0.f;
 #pragma unroll
-        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILE + e];
-        bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum);
+        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+        bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum, pre[j]);
       }
       __syncthreads();   // before the next pass refills the stages
     } else {
+      // this rank's partial sums go straight into the shared memory of the rank that finishes the element
+      // (element e belongs to rank e % CS), one slice per sending rank
+      const int per = TILE / CS;
       for (int e = tid; e < TILE; e += NT) {
         float sum = 0.f;
 #pragma unroll
-        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILE + e];
-        s_part[e] = sum;
+        for (int w = 0; w < NWARP; ++w) sum += s_tiles[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+        cluster.map_shared_rank(s_part, e % CS)[rank * per + e / CS] = sum;
       }
       cluster.sync();
-      // every rank finishes a share of the tile: totals summed over the ranks in rank order
-      for (int e = rank + CS * tid; e < TILE; e += CS * NT) {
-        float sum = 0.f;
-        for (int r = 0; r < CS; ++r) sum += cluster.map_shared_rank(s_part, r)[e];
-        bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum);
+      // totals summed over the ranks in rank order
+#pragma unroll
+      for (int j = 0; j < EPI; ++j) {
+        const int q = tid + j * NT;   // q-th element of this rank: e = rank + CS q
+        if (q < per) {
+          float sum = 0.f;
+          for (int r = 0; r < CS; ++r) sum += s_part[r * per + q];
+          const int e = rank + CS * q;
+          bwd_epilogue(p, L, tile_row0 + e / BP, bp0 + e % BP, sum, pre[j]);
+        }
       }
-      cluster.sync();  // nobody leaves or overwrites s_part / the stages while another rank still reads
+      // no rank reads another one's memory after the barrier above: a rank may leave on its own; before
+      // another pass, though, everybody must have read the slices this pass delivered
+      if (bp0 + BP < p.B) cluster.sync();
     }
   }
 }
