@@ -39,6 +39,23 @@ def read_peaks():
     return 6650.0, "fallback"
 
 
+# DRAM bytes (read + written) of one launch of a pass's kernel from one ncu capture of this workload
+# (dram__bytes_read.sum + dram__bytes_write.sum; summaries under profiles/).  Reported only while the
+# kernel source still has the hash it had when the counters were taken.
+NCU_KERNELS_SHA256 = ""
+NCU_TRAFFIC = {}   # (workload, phase) -> bytes per launch
+
+
+def ncu_traffic(workload: str, phase: str):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2412_11810_b200", "csrc", "kernels.cuh")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    return NCU_TRAFFIC.get((workload, phase)) if sha == NCU_KERNELS_SHA256 else None
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -253,14 +270,19 @@ def run_ours(args, rank, world):
                             "dw": dw_bytes(w, activity, w.B, min(seg, w.T))}.get(dominant)
         roof = None
         if per_launch_bytes and ph[dominant][1] > 0:
-            avg_s = ph[dominant][0] / 1e3 / ph[dominant][1]
+            kernel = {"fwd": "fwd_step_kernel<true>", "refwd1": "fwd_step_kernel<false>",
+                      "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel", "dw": "dw_kernel"}[dominant]
+            units = ph[dominant][1]
+            if dominant == "fwd" and ph["fwd"][1] < w.T:
+                # small spiking networks: one cooperative launch per forward operation, T steps in all;
+                # the bytes are per step, so the launch count is replaced by the step count
+                kernel, units = "fwd_resident_kernel / fwd_segment_kernel (per step)", w.T
+            avg_s = ph[dominant][0] / 1e3 / units
             ach = per_launch_bytes / avg_s / 1e9
-            roof = {"bound": "hbm", "kernel": {"fwd": "fwd_step_kernel<true>", "refwd1": "fwd_step_kernel<false>",
-                                               "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel",
-                                               "dw": "dw_kernel"}[dominant],
+            roof = {"bound": "hbm", "kernel": kernel,
                     "phase": dominant,
                     "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak,
-                    "traffic": None, "algorithmic_bytes_per_launch": per_launch_bytes,
+                    "traffic": ncu_traffic(w.name, dominant), "algorithmic_bytes_per_launch": per_launch_bytes,
                     "avg_launch_us": avg_s * 1e6, "launches_per_step": ph[dominant][1]}
         # the other strategies on the same workload (fewer steps), for the per-strategy table
         per_strategy = {}

@@ -645,7 +645,7 @@ __global__ void __launch_bounds__(128) refwd_scan_kernel(const __grid_constant__
 // layer l) can start step t only when the spike words of (l, t-1, b) and (l-1, t, b) are complete.
 // These are the only dependences: samples never wait for one another and a lower layer may run
 // ahead of a higher one.  Each (layer, sample) has a counter of finished (tile, step) pairs; a
-// producer publishes its words with a fence and an atomic add, a consumer polls the counter with
+// producer publishes its words with a release add to the counter, a consumer polls the counter with
 // acquire loads and then reads the words past L1.  Every buffer a step writes is indexed by the
 // step or owned by the writing thread, so running ahead overwrites nothing that is still needed.
 // All CTAs must be resident together (cooperative launch); a wait that does not end within
@@ -688,6 +688,12 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+
+// Publishes one more finished (tile, step) pair.  Called by one thread after a CTA barrier: the release makes
+// everything the CTA wrote before that barrier visible to whoever reads the new count with an acquire load.
+__device__ __forceinline__ void publish_progress(uint32_t* counter) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
 }
 
 __device__ __forceinline__ bool wait_progress(const uint32_t* counter, uint32_t target) {
@@ -837,8 +843,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
     }
     __syncthreads();
     if (tid == 0) {   // publish: this tile's words of step t are complete
-      __threadfence();
-      atomicAdd(my_progress, 1u);
+      publish_progress(my_progress);
     }
   }
 }
@@ -1152,8 +1157,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
     }
     __syncthreads();
     if (tid == 0) {   // publish: this CTA's spike bits of step t are complete
-      __threadfence();
-      atomicAdd(my_progress, 1u);
+      publish_progress(my_progress);
     }
   }
 }
