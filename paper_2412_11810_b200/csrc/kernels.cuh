@@ -1629,8 +1629,8 @@ struct DwParams {
 
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
 constexpr int DW_WINDOW = 1024;   // (t, b) pairs compacted at a time
-// delta rows per copy group: 4, or 2 for the widest column tile (keeps the ring at 64 KB per CTA)
-template <int U> __host__ __device__ constexpr int dw_group() { return U >= 4 ? 2 : 4; }
+// delta rows per copy group: 4, 2 or 1 as the column tile widens (keeps the ring at 64 KB per CTA)
+template <int U> __host__ __device__ constexpr int dw_group() { return U >= 8 ? 1 : U >= 4 ? 2 : 4; }
 constexpr int DW_STAGES = 2;      // copy groups in flight per warp
 
 // shared memory of dw_kernel in bytes for a window of `window` pairs

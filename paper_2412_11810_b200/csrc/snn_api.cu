@@ -747,8 +747,9 @@ struct Exec {
         if (graded()) { r.off_row0 = off(l, ta); r.pref_row0 = pref(l, ta); r.vals = vals(l); r.cap = lo.cap[l]; }
       }
       // wider column tiles for wider layers: the per-CTA compaction of the pair lists is amortised over more columns
-      if (maxN >= 4096) launch_dw<4>(d, maxN, maxNpre);
-      else if (maxN >= 1024) launch_dw<2>(d, maxN, maxNpre);
+      if (maxN >= 1024) launch_dw<8>(d, maxN, maxNpre);
+      else if (maxN >= 512) launch_dw<4>(d, maxN, maxNpre);
+      else if (maxN >= 256) launch_dw<2>(d, maxN, maxNpre);
       else launch_dw<1>(d, maxN, maxNpre);
     }
     end_span(span);
@@ -871,6 +872,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, true>(DW_WINDOW)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, true>(DW_WINDOW)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<4, false>(DW_WINDOW)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<8, false>(DW_WINDOW)));
+      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<8, true>(DW_WINDOW)));
       CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<4, true>(DW_WINDOW)));
       smem_opt_in = true;
     }
