@@ -142,6 +142,11 @@ snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const s
  * 200 KB; at most one thread block of 16 neurons per SM over all layers) keep their weights in shared
  * memory during a forward launch.  This flag makes them stream the weights from L2 like larger ones. */
 #define SNN_FLAG_FORWARD_STREAM_WEIGHTS 128u
+/* Networks small enough that 32 rows of a layer's recurrent and next feed-forward matrix fit in shared
+ * memory beside the staging buffers (per cluster rank) run the backward pass of a segment as one
+ * cooperative launch with those weights resident.  This flag forces one launch per step.  Results are
+ * bit-identical either way. */
+#define SNN_FLAG_BACKWARD_PER_STEP 256u
 
 typedef struct {
   int32_t T, B;

@@ -1474,6 +1474,275 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
 }
 
 // ------------------------------------------------------------------------------------------
+// Backward pass over a whole segment in one cooperative launch, the weights resident in shared memory
+// (networks small enough that a CTA's slice of both matrices, 32 rows x its share of the contraction
+// index, fits beside the staging ring).
+//
+// Same tiling, same arithmetic and the same order of additions as bwd_step_kernel (results are
+// bit-identical), but a CTA loads its slice of W_ff(l+1) and W_rec once and then walks through the steps
+// t1 .. t0+1 itself; per step only delta streams through the cp.async ring.  Layer l may start step t
+// when all of delta^l_{t+1} and delta^{l+1}_t is written: one counter of finished (CTA, step) pairs per
+// layer, published with a release add after a CTA barrier, polled with acquire loads; delta is then
+// read past L1.  The slices a rank receives from the other ranks of its cluster alternate between two
+// buffers, so a rank that is one step ahead never overwrites what a slower one still reads.  A wait
+// that runs out raises STATUS_SYNC_TIMEOUT; the CTA then stops waiting but keeps taking part in every
+// barrier until the end of the launch (a CTA that left early would block its cluster).
+struct BwdSegLayer {
+  const float* W_rec;       // [N][N]
+  const float* W_ffa;       // W_ff of the layer above [N][N_post] or null
+  const float* g_out;       // [B][N] (last layer) or null
+  const float* carry_in;    // [B][N] delta^l_{t1+1}
+  float* carry_out;         // [B][N] receives delta^l_{t0+1}
+  size_t state_off;         // offset of this layer inside a state slot, in floats
+  size_t state_off_above;   // of the layer above
+  int N, N_post;
+  int ctas;                 // CTAs of this layer (row tiles x cluster size)
+  int cta0;                 // blockIdx.x of its first CTA (a multiple of the cluster size)
+};
+
+struct BwdSegParams {
+  BwdSegLayer lay[MAXL];
+  float* slots;
+  size_t slot_stride;       // floats
+  uint32_t* status;
+  uint32_t* progress;       // [L] finished (CTA, step) pairs per layer, zero at launch
+  int L, B, t0, t1, buf_slot;   // step t lives in slot buf_slot + (t - t0 - 1): V_t on entry, delta_t on exit
+  float alpha, theta, beta;
+  int surrogate, cell;
+};
+
+constexpr int BSEG_STAGES = 4;   // chunks of delta in flight per CTA
+
+// floats of the resident slice per row: every chunk of 128 k (feed-forward part first, each part padded to
+// whole chunks with zeros) plus 4 so that fragment loads hit 32 banks
+__host__ __device__ inline int bwd_resident_ld(int k_ff, int k_rec) {
+  return ((k_ff + 127) / 128 + (k_rec + 127) / 128) * 128 + 4;
+}
+template <int NTN, int NWARP> __host__ __device__ constexpr size_t bwd_segment_region_floats() {
+  // the delta ring, reused for the warps' partial tiles
+  return (size_t)(BSEG_STAGES * 8 * NTN * BWD_LD) > (size_t)(NWARP * BWD_TM * (8 * NTN + 8))
+             ? (size_t)(BSEG_STAGES * 8 * NTN * BWD_LD) : (size_t)(NWARP * BWD_TM * (8 * NTN + 8));
+}
+
+template <int NTN, int NWARP>
+__global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid_constant__ BwdSegParams p) {
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, DSTAGE_F = BP * BWD_LD, TILE = BWD_TM * BP;
+  constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
+  constexpr int EPI = TILE / NT;
+  constexpr int ITER = BP * 32 / NT;   // 16-byte pieces of a delta chunk per thread
+  static_assert(TILE % NT == 0 && BP * 32 % NT == 0, "tiles divide evenly among the threads");
+  cg::cluster_group cluster = cg::this_cluster();
+  const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  int l = 0;
+  while (l + 1 < p.L && (int)blockIdx.x >= p.lay[l + 1].cta0) ++l;
+  const BwdSegLayer& L = p.lay[l];
+  const int tile_row0 = (((int)blockIdx.x - L.cta0) / CS) * BWD_TM;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t4 = lane & 3;
+  const bool above = L.W_ffa != nullptr;
+  __shared__ float s_part[2][TILE];
+  __shared__ int s_ok, s_dead;
+  extern __shared__ float4 s_dyn[];
+  // this rank's slice of each contraction range, in units of 4 floats
+  const int q_rec = L.N / 4, q_ff = above ? L.N_post / 4 : 0;
+  const int lo_rec = (int)((long long)q_rec * rank / CS) * 4, hi_rec = (int)((long long)q_rec * (rank + 1) / CS) * 4;
+  const int lo_ff = (int)((long long)q_ff * rank / CS) * 4, hi_ff = (int)((long long)q_ff * (rank + 1) / CS) * 4;
+  const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
+  const int LDW = it_all * 128 + 4;
+  float* const Wres = reinterpret_cast<float*>(s_dyn);             // [32][LDW]
+  float* const s_reg = Wres + (size_t)BWD_TM * LDW;                // delta ring [BSEG_STAGES][BP][BWD_LD]; later partial tiles
+  const int rlast = L.N - 1, blast = p.B - 1;
+
+  // ---- the resident slice: rows tile_row0 .. +31, chunk by chunk, zeros past a part's end and past row N-1
+  for (int q = tid; q < BWD_TM * it_all * 32; q += NT) {
+    const int rr = q / (it_all * 32), c4 = q % (it_all * 32), it = c4 >> 5, kc = (c4 & 31) * 4;
+    const bool ff = it < it_ff;
+    const int k = ff ? lo_ff + it * 128 + kc : lo_rec + (it - it_ff) * 128 + kc;
+    const bool real = tile_row0 + rr <= rlast && k < (ff ? hi_ff : hi_rec);
+    const float* src = ff ? L.W_ffa + (size_t)(tile_row0 + rr) * L.N_post + k : L.W_rec + (size_t)(tile_row0 + rr) * L.N + k;
+    cp_async16_or_zero(Wres + (size_t)rr * LDW + c4 * 4, real ? src : L.W_rec, real);
+  }
+  cp_async_commit();
+  if (tid == 0) s_dead = 0;
+  cp_async_wait<0>();
+  __syncthreads();
+
+  uint32_t* const my_progress = p.progress + l;
+  const int n_steps = p.t1 - p.t0;
+  for (int d = 1; d <= n_steps; ++d) {
+    const int t = p.t1 - d + 1;
+    if (tid == 0) {
+      bool ok = s_dead == 0;
+      if (ok) ok = wait_progress(my_progress, (uint32_t)L.ctas * (uint32_t)(d - 1));
+      if (ok && above) ok = wait_progress(p.progress + (l + 1), (uint32_t)p.lay[l + 1].ctas * (uint32_t)d);
+      if (!ok && s_dead == 0) { atomicOr(p.status, STATUS_SYNC_TIMEOUT); s_dead = 1; }
+      s_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    const bool live = s_ok != 0;   // after a timeout the CTA only keeps the barriers going
+    float* const Vd = p.slots + (size_t)(p.buf_slot + (t - p.t0 - 1)) * p.slot_stride + L.state_off;
+    const float* const dn = d == 1 ? L.carry_in
+                                   : p.slots + (size_t)(p.buf_slot + (t - p.t0)) * p.slot_stride + L.state_off;
+    const float* const da = above ? p.slots + (size_t)(p.buf_slot + (t - p.t0 - 1)) * p.slot_stride + L.state_off_above
+                                  : nullptr;
+    float* const part = s_part[d & 1];
+
+    for (int bp0 = 0; bp0 < p.B; bp0 += BP) {
+      // what the epilogue needs, fetched now (delta_{t+1} was written by other CTAs of this launch: past L1)
+      float pre_dn[EPI], pre_go[EPI], pre_v[EPI];
+#pragma unroll
+      for (int j = 0; j < EPI; ++j) {
+        const int q = tid + j * NT, e = CS == 1 ? q : rank + CS * q;
+        const int i = tile_row0 + e / BP, b = bp0 + e % BP;
+        pre_dn[j] = pre_go[j] = pre_v[j] = 0.f;
+        if (live && e < TILE && i < L.N && b < p.B) {
+          const size_t k = (size_t)b * L.N + i;
+          pre_dn[j] = __ldcg(dn + k);
+          pre_go[j] = L.g_out ? L.g_out[k] : 0.f;
+          pre_v[j] = Vd[k];
+        }
+      }
+      // delta rows of this pass: fixed (sample, 16-byte column) positions per thread
+      const float* src_rec[ITER];
+      const float* src_ff[ITER];
+      int dst_off[ITER], kcol[ITER];
+#pragma unroll
+      for (int j = 0; j < ITER; ++j) {
+        const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
+        kcol[j] = 4 * c4;
+        dst_off[j] = rr * BWD_LD + 4 * c4;
+        const size_t b = bp0 + rr < blast ? bp0 + rr : blast;   // samples past the batch: a valid row, never used
+        src_rec[j] = dn + b * L.N + 4 * c4;
+        src_ff[j] = above ? da + b * L.N_post + 4 * c4 : nullptr;
+      }
+      auto issue_part = [&](int it, int j0, int j1) {
+        if (it < it_all) {
+          const bool ff = it < it_ff;
+          const int k0 = ff ? lo_ff + it * 128 : lo_rec + (it - it_ff) * 128;
+          const int hi = ff ? hi_ff : hi_rec;
+          float* st = s_reg + (size_t)(it % BSEG_STAGES) * DSTAGE_F;
+#pragma unroll
+          for (int j = 0; j < ITER; ++j) {
+            if (j < j0 || j >= j1) continue;
+            if (k0 + kcol[j] < hi) cp_async16(st + dst_off[j], (ff ? src_ff[j] : src_rec[j]) + k0);
+            else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+      };
+      float acc[2][NTN][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+      for (int it = 0; it < BSEG_STAGES - 1; ++it) { issue_part(it, 0, ITER); cp_async_commit(); }
+      for (int it = 0; it < it_all; ++it) {
+        cp_async_wait<BSEG_STAGES - 2>();
+        __syncthreads();
+        const int it_refill = it + BSEG_STAGES - 1;
+        bool refill = true;
+        const float* Wc = Wres + it * 128;
+        const float* Ds = s_reg + (size_t)(it % BSEG_STAGES) * DSTAGE_F;
+#pragma unroll 1
+        for (int ks = warp; ks < 16; ks += NWARP) {
+          const int kk = ks * 8 + t4;
+          uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            const float* r0 = Wc + (size_t)(mt * 16 + g) * LDW + kk;
+            split_tf32(r0[0], a_hi[mt][0], a_lo[mt][0]);
+            split_tf32(r0[(size_t)8 * LDW], a_hi[mt][1], a_lo[mt][1]);
+            split_tf32(r0[4], a_hi[mt][2], a_lo[mt][2]);
+            split_tf32(r0[(size_t)8 * LDW + 4], a_hi[mt][3], a_lo[mt][3]);
+          }
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) {
+            const float* r0 = Ds + (nt * 8 + g) * BWD_LD + kk;
+            split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
+            split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
+          }
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
+          if (refill) issue_part(it_refill, 0, ITER / 2);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
+          if (refill) {
+            issue_part(it_refill, ITER / 2, ITER);
+            cp_async_commit();
+            refill = false;
+          }
+        }
+      }
+      cp_async_wait<0>();
+      __syncthreads();   // the ring is free: it now holds the warps' partial tiles [NWARP][32][TS]
+      {
+        float* mine = s_reg + (size_t)warp * TILEP;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) {
+            const int r = mt * 16 + g, c = nt * 8 + 2 * t4;
+            *reinterpret_cast<float2*>(mine + r * TS + c) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2*>(mine + (r + 8) * TS + c) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+          }
+      }
+      __syncthreads();
+      auto finish = [&](int e, float sum, int j) {
+        const int i = tile_row0 + e / BP, b = bp0 + e % BP;
+        if (!live || i >= L.N || b >= p.B) return;
+        const size_t k = (size_t)b * L.N + i;
+        float gsum = sum + pre_go[j];
+        if (p.cell == 0) gsum = fmaf(-p.theta, pre_dn[j], gsum);
+        const float sp = surrogate_grad(pre_v[j], p.theta, p.beta, p.surrogate, p.cell);
+        const float dl = fmaf(gsum, sp, p.alpha * pre_dn[j]);
+        Vd[k] = dl;
+        if (t == p.t0 + 1) L.carry_out[k] = dl;
+      };
+      if (CS == 1) {
+#pragma unroll
+        for (int j = 0; j < EPI; ++j) {
+          const int e = tid + j * NT;
+          float sum = 0.f;
+#pragma unroll
+          for (int w = 0; w < NWARP; ++w) sum += s_reg[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+          finish(e, sum, j);
+        }
+        __syncthreads();   // before the ring is refilled
+      } else {
+        const int per = TILE / CS;
+        for (int e = tid; e < TILE; e += NT) {
+          float sum = 0.f;
+#pragma unroll
+          for (int w = 0; w < NWARP; ++w) sum += s_reg[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+          cluster.map_shared_rank(part, e % CS)[rank * per + e / CS] = sum;
+        }
+        cluster.sync();   // also a CTA barrier: the ring may be refilled after it
+#pragma unroll
+        for (int j = 0; j < EPI; ++j) {
+          const int q = tid + j * NT;
+          if (q < per) {
+            float sum = 0.f;
+            for (int r = 0; r < CS; ++r) sum += part[r * per + q];
+            finish(rank + CS * q, sum, j);
+          }
+        }
+        if (bp0 + BP < p.B) cluster.sync();   // another pass of this step reuses the same buffer
+      }
+    }
+    __syncthreads();
+    if (tid == 0 && live) publish_progress(my_progress);   // this CTA's share of delta_t is written
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Time-batched feed-forward part of the backward pass: for a run of steps the deltas of the layer
 // above are all known before the layer below starts, so W_ff^{l+1} delta^{l+1}_t is one product
 // with M = steps x B columns instead of one per step:

@@ -629,6 +629,66 @@ struct Exec {
 
   // BWD: layer wavefront, layer l runs L-l steps behind the last layer; then the weight
   // gradients of the whole segment.
+  // BWD as one cooperative launch of thread-block clusters (bwd_segment_kernel), if every CTA's slice of the
+  // weights fits in shared memory and the device can hold all clusters at once; otherwise `done` stays false.
+  template <int NTN, int NWARP> snn_status try_backward_segment(const snn_op& op, int CS, bool& done) {
+    const auto& sz = net->sizes;
+    done = false;
+    BwdSegParams p;
+    std::memset(&p, 0, sizeof p);
+    size_t res_floats = 0;
+    int ctas = 0;
+    for (int l = 1; l <= L; ++l) {
+      BwdSegLayer& f = p.lay[l - 1];
+      f.N = sz[l]; f.N_post = l < L ? sz[l + 1] : 0;
+      f.W_rec = a->W_rec[l - 1];
+      f.W_ffa = l < L ? a->W_ff[l] : nullptr;
+      f.g_out = l == L ? at<float>(lo.g_out) : nullptr;
+      f.carry_in = carry(carry_cur, l);
+      f.carry_out = carry(carry_cur ^ 1, l);
+      f.state_off = lo.layer_off[l];
+      f.state_off_above = l < L ? lo.layer_off[l + 1] : 0;
+      f.ctas = (sz[l] + BWD_TM - 1) / BWD_TM * CS;
+      f.cta0 = ctas;
+      ctas += f.ctas;
+      const int q_rec = f.N / 4, q_ff = f.N_post / 4;
+      for (int r = 0; r < CS; ++r) {
+        const int k_rec = (int)((long long)q_rec * (r + 1) / CS) * 4 - (int)((long long)q_rec * r / CS) * 4;
+        const int k_ff = (int)((long long)q_ff * (r + 1) / CS) * 4 - (int)((long long)q_ff * r / CS) * 4;
+        res_floats = std::max(res_floats, (size_t)BWD_TM * bwd_resident_ld(k_ff, k_rec));
+      }
+    }
+    const size_t smem = 4 * (res_floats + bwd_segment_region_floats<NTN, NWARP>());
+    if (smem > ((size_t)218 << 10)) return SNN_OK;
+    void (*k)(BwdSegParams) = bwd_segment_kernel<NTN, NWARP>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(32 * NWARP); cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cudaLaunchAttribute at2[2];
+    at2[0].id = cudaLaunchAttributeCooperative; at2[0].val.cooperative = 1;
+    at2[1].id = cudaLaunchAttributeClusterDimension;
+    at2[1].val.clusterDim.x = CS; at2[1].val.clusterDim.y = 1; at2[1].val.clusterDim.z = 1;
+    cfg.attrs = at2; cfg.numAttrs = 2;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      cudaGetLastError();
+      return SNN_OK;
+    }
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) != cudaSuccess || (long long)clusters * CS < ctas) {
+      cudaGetLastError();
+      return SNN_OK;
+    }
+    p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
+    p.status = at<uint32_t>(lo.status); p.progress = at<uint32_t>(lo.progress);
+    p.L = L; p.B = B; p.t0 = op.t0; p.t1 = op.t1; p.buf_slot = op.buf_slot;
+    p.alpha = net->alpha; p.theta = net->theta; p.beta = net->beta;
+    p.surrogate = net->surrogate; p.cell = net->cell;
+    CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L, main));
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, p));
+    ++launches;
+    done = true;
+    return SNN_OK;
+  }
+
   snn_status run_backward(const snn_op& op) {
     const auto& sz = net->sizes;
     const int n = op.t1 - op.t0;
@@ -650,7 +710,17 @@ struct Exec {
     int span = begin_span(SNN_PHASE_BWD);
     const bool layer_major = L > 1 && ((a->flags & SNN_FLAG_BACKWARD_LAYER_BY_LAYER) ||
                                        (lo.layer_major && !(a->flags & SNN_FLAG_BACKWARD_WAVEFRONT)));
-    if (layer_major) {
+    bool segment_done = false;
+    if (!layer_major && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
+      // small networks: the whole segment in one cooperative launch, the weights resident in shared memory
+      snn_status st = SNN_OK;
+      if (B <= 8) st = try_backward_segment<1, 8>(op, CS, segment_done);
+      else if (B <= 16) st = try_backward_segment<2, 8>(op, CS, segment_done);
+      else st = try_backward_segment<4, 16>(op, CS, segment_done);
+      if (st != SNN_OK) return st;
+    }
+    if (segment_done) {
+    } else if (layer_major) {
       // Runs of at most BWD_RUN steps, latest first; within a run the layers go from the last to the first:
       // the feed-forward term of layer l for the whole run is one product (ff_gemm_kernel), then the steps
       // of layer l follow one launch each.

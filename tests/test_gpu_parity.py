@@ -473,3 +473,32 @@ def test_graded_reforward_as_one_launch_per_segment(orc32):
             for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
                 assert np.array_equal(x, y), (strat, K, R, flags)
     s.close()
+
+
+def test_backward_as_one_launch_per_segment(orc32):
+    """Small networks run the backward pass of a segment as one cooperative launch with the weights in
+    shared memory; it must give the bits of the one-launch-per-step kernel, for every batch tiling
+    (1, 8, 16, 32 samples per pass, several passes), ragged row tiles, clusters of several sizes, one to
+    three layers, and agree with the oracle."""
+    b = sb()
+    cases = [
+        wl.small(sizes=(70, 700, 1300, 7), T=37, B=5, p_in=0.05, g_ff=(2.5, 1.4), g_rec=(1.0, 1.0), seed=61),
+        wl.small(sizes=(33, 520, 260, 600, 9), T=29, B=11, p_in=0.1, g_ff=(2.5, 1.5, 1.5), g_rec=(1.0, 1.0, 1.0), seed=62),
+        wl.small(sizes=(64, 1024, 6), T=21, B=32, p_in=0.05, g_ff=(2.5,), g_rec=(1.0,), seed=63),
+        wl.small(sizes=(64, 300, 200, 6), T=17, B=40, p_in=0.1, g_ff=(2.5, 1.5), g_rec=(1.0, 1.0), seed=64),
+        wl.small(sizes=(20, 24, 12, 5), T=13, B=1, p_in=0.2, seed=65),
+    ]
+    for w in cases:
+        d = wl.make(w)
+        ref = run_oracle(orc32, w, d)
+        s, bits, targets = make_session(w, d)
+        s.train_step(bits, targets, strategy=0, max_activity=1.0, extra_flags=b.SNN_FLAG_BACKWARD_PER_STEP)
+        assert_grads_close(s.gradients(), ref)
+        base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+        for strat, K, R in [(0, 0, 0), (1, 7, 0), (1, 40, 0), (3, 4, 16), (2, 5, 0)]:
+            for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+                g.fill_(float("nan"))
+            s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0)
+            for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+                assert np.array_equal(x, y), (w.sizes, w.B, strat, K, R)
+        s.close()
