@@ -277,6 +277,9 @@ def run_ours(args, rank, world):
                 # small spiking networks: one cooperative launch per forward operation, T steps in all;
                 # the bytes are per step, so the launch count is replaced by the step count
                 kernel, units = "fwd_resident_kernel / fwd_segment_kernel (per step)", w.T
+            if dominant == "bwd" and ph["bwd"][1] < w.T:
+                # small networks: one cooperative launch per segment with the weights resident
+                kernel, units = "bwd_segment_kernel (per step)", w.T
             avg_s = ph[dominant][0] / 1e3 / units
             ach = per_launch_bytes / avg_s / 1e9
             roof = {"bound": "hbm", "kernel": kernel,
