@@ -212,7 +212,7 @@ def run_ours(args, rank, world):
     bits, targets = bits_host.to(s.device), tg_host.to(s.device)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=s.device)   # larger than the 126 MB L2
     kw = dict(strategy=w.strategy, chunk_size=w.chunk_size, remote_chunk_size=w.remote_chunk_size,
-              max_activity=args.max_activity)
+              max_activity=args.max_activity, extra_flags=args.flags)
 
     def timed_steps(n, inp, tg, **extra):
         """n steps, each bracketed by CUDA events on the library's main stream; L2 flushed between."""
@@ -372,6 +372,8 @@ def main():
     ap.add_argument("--max-activity", type=float, default=0.25)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-strategies", action="store_true", help="skip the per-strategy table")
+    ap.add_argument("--flags", type=int, default=0,
+                    help="extra SNN_FLAG_* bits for the timed strategy, e.g. 256 = backward with one launch per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -1480,7 +1480,8 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
 //
 // Same tiling, same arithmetic and the same order of additions as bwd_step_kernel (results are
 // bit-identical), but a CTA loads its slice of W_ff(l+1) and W_rec once and then walks through the steps
-// t1 .. t0+1 itself; per step only delta streams through the cp.async ring.  Layer l may start step t
+// t1 .. t0+1 itself; per step only delta streams in, every warp staging the values of its own k-steps
+// in a cp.async ring of its own (no barrier between warps inside the contraction).  Layer l may start step t
 // when all of delta^l_{t+1} and delta^{l+1}_t is written: one counter of finished (CTA, step) pairs per
 // layer, published with a release add after a CTA barrier, polled with acquire loads; delta is then
 // read past L1.  The slices a rank receives from the other ranks of its cluster alternate between two
@@ -1511,7 +1512,8 @@ struct BwdSegParams {
   int surrogate, cell;
 };
 
-constexpr int BSEG_STAGES = 4;   // chunks of delta in flight per CTA
+constexpr int BSEG_STAGES = 3;   // chunks of delta in flight per warp
+constexpr int BSEG_LD = 12;      // floats per (k-step, sample) row of a warp's delta stage: 8 k + 4, fragment loads hit 32 banks
 
 // floats of the resident slice per row: every chunk of 128 k (feed-forward part first, each part padded to
 // whole chunks with zeros) plus 4 so that fragment loads hit 32 banks
@@ -1519,18 +1521,21 @@ __host__ __device__ inline int bwd_resident_ld(int k_ff, int k_rec) {
   return ((k_ff + 127) / 128 + (k_rec + 127) / 128) * 128 + 4;
 }
 template <int NTN, int NWARP> __host__ __device__ constexpr size_t bwd_segment_region_floats() {
-  // the delta ring, reused for the warps' partial tiles
-  return (size_t)(BSEG_STAGES * 8 * NTN * BWD_LD) > (size_t)(NWARP * BWD_TM * (8 * NTN + 8))
-             ? (size_t)(BSEG_STAGES * 8 * NTN * BWD_LD) : (size_t)(NWARP * BWD_TM * (8 * NTN + 8));
+  // the warps' delta rings (16 k-steps of a chunk x BP samples x BSEG_LD per stage), reused for their partial tiles
+  return (size_t)(BSEG_STAGES * 16 * 8 * NTN * BSEG_LD) > (size_t)(NWARP * BWD_TM * (8 * NTN + 8))
+             ? (size_t)(BSEG_STAGES * 16 * 8 * NTN * BSEG_LD) : (size_t)(NWARP * BWD_TM * (8 * NTN + 8));
 }
 
 template <int NTN, int NWARP>
 __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid_constant__ BwdSegParams p) {
-  constexpr int NT = 32 * NWARP, BP = 8 * NTN, DSTAGE_F = BP * BWD_LD, TILE = BWD_TM * BP;
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, TILE = BWD_TM * BP;
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
   constexpr int EPI = TILE / NT;
-  constexpr int ITER = BP * 32 / NT;   // 16-byte pieces of a delta chunk per thread
-  static_assert(TILE % NT == 0 && BP * 32 % NT == 0, "tiles divide evenly among the threads");
+  constexpr int KS = 16 / NWARP;                 // k-steps of a chunk per warp
+  constexpr int WSTAGE_F = KS * BP * BSEG_LD;    // floats of one warp's stage: its k-steps x BP samples x 8 k (padded)
+  constexpr int PIECES = KS * BP * 2;            // 16-byte pieces of it
+  constexpr int ITER = (PIECES + 31) / 32;       // per lane
+  static_assert(TILE % NT == 0 && 16 % NWARP == 0, "tiles divide evenly among the threads");
   cg::cluster_group cluster = cg::this_cluster();
   const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   int l = 0;
@@ -1549,7 +1554,8 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
   const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
   const int LDW = it_all * 128 + 4;
   float* const Wres = reinterpret_cast<float*>(s_dyn);             // [32][LDW]
-  float* const s_reg = Wres + (size_t)BWD_TM * LDW;                // delta ring [BSEG_STAGES][BP][BWD_LD]; later partial tiles
+  float* const s_reg = Wres + (size_t)BWD_TM * LDW;                // per-warp delta rings [NWARP][BSEG_STAGES][KS][BP][BSEG_LD]; later partial tiles
+  float* const ring = s_reg + (size_t)warp * BSEG_STAGES * WSTAGE_F;
   const int rlast = L.N - 1, blast = p.B - 1;
 
   // ---- the resident slice: rows tile_row0 .. +31, chunk by chunk, zeros past a part's end and past row N-1
@@ -1601,32 +1607,36 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
           pre_v[j] = Vd[k];
         }
       }
-      // delta rows of this pass: fixed (sample, 16-byte column) positions per thread
+      // Every warp stages the delta values of its own k-steps (8 k x BP samples each: two 16-byte pieces per
+      // sample) in a ring of its own, so that no warp waits for another one inside the contraction and the
+      // loads, splits and tensor-core passes of different warps overlap.  A lane copies fixed pieces.
       const float* src_rec[ITER];
       const float* src_ff[ITER];
-      int dst_off[ITER], kcol[ITER];
+      int dst_off[ITER], kofs[ITER];
 #pragma unroll
       for (int j = 0; j < ITER; ++j) {
-        const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
-        kcol[j] = 4 * c4;
-        dst_off[j] = rr * BWD_LD + 4 * c4;
-        const size_t b = bp0 + rr < blast ? bp0 + rr : blast;   // samples past the batch: a valid row, never used
-        src_rec[j] = dn + b * L.N + 4 * c4;
-        src_ff[j] = above ? da + b * L.N_post + 4 * c4 : nullptr;
+        const int q = lane + j * 32;                                   // piece: (k-step of the warp, sample, half)
+        const int ksl = q / (BP * 2), sm = (q / 2) % BP, half = q & 1;
+        kofs[j] = q < PIECES ? (warp + ksl * NWARP) * 8 + half * 4 : -1;   // k inside the chunk
+        dst_off[j] = (ksl * BP + sm) * BSEG_LD + half * 4;
+        const size_t b = bp0 + sm < blast ? bp0 + sm : blast;           // samples past the batch: a valid row, never used
+        src_rec[j] = dn + b * L.N;
+        src_ff[j] = above ? da + b * L.N_post : nullptr;
       }
-      auto issue_part = [&](int it, int j0, int j1) {
+      auto issue = [&](int it) {
         if (it < it_all) {
           const bool ff = it < it_ff;
           const int k0 = ff ? lo_ff + it * 128 : lo_rec + (it - it_ff) * 128;
           const int hi = ff ? hi_ff : hi_rec;
-          float* st = s_reg + (size_t)(it % BSEG_STAGES) * DSTAGE_F;
+          float* st = ring + (size_t)(it % BSEG_STAGES) * WSTAGE_F;
 #pragma unroll
           for (int j = 0; j < ITER; ++j) {
-            if (j < j0 || j >= j1) continue;
-            if (k0 + kcol[j] < hi) cp_async16(st + dst_off[j], (ff ? src_ff[j] : src_rec[j]) + k0);
-            else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kofs[j] < 0) continue;
+            const int k = k0 + kofs[j];
+            cp_async16_or_zero(st + dst_off[j], k < hi ? (ff ? src_ff[j] : src_rec[j]) + k : L.W_rec, k < hi);
           }
         }
+        cp_async_commit();
       };
       float acc[2][NTN][4];
 #pragma unroll
@@ -1635,17 +1645,16 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
         for (int nt = 0; nt < NTN; ++nt)
 #pragma unroll
           for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
-      for (int it = 0; it < BSEG_STAGES - 1; ++it) { issue_part(it, 0, ITER); cp_async_commit(); }
+      for (int it = 0; it < BSEG_STAGES - 1; ++it) issue(it);
       for (int it = 0; it < it_all; ++it) {
-        cp_async_wait<BSEG_STAGES - 2>();
-        __syncthreads();
-        const int it_refill = it + BSEG_STAGES - 1;
-        bool refill = true;
+        cp_async_wait<BSEG_STAGES - 2>();   // this lane's pieces of chunk `it` have landed
+        __syncwarp();                       // ... the whole warp's have, and the warp is done with chunk it-1
+        issue(it + BSEG_STAGES - 1);        // refills the stage chunk it-1 used
         const float* Wc = Wres + it * 128;
-        const float* Ds = s_reg + (size_t)(it % BSEG_STAGES) * DSTAGE_F;
-#pragma unroll 1
-        for (int ks = warp; ks < 16; ks += NWARP) {
-          const int kk = ks * 8 + t4;
+        const float* Ds = ring + (size_t)(it % BSEG_STAGES) * WSTAGE_F;
+#pragma unroll
+        for (int ksl = 0; ksl < KS; ++ksl) {
+          const int kk = (warp + ksl * NWARP) * 8 + t4;
           uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
@@ -1657,15 +1666,15 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
           }
 #pragma unroll
           for (int nt = 0; nt < NTN; ++nt) {
-            const float* r0 = Ds + (nt * 8 + g) * BWD_LD + kk;
+            const float* r0 = Ds + (ksl * BP + nt * 8 + g) * BSEG_LD + t4;
             split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
             split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
           }
+          // small terms first; consecutive instructions go to different accumulators
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
             for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
-          if (refill) issue_part(it_refill, 0, ITER / 2);
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -1674,11 +1683,6 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
           for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
             for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
-          if (refill) {
-            issue_part(it_refill, ITER / 2, ITER);
-            cp_async_commit();
-            refill = false;
-          }
         }
       }
       cp_async_wait<0>();

@@ -683,7 +683,10 @@ struct Exec {
     p.alpha = net->alpha; p.theta = net->theta; p.beta = net->beta;
     p.surrogate = net->surrogate; p.cell = net->cell;
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L, main));
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, p));
+    if (cudaLaunchKernelEx(&cfg, k, p) != cudaSuccess) {   // e.g. refused under a profiler: one launch per step instead
+      cudaGetLastError();
+      return SNN_OK;
+    }
     ++launches;
     done = true;
     return SNN_OK;
