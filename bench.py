@@ -40,20 +40,42 @@ def read_peaks():
 
 
 # DRAM bytes (read + written) of one launch of a pass's kernel from one ncu capture of this workload
-# (dram__bytes_read.sum + dram__bytes_write.sum; summaries under profiles/).  Reported only while the
-# kernel source still has the hash it had when the counters were taken.
-NCU_KERNELS_SHA256 = ""
-NCU_TRAFFIC = {}   # (workload, phase) -> bytes per launch
+# (dram__bytes_read.sum + dram__bytes_write.sum; summaries under profiles/): (workload, phase) -> (kernel,
+# sha256 of the kernel's source text when the counters were taken, bytes per launch).  Reported only while
+# the kernel still has that text.  The backward pass of c2 now runs in bwd_segment_kernel, a cooperative launch
+# of thread-block clusters that the profiler cannot launch: no counters, hence no entry.
+NCU_TRAFFIC = {
+    ("c4", "bwd"): ("bwd_step_kernel", "41ed2477e69ea0abdff4478e5d8fcc71fbe2997db65a8bf332fd66406d046db3",
+                    269443328 + 4209920),
+    ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
+                    388252416 + 4982784),
+    ("c2", "fwd"): ("fwd_resident_kernel", "8d4545f335b45a20c621c65a3d69f3902bf7caa9afc91474c11ba02ae301b49b",
+                    15204864),
+}
 
 
-def ncu_traffic(workload: str, phase: str):
+def kernel_source_sha(name: str):
+    """sha256 of the text of kernel `name` in kernels.cuh: from its __global__ line to the next section rule."""
     import hashlib
     src = os.path.join(ROOT, "paper_2412_11810_b200", "csrc", "kernels.cuh")
     try:
-        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+        text = open(src).read()
     except OSError:
         return None
-    return NCU_TRAFFIC.get((workload, phase)) if sha == NCU_KERNELS_SHA256 else None
+    at = text.find(" " + name + "(const __grid_constant__")
+    if at < 0:
+        return None
+    start = text.rfind("__global__", 0, at)
+    end = text.find("\n// ----", at)
+    return hashlib.sha256(text[start:end if end > 0 else len(text)].encode()).hexdigest()
+
+
+def ncu_traffic(workload: str, phase: str):
+    entry = NCU_TRAFFIC.get((workload, phase))
+    if not entry:
+        return None
+    kernel, sha, nbytes = entry
+    return nbytes if sha and kernel_source_sha(kernel) == sha else None
 
 
 class ClockSampler:
