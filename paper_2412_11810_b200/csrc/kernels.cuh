@@ -1772,15 +1772,16 @@ __global__ void __launch_bounds__(32 * FFG_NWARP, 1) ff_gemm_kernel(const __grid
   constexpr int BPP = BP + 1, TILEP = BWD_TM * BPP;   // partial tiles padded: conflict-free column reads
   static_assert(ROWS * 32 % NT == 0, "the staged tile divides evenly among the threads");
   pdl_launch_dependents();
-  const int tile_row0 = blockIdx.x * BWD_TM;
+  const int tile_row0 = blockIdx.y * BWD_TM;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   extern __shared__ float4 s_dyn[];
   float* const s_tiles = reinterpret_cast<float*>(s_dyn);   // [BWD_STAGES][ROWS][BWD_LD]; later [NWARP][32][BP]
   const int M = p.n_steps * p.B, it_all = (p.K + 127) / 128;
   const int rlast = p.N - 1;
   pdl_wait();
-  {   // one pass of 64 (step, sample) pairs per CTA: blockIdx.y selects it
-    const int bp0 = blockIdx.y * BP;
+  {   // one pass of 64 (step, sample) pairs per CTA: blockIdx.x selects it, so that the CTAs that read the
+      // same rows of W run at the same time and all but the first find them in L2
+    const int bp0 = blockIdx.x * BP;
     const float* src[ITER];
     int dst_off[ITER], kcol[ITER];
 #pragma unroll

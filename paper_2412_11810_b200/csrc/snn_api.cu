@@ -737,7 +737,7 @@ struct Exec {
             gp.out = at<float>(lo.gff);
             end_span(span);
             span = begin_span(SNN_PHASE_FFGEMM);
-            CUDA_TRY(launch_pdl(ff_gemm_kernel, dim3((sz[l] + BWD_TM - 1) / BWD_TM, (gp.n_steps * B + 8 * FFG_NTN - 1) / (8 * FFG_NTN)),
+            CUDA_TRY(launch_pdl(ff_gemm_kernel, dim3((gp.n_steps * B + 8 * FFG_NTN - 1) / (8 * FFG_NTN), (sz[l] + BWD_TM - 1) / BWD_TM),
                                 dim3(32 * FFG_NWARP),
                                 bwd_smem_bytes(8 * FFG_NTN), gp));
             ++launches;
