@@ -256,6 +256,16 @@ typedef struct {
 snn_status snn_plan(int32_t T, const snn_ckpt* ckpt, snn_op* ops, int32_t max_ops, int32_t* n_ops,
                     int32_t* n_local_slots, int32_t* n_remote_slots);
 
+/* ---- self-test of the bounded waits ---------------------------------------------------------
+ * The cooperative kernels (forward and backward passes of small networks) wait for one another's results
+ * by polling counters in device memory; every such wait gives up after a fixed number of polls, raises a
+ * status bit and lets the kernel end, and the train step then returns SNN_ERR_DEVICE_TIMEOUT.  This call
+ * runs that wait alone: one thread block waits, for at most poll_limit polls, for a count that nobody
+ * publishes.  device_scratch: 256 bytes of device memory (overwritten).  Returns SNN_ERR_DEVICE_TIMEOUT
+ * when the wait gave up as it must, SNN_OK if it did not, SNN_ERR_CUDA on a CUDA error.  The context
+ * stays usable. */
+snn_status snn_selftest_wait_timeout(void* device_scratch, uint32_t poll_limit, void* stream);
+
 /* ---- spike compaction on its own ("Spike Generation": dense state -> sparse events) -----
  * For each of n_rows rows of n_words uint32 spike words (device), writes the ascending list
  * of set-bit indices to idx_out[row * capacity ..] (device) and its length to count_out[row]

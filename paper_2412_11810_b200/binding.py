@@ -32,7 +32,7 @@ STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "rem
 
 EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_train_step", "snn_peak_memory",
            "snn_memory_stats_get", "snn_last_error", "snn_plan", "snn_compact_spikes", "snn_get_event_layout",
-           "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt"]
+           "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt", "snn_selftest_wait_timeout"]
 SNN_STATIC_WORKSPACE_BYTES = 32 << 20
 
 
@@ -103,6 +103,7 @@ def _load() -> C.CDLL:
     lib.snn_suggest_ckpt.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_size_t, C.c_float,
                                      C.POINTER(snn_ckpt)]
     lib.snn_get_event_layout.argtypes = [C.c_void_p, C.c_int32, C.POINTER(snn_event_layout)]
+    lib.snn_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
     return lib
 
 
@@ -202,6 +203,11 @@ def snn_suggest_ckpt(net, T: int, B: int, strategy: int, device_budget_bytes: in
 def snn_compact_spikes(masks_ptr: int, n_rows: int, n_words: int, idx_out_ptr: int, capacity: int,
                        count_out_ptr: int, stream: int = 0) -> None:
     _check(lib.snn_compact_spikes(masks_ptr, n_rows, n_words, idx_out_ptr, capacity, count_out_ptr, stream))
+
+
+def snn_selftest_wait_timeout(device_scratch_ptr: int, poll_limit: int, stream: int = 0) -> int:
+    """Returns the status itself (SNN_ERR_DEVICE_TIMEOUT is the expected outcome)."""
+    return lib.snn_selftest_wait_timeout(device_scratch_ptr, poll_limit, stream)
 
 
 def snn_get_event_layout(net, layer: int) -> snn_event_layout:

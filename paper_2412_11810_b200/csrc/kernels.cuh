@@ -696,12 +696,27 @@ __device__ __forceinline__ void publish_progress(uint32_t* counter) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(counter), "r"(1u) : "memory");
 }
 
-__device__ __forceinline__ bool wait_progress(const uint32_t* counter, uint32_t target) {
-  for (uint32_t i = 0; i < SYNC_POLL_LIMIT; ++i) {
+__device__ __forceinline__ bool wait_progress(const uint32_t* counter, uint32_t target,
+                                              uint32_t poll_limit = SYNC_POLL_LIMIT) {
+  for (uint32_t i = 0; i < poll_limit; ++i) {
     if (ld_acquire_gpu(counter) >= target) return true;
     if (i > 32) __nanosleep(64);
   }
   return false;
+}
+
+// The waiting protocol on its own, for a self-test: one CTA waits for a count that nobody publishes; the
+// wait must give up after poll_limit polls, raise the status bit and let the kernel end.
+__global__ void wait_selftest_kernel(uint32_t* status, const uint32_t* counter, uint32_t poll_limit) {
+  __shared__ int s_ok;
+  if (threadIdx.x == 0) {
+    const bool ok = wait_progress(counter, 1u, poll_limit);
+    if (!ok) atomicOr(status, STATUS_SYNC_TIMEOUT);
+    s_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  status[1] = 1u;   // not reached unless somebody published
 }
 
 __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_constant__ FwdSegParams p) {

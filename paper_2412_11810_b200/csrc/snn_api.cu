@@ -1051,6 +1051,20 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   return SNN_OK;
 }
 
+// Self-test of the bounded waits between thread blocks (see snn.h).
+extern "C" snn_status snn_selftest_wait_timeout(void* device_scratch, uint32_t poll_limit, void* stream) {
+  if (!device_scratch || poll_limit == 0) return SNN_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t* words = reinterpret_cast<uint32_t*>(device_scratch);
+  if (cudaMemsetAsync(words, 0, 256, st) != cudaSuccess) return SNN_ERR_CUDA;
+  wait_selftest_kernel<<<1, 64, 0, st>>>(words, words + 32, poll_limit);
+  uint32_t host[2] = {0, 0};
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess ||
+      cudaMemcpy(host, words, 8, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return SNN_ERR_CUDA;
+  return (host[0] & STATUS_SYNC_TIMEOUT) && host[1] == 0 ? SNN_ERR_DEVICE_TIMEOUT : SNN_OK;
+}
+
 // ------------------------------------------------------------------------------------------
 // Training step on the library's own, statically reserved device workspace, for callers that
 // have no way to allocate device memory when the step is due (no PyTorch in the process, the

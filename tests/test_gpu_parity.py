@@ -502,3 +502,19 @@ def test_backward_as_one_launch_per_segment(orc32):
             for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
                 assert np.array_equal(x, y), (w.sizes, w.B, strat, K, R)
         s.close()
+
+
+def test_a_wait_that_cannot_end_gives_up():
+    """The waits between thread blocks are bounded: one that nothing satisfies raises the time-out status
+    after its poll limit and the kernel ends; the context stays usable for a normal step afterwards."""
+    import torch
+    b = sb()
+    scratch = torch.zeros(256, dtype=torch.uint8, device="cuda:0")
+    for polls in (1, 1000, 200000):
+        assert b.snn_selftest_wait_timeout(scratch.data_ptr(), polls) == b.SNN_ERR_DEVICE_TIMEOUT
+    assert b.snn_selftest_wait_timeout(0, 10) == b.SNN_ERR_INVALID_ARG
+    w = wl.small()
+    d = wl.make(w)
+    s, bits, targets = make_session(w, d)
+    assert np.isfinite(s.train_step(bits, targets, strategy=1, chunk_size=4, max_activity=1.0))
+    s.close()
