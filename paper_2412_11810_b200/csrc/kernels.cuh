@@ -870,14 +870,15 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
 // A CTA owns RS_COLS columns of one layer and keeps those columns of W_ff and W_rec (every row) in
 // shared memory for all steps of the launch, so an event costs a shared-memory read instead of an
 // L2 gather.  Per step a half-warp turns the spike words of one sample into the list of weight rows
-// in canonical order (feed-forward events, then recurrent ones, ascending); then the first four
-// warps add the rows, one thread per sample and four columns, apply leak, reset and threshold, and
+// in canonical order (feed-forward events, then recurrent ones, ascending); then the first eight
+// warps add the rows, one thread per sample and two columns, apply leak, reset and threshold, and
 // publish 16 spike bits per sample.  The event pools of a sample are appended to by one CTA of the
 // layer (sample index modulo the number of CTAs).  Every CTA of a layer needs the words of all
 // columns, so the layers synchronise through one counter each (finished (CTA, step) pairs), with
 // the publish / poll protocol of fwd_segment_kernel.  Cooperative launch; bounded waits.
 constexpr int RS_COLS = 16;        // columns of a layer per CTA
-constexpr int RS_THREADS = 512;    // 32 samples x RS_COLS columns
+constexpr int RS_THREADS = 512;    // 32 half-warps: one per sample of a group
+constexpr int RS_ADDERS = 256;     // threads that add rows: 32 samples x 8 column pairs
 constexpr int RS_LIST = 256;       // list entries per sample staged at a time
 constexpr int RS_MAX_GROUPS = 2;   // groups of 32 samples a thread can own: B <= 64
 
@@ -937,13 +938,13 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
   __shared__ uint32_t s_ends[32][3];   // per sample: end of its recurrent and feed-forward pool lists, feed-forward events now
 
   // Two roles.  Compaction: half-warp `bl` (16 lanes, lane index c) turns the words of sample 32 gi + bl into
-  // its list.  Accumulation: the first 128 threads; thread (sb, quad) owns columns 4 quad .. 4 quad + 3 of
-  // sample 32 gi + sb.
+  // its list.  Accumulation: the first 256 threads; thread (sb, pair) owns columns 2 pair, 2 pair + 1 of
+  // sample 32 gi + sb (eight warps: two per scheduler hide the shared-memory latency of one another).
   const int c = tid & (RS_COLS - 1), bl = tid >> 4;
-  const bool adder = tid < 128;
-  const int sb = tid >> 2, quad = tid & 3;
-  const int acol = col0 + quad * 4;            // first of this thread's four columns (accumulation role)
-  const bool acol_ok = adder && acol < L.N;    // N is a multiple of 4: all four or none
+  const bool adder = tid < RS_ADDERS;
+  const int sb = tid >> 3, pair = tid & 7;
+  const int acol = col0 + pair * 2;            // first of this thread's two columns (accumulation role)
+  const bool acol_ok = adder && acol < L.N;    // N is even: both or none
 
   // ---- this CTA's columns of both matrices, every row, once per launch
   for (int q = tid; q < rows * (RS_COLS / 4); q += RS_THREADS) {
@@ -954,16 +955,16 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
   }
   cp_async_commit();
 
-  float4 v[RS_MAX_GROUPS];
+  float2 v[RS_MAX_GROUPS];
   uint32_t rec_end[RS_MAX_GROUPS], ff_end[RS_MAX_GROUPS];
   bool owner[RS_MAX_GROUPS];   // this CTA appends the lists of the half-warp's sample to the event pools
 #pragma unroll
   for (int gi = 0; gi < RS_MAX_GROUPS; ++gi) {
-    v[gi] = make_float4(0.f, 0.f, 0.f, 0.f); rec_end[gi] = 0; ff_end[gi] = 0; owner[gi] = false;
+    v[gi] = make_float2(0.f, 0.f); rec_end[gi] = 0; ff_end[gi] = 0; owner[gi] = false;
     if (gi < groups) {
       const int ba = gi * 32 + sb, bc = gi * 32 + bl;
       if (acol_ok && ba < B)
-        v[gi] = *reinterpret_cast<const float4*>(p.slots + (size_t)p.in_slot * p.slot_stride + L.state_off +
+        v[gi] = *reinterpret_cast<const float2*>(p.slots + (size_t)p.in_slot * p.slot_stride + L.state_off +
                                                  (size_t)ba * L.N + acol);
       owner[gi] = bc < B && bc % L.tiles == tile;
       if (owner[gi]) {
@@ -1035,22 +1036,30 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
       const bool pools = owner[gi];
       const uint32_t room_rec = L.rec_cap - rec_end[gi], room_ff = L.write_ff_list ? L.ff_cap - ff_end[gi] : 0u;
 
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float2 acc = make_float2(0.f, 0.f);
       for (uint32_t c0 = 0;; c0 += RS_LIST) {
         // this lane's events that fall into [c0, c0 + RS_LIST): row of Ws into the list, index into the pools
         uint32_t pos = first;
-        for (int w = w_lo; w < w_hi && pos < c0 + RS_LIST; ++w) {
-          uint32_t bits = b_ok ? wrow[w] : 0u;
-          const bool ff = w < L.W_pre;
-          const uint32_t idx0 = (uint32_t)(ff ? w : w - L.W_pre) * 32u;
-          if (pos + __popc(bits) <= c0) { pos += __popc(bits); continue; }
-          while (bits) {
-            const uint32_t idx = idx0 + (uint32_t)(__ffs(bits) - 1);
-            bits &= bits - 1;
-            if (pos >= c0 && pos < c0 + RS_LIST) {
-              lst[pos - c0] = (uint16_t)(ff ? idx : idx + (uint32_t)L.N_pre);
+        if (n_tot <= (uint32_t)RS_LIST) {   // the usual case: the whole list fits, no window to test against
+          for (int w = w_lo; w < w_hi; ++w) {
+            uint32_t bits = b_ok ? wrow[w] : 0u;
+            const uint32_t idx0 = w < L.W_pre ? (uint32_t)w * 32u : (uint32_t)(w - L.W_pre) * 32u + (uint32_t)L.N_pre;
+            while (bits) {
+              lst[pos++] = (uint16_t)(idx0 + (uint32_t)(__ffs(bits) - 1));
+              bits &= bits - 1;
             }
-            ++pos;
+          }
+        } else {
+          for (int w = w_lo; w < w_hi && pos < c0 + RS_LIST; ++w) {
+            uint32_t bits = b_ok ? wrow[w] : 0u;
+            const uint32_t idx0 = w < L.W_pre ? (uint32_t)w * 32u : (uint32_t)(w - L.W_pre) * 32u + (uint32_t)L.N_pre;
+            if (pos + __popc(bits) <= c0) { pos += __popc(bits); continue; }
+            while (bits) {
+              const uint32_t idx = idx0 + (uint32_t)(__ffs(bits) - 1);
+              bits &= bits - 1;
+              if (pos >= c0 && pos < c0 + RS_LIST) lst[pos - c0] = (uint16_t)idx;
+              ++pos;
+            }
           }
         }
         if (c == 0) {
@@ -1062,25 +1071,22 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
         if (adder) {
           const int n = s_n[sb];
           const uint16_t* const al = s_list + (size_t)sb * RS_LIST;
-          const float4* const Wq = reinterpret_cast<const float4*>(Ws) + quad;
-          auto add4 = [&](const float4 r) {
-            acc.x = __fadd_rn(acc.x, r.x); acc.y = __fadd_rn(acc.y, r.y);
-            acc.z = __fadd_rn(acc.z, r.z); acc.w = __fadd_rn(acc.w, r.w);
-          };
+          const float2* const Wp = reinterpret_cast<const float2*>(Ws) + pair;
+          auto add2 = [&](const float2 r) { acc.x = __fadd_rn(acc.x, r.x); acc.y = __fadd_rn(acc.y, r.y); };
           // eight rows at a time, the next eight already on their way while these are added
-          auto load8 = [&](int e, float4 (&w)[8]) {
+          auto load8 = [&](int e, float2 (&w)[8]) {
             const uint4 pk = *reinterpret_cast<const uint4*>(al + e);
-            w[0] = Wq[(pk.x & 0xffffu) * (RS_COLS / 4)]; w[1] = Wq[(pk.x >> 16) * (RS_COLS / 4)];
-            w[2] = Wq[(pk.y & 0xffffu) * (RS_COLS / 4)]; w[3] = Wq[(pk.y >> 16) * (RS_COLS / 4)];
-            w[4] = Wq[(pk.z & 0xffffu) * (RS_COLS / 4)]; w[5] = Wq[(pk.z >> 16) * (RS_COLS / 4)];
-            w[6] = Wq[(pk.w & 0xffffu) * (RS_COLS / 4)]; w[7] = Wq[(pk.w >> 16) * (RS_COLS / 4)];
+            w[0] = Wp[(pk.x & 0xffffu) * (RS_COLS / 2)]; w[1] = Wp[(pk.x >> 16) * (RS_COLS / 2)];
+            w[2] = Wp[(pk.y & 0xffffu) * (RS_COLS / 2)]; w[3] = Wp[(pk.y >> 16) * (RS_COLS / 2)];
+            w[4] = Wp[(pk.z & 0xffffu) * (RS_COLS / 2)]; w[5] = Wp[(pk.z >> 16) * (RS_COLS / 2)];
+            w[6] = Wp[(pk.w & 0xffffu) * (RS_COLS / 2)]; w[7] = Wp[(pk.w >> 16) * (RS_COLS / 2)];
           };
-          auto add8 = [&](const float4 (&w)[8]) {
+          auto add8 = [&](const float2 (&w)[8]) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) add4(w[j]);
+            for (int j = 0; j < 8; ++j) add2(w[j]);
           };
           const int n8 = n & ~7;
-          float4 wa[8], wb[8];
+          float2 wa[8], wb[8];
           int e = 0;
           if (n8 > 0) load8(0, wa);
           while (e < n8) {
@@ -1093,11 +1099,11 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
             e += 8;
           }
           for (; e < n; ++e) {
-            add4(Wq[(uint32_t)al[e] * (RS_COLS / 4)]);
+            add2(Wp[(uint32_t)al[e] * (RS_COLS / 2)]);
           }
         } else {
           // ---- meanwhile the other warps append the lists of the samples this CTA owns to the event pools
-          const int h = (tid - 128) >> 4, n_helpers = (RS_THREADS - 128) >> 4;
+          const int h = (tid - RS_ADDERS) >> 4, n_helpers = (RS_THREADS - RS_ADDERS) >> 4;
           int bb = tile;
           while (bb < 32 * gi) bb += L.tiles;
           for (int k = 0; bb < B && bb < 32 * gi + 32; bb += L.tiles, ++k) {
@@ -1120,34 +1126,32 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
 
       // ---- leak, reset by subtraction of the previous step's own spike, threshold (accumulation role)
       const int ba = gi * 32 + sb;
-      uint32_t nib = 0;
+      uint32_t two = 0;
       if (acol_ok && ba < B) {
         const uint32_t pw = s_words[(size_t)ba * Wtot + L.W_pre + (acol >> 5)] >> (acol & 31);
-        float4 vn;
+        float2 vn;
         vn.x = __fsub_rn(__fmaf_rn(p.alpha, v[gi].x, acc.x), __fmul_rn(p.theta, (float)(pw & 1u)));
         vn.y = __fsub_rn(__fmaf_rn(p.alpha, v[gi].y, acc.y), __fmul_rn(p.theta, (float)((pw >> 1) & 1u)));
-        vn.z = __fsub_rn(__fmaf_rn(p.alpha, v[gi].z, acc.z), __fmul_rn(p.theta, (float)((pw >> 2) & 1u)));
-        vn.w = __fsub_rn(__fmaf_rn(p.alpha, v[gi].w, acc.w), __fmul_rn(p.theta, (float)((pw >> 3) & 1u)));
         v[gi] = vn;
         float* const st = p.slots + L.state_off + (size_t)ba * L.N + acol;
-        *reinterpret_cast<float4*>(st + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = vn;
+        *reinterpret_cast<float2*>(st + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride) = vn;
         if (p.keep_every > 0 && d % p.keep_every == 0)
-          *reinterpret_cast<float4*>(st + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = vn;
-        if (L.V_dbg) *reinterpret_cast<float4*>(L.V_dbg + ((size_t)t * B + ba) * L.N + acol) = vn;
-        nib = (vn.x > p.theta ? 1u : 0u) | (vn.y > p.theta ? 2u : 0u) | (vn.z > p.theta ? 4u : 0u) |
-              (vn.w > p.theta ? 8u : 0u);
-        if (L.counts && nib) {
-          uint4* cp = reinterpret_cast<uint4*>(L.counts + (size_t)ba * L.N + acol);
-          uint4 cv = *cp;
-          cv.x += nib & 1u; cv.y += (nib >> 1) & 1u; cv.z += (nib >> 2) & 1u; cv.w += (nib >> 3) & 1u;
+          *reinterpret_cast<float2*>(st + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = vn;
+        if (L.V_dbg) *reinterpret_cast<float2*>(L.V_dbg + ((size_t)t * B + ba) * L.N + acol) = vn;
+        two = (vn.x > p.theta ? 1u : 0u) | (vn.y > p.theta ? 2u : 0u);
+        if (L.counts && two) {
+          uint2* cp = reinterpret_cast<uint2*>(L.counts + (size_t)ba * L.N + acol);
+          uint2 cv = *cp;
+          cv.x += two & 1u; cv.y += (two >> 1) & 1u;
           *cp = cv;
         }
       }
-      if (adder) {   // whole warps: four neighbouring lanes hold the 16 spike bits of one sample
-        uint32_t half = nib << (4 * quad);
+      if (adder) {   // whole warps: eight neighbouring lanes hold the 16 spike bits of one sample
+        uint32_t half = two << (2 * pair);
         half |= __shfl_xor_sync(0xffffffffu, half, 1);
         half |= __shfl_xor_sync(0xffffffffu, half, 2);
-        if (quad == 0 && ba < B) {
+        half |= __shfl_xor_sync(0xffffffffu, half, 4);
+        if (pair == 0 && ba < B) {
           uint16_t* const hrow = reinterpret_cast<uint16_t*>(L.words + ((size_t)t * B + ba) * L.W);
           hrow[tile] = (uint16_t)half;
           if (tile == L.tiles - 1 && (L.tiles & 1)) hrow[tile + 1] = 0;   // the unused half of the last word
