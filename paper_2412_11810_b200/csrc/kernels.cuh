@@ -956,11 +956,12 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
   cp_async_commit();
 
   float2 v[RS_MAX_GROUPS];
+  uint2 fired[RS_MAX_GROUPS];   // spikes of this thread's two neurons during this launch (last layer: for the readout)
   uint32_t rec_end[RS_MAX_GROUPS], ff_end[RS_MAX_GROUPS];
   bool owner[RS_MAX_GROUPS];   // this CTA appends the lists of the half-warp's sample to the event pools
 #pragma unroll
   for (int gi = 0; gi < RS_MAX_GROUPS; ++gi) {
-    v[gi] = make_float2(0.f, 0.f); rec_end[gi] = 0; ff_end[gi] = 0; owner[gi] = false;
+    v[gi] = make_float2(0.f, 0.f); fired[gi] = make_uint2(0u, 0u); rec_end[gi] = 0; ff_end[gi] = 0; owner[gi] = false;
     if (gi < groups) {
       const int ba = gi * 32 + sb, bc = gi * 32 + bl;
       if (acol_ok && ba < B)
@@ -1139,12 +1140,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
           *reinterpret_cast<float2*>(st + (size_t)(p.keep_slot + d / p.keep_every - 1) * p.slot_stride) = vn;
         if (L.V_dbg) *reinterpret_cast<float2*>(L.V_dbg + ((size_t)t * B + ba) * L.N + acol) = vn;
         two = (vn.x > p.theta ? 1u : 0u) | (vn.y > p.theta ? 2u : 0u);
-        if (L.counts && two) {
-          uint2* cp = reinterpret_cast<uint2*>(L.counts + (size_t)ba * L.N + acol);
-          uint2 cv = *cp;
-          cv.x += two & 1u; cv.y += (two >> 1) & 1u;
-          *cp = cv;
-        }
+        fired[gi].x += two & 1u; fired[gi].y += (two >> 1) & 1u;
       }
       if (adder) {   // whole warps: eight neighbouring lanes hold the 16 spike bits of one sample
         uint32_t half = two << (2 * pair);
@@ -1177,6 +1173,19 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
     __syncthreads();
     if (tid == 0) {   // publish: this CTA's spike bits of step t are complete
       publish_progress(my_progress);
+    }
+  }
+  // spike counts of the launch into the time-summed counts the readout uses (this thread is their only writer)
+  if (L.counts && acol_ok) {
+#pragma unroll
+    for (int gi = 0; gi < RS_MAX_GROUPS; ++gi) {
+      const int ba = gi * 32 + sb;
+      if (gi < groups && ba < B) {
+        uint2* cp = reinterpret_cast<uint2*>(L.counts + (size_t)ba * L.N + acol);
+        uint2 cv = *cp;
+        cv.x += fired[gi].x; cv.y += fired[gi].y;
+        *cp = cv;
+      }
     }
   }
 }
