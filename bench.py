@@ -49,8 +49,8 @@ NCU_TRAFFIC = {
                     269443328 + 4209920),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
                     388252416 + 4982784),
-    ("c2", "fwd"): ("fwd_resident_kernel", "8d4545f335b45a20c621c65a3d69f3902bf7caa9afc91474c11ba02ae301b49b",
-                    15204864),
+    ("c2", "fwd"): ("fwd_resident_kernel", "0d6da12b003e9d7942f18dfc1f0a724c029951a870a748a04acca7060137967b",
+                    15203584),
 }
 
 
