@@ -1405,12 +1405,12 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
       // warp's first k-step: copy instructions and mma instructions queue on different pipes, and in program
       // order one after the other they would take turns instead of overlapping.
       const int it_refill = it + BWD_STAGES - 1;
-      bool refill = true;
       const float* Ws = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
       const float* Ds = Ws + BWD_TM * BWD_LD;
-#pragma unroll 1
-      for (int ks = warp; ks < 16; ks += NWARP) {
-        const int kk = ks * 8 + t;
+#pragma unroll
+      for (int ksl = 0; ksl < 16 / NWARP; ++ksl) {   // this warp's k-steps of the chunk: warp, warp + NWARP, ...
+        const bool refill = ksl == 0;
+        const int kk = (warp + ksl * NWARP) * 8 + t;
         uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
@@ -1444,7 +1444,6 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
         if (refill) {
           issue_part(it_refill, 2 * ITER / 3, ITER);
           cp_async_commit();
-          refill = false;
         }
       }
     }
