@@ -45,8 +45,8 @@ def read_peaks():
 # the kernel still has that text.  The backward pass of c2 now runs in bwd_segment_kernel, a cooperative launch
 # of thread-block clusters that the profiler cannot launch: no counters, hence no entry.
 NCU_TRAFFIC = {
-    ("c4", "bwd"): ("bwd_step_kernel", "41ed2477e69ea0abdff4478e5d8fcc71fbe2997db65a8bf332fd66406d046db3",
-                    269443328 + 4209920),
+    ("c4", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
+                    269405952 + 3885312),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
                     388252416 + 4982784),
     ("c2", "fwd"): ("fwd_resident_kernel", "0d6da12b003e9d7942f18dfc1f0a724c029951a870a748a04acca7060137967b",
