@@ -459,7 +459,9 @@ struct Exec {
     return ctas <= net->coop_sms;   // one CTA per SM (more than half of its shared memory each)
   }
 
-  snn_status run_forward_resident(const snn_op& op) {
+  // `done` stays false when the device refuses the cooperative launch: the caller then takes the next path.
+  snn_status run_forward_resident(const snn_op& op, bool& done) {
+    done = false;
     ResParams p;
     std::memset(&p, 0, sizeof p);
     p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
@@ -498,12 +500,17 @@ struct Exec {
     at1[0].id = cudaLaunchAttributeCooperative;
     at1[0].val.cooperative = 1;
     cfg.attrs = at1; cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, fwd_resident_kernel, p));
+    if (cudaLaunchKernelEx(&cfg, fwd_resident_kernel, p) != cudaSuccess) {
+      cudaGetLastError();
+      return SNN_OK;
+    }
     ++launches;
+    done = true;
     return SNN_OK;
   }
 
-  snn_status run_forward_segment(const snn_op& op) {
+  snn_status run_forward_segment(const snn_op& op, bool& done) {
+    done = false;
     FwdSegParams p;
     std::memset(&p, 0, sizeof p);
     p.slots = at<float>(lo.slots); p.slot_stride = lo.state_bytes / 4;
@@ -534,8 +541,12 @@ struct Exec {
     at1[0].id = cudaLaunchAttributeCooperative;
     at1[0].val.cooperative = 1;
     cfg.attrs = at1; cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, fwd_segment_kernel, p));
+    if (cudaLaunchKernelEx(&cfg, fwd_segment_kernel, p) != cudaSuccess) {
+      cudaGetLastError();
+      return SNN_OK;
+    }
     ++launches;
+    done = true;
     return SNN_OK;
   }
 
@@ -551,14 +562,14 @@ struct Exec {
       return st;
     }
     if (gen && forward_resident_possible()) {
-      const snn_status st = run_forward_resident(op);
-      end_span(span);
-      return st;
+      bool done = false;
+      const snn_status st = run_forward_resident(op, done);
+      if (st != SNN_OK || done) { end_span(span); return st; }
     }
     if (gen && forward_segment_possible()) {
-      const snn_status st = run_forward_segment(op);
-      end_span(span);
-      return st;
+      bool done = false;
+      const snn_status st = run_forward_segment(op, done);
+      if (st != SNN_OK || done) { end_span(span); return st; }
     }
     FwdParams p;
     std::memset(&p, 0, sizeof p);
