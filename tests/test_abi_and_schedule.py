@@ -26,6 +26,19 @@ def test_library_exports_every_declared_symbol():
         assert getattr(sb.lib, name) is not None
 
 
+def test_binding_constants_match_the_header():
+    """Flags and enumerators are spelled twice (include/snn.h and binding.py): same names, same values."""
+    header = open(os.path.join(ROOT, "include", "snn.h")).read()
+    flags = dict(re.findall(r"#define\s+(SNN_FLAG_[A-Z_]+)\s+(\d+)u", header))
+    assert len(flags) >= 9
+    for name, value in flags.items():
+        assert getattr(sb, name) == int(value), name
+    for name, value in re.findall(r"\b(SNN_(?:ERR_[A-Z_]+|OK|STANDARD|CHUNK|REMOTE|DOUBLE|HIERARCHICAL|DOUBLE_LOCAL|CELL_[A-Z]+))\s*=\s*(\d+)", header):
+        assert getattr(sb, name) == int(value), name
+    m = re.search(r"#define\s+SNN_STATIC_WORKSPACE_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", header)
+    assert m and sb.SNN_STATIC_WORKSPACE_BYTES == int(m.group(1)) << int(m.group(2))
+
+
 def test_create_validates():
     net = sb.snn_create([8, 16, 4], 20.0, 1.0)
     assert abs(sb.snn_alpha(net) - float(leak_from_tau(20.0))) == 0.0
