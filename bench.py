@@ -47,6 +47,8 @@ def read_peaks():
 NCU_TRAFFIC = {
     ("c4", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
                     269405952 + 3885312),
+    ("c3", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
+                    51018240 + 43264),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
                     388252416 + 4982784),
     ("c2", "fwd"): ("fwd_resident_kernel", "0d6da12b003e9d7942f18dfc1f0a724c029951a870a748a04acca7060137967b",
