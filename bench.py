@@ -80,6 +80,15 @@ def ncu_traffic(workload: str, phase: str):
     return nbytes if sha and kernel_source_sha(kernel) == sha else None
 
 
+def read_tensor_peak():
+    """Dense tf32 peak in TFLOP/s: the measured bf16 figure times the nominal tf32 : bf16 ratio."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["bf16_tflops"]) * 1.1 / 2.25, "measured bf16 x 1.1/2.25"
+    return 1590.0 * 1.1 / 2.25, "fallback bf16 x 1.1/2.25"
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -311,6 +320,20 @@ def run_ours(args, rank, world):
                     "achieved": ach, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": ach / peak,
                     "traffic": ncu_traffic(w.name, dominant), "algorithmic_bytes_per_launch": per_launch_bytes,
                     "avg_launch_us": avg_s * 1e6, "launches_per_step": ph[dominant][1]}
+            if dominant == "bwd":
+                # the backward step is the one dense contraction of the path (delta x W^T, fp32 result through three
+                # TF32 passes): its rate against the tensor peak for tf32 (measured bf16 peak x nominal 1.1 / 2.25)
+                sz = w.sizes
+                if ph["ffgemm"][1] > 0:     # one layer per launch, recurrent matrix only
+                    flops = 2.0 * w.B * sum(n * n for n in sz[1:-1]) / w.L
+                else:
+                    flops = 2.0 * w.B * sum(sz[l] * sz[l] + (sz[l] * sz[l + 1] if l < w.L else 0)
+                                            for l in range(1, w.L + 1))
+                tpeak, tkind = read_tensor_peak()
+                roof["tensor"] = {"achieved": flops / avg_s / 1e12, "peak": tpeak, "peak_kind": tkind,
+                                  "unit": "TFLOP/s", "frac": flops / avg_s / 1e12 / tpeak,
+                                  "flops_per_launch": flops,
+                                  "note": "fp32-equivalent flops; the kernel issues three tf32 mma.sync passes per product"}
         # the other strategies on the same workload (fewer steps), for the per-strategy table
         per_strategy = {}
         T = w.T
