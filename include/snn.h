@@ -50,7 +50,10 @@ typedef enum {
 typedef enum { SNN_STANDARD = 0, SNN_CHUNK = 1, SNN_REMOTE = 2, SNN_DOUBLE = 3, SNN_HIERARCHICAL = 4,
                SNN_DOUBLE_LOCAL = 5 } snn_strategy;
 typedef enum { SNN_CELL_LIF = 0, SNN_CELL_GRADED = 1 } snn_cell;
-typedef enum { SNN_SURR_FAST_SIGMOID = 0, SNN_SURR_SIGMOID = 1 } snn_surrogate;
+/* Pseudo-derivative of the spike, x = V - threshold.  The paper names none; 0 is the default of the
+ * benchmark definition.  0: 1 / (1 + beta |x|)^2.  1: beta s (1 - s), s = sigmoid(beta x).
+ * 2 (an extension): beta max(0, 1 - beta |x|), zero outside |x| < 1 / beta. */
+typedef enum { SNN_SURR_FAST_SIGMOID = 0, SNN_SURR_SIGMOID = 1, SNN_SURR_TRIANGLE = 2 } snn_surrogate;
 
 #define SNN_MAX_LAYERS 8      /* hidden layers                                   */
 #define SNN_MAX_NEURONS 65536 /* per layer; hidden sizes must be multiples of 4  */

@@ -15,7 +15,7 @@ import numpy as np
 from . import build_oracle
 
 CELL_LIF, CELL_GRADED = 0, 1
-SURR_FAST_SIGMOID, SURR_SIGMOID = 0, 1
+SURR_FAST_SIGMOID, SURR_SIGMOID, SURR_TRIANGLE = 0, 1, 2
 
 
 class _Params(C.Structure):

@@ -67,11 +67,12 @@ typedef REAL real;
 #define CELL_GRADED 1
 #define SURR_FAST_SIGMOID 0
 #define SURR_SIGMOID 1
+#define SURR_TRIANGLE 2   /* compact support; not in the paper (see surrogate_grad) */
 
 typedef struct {
   int32_t L;        /* number of hidden (recurrent) layers                 */
   int32_t cell;     /* CELL_LIF | CELL_GRADED                               */
-  int32_t surrogate;/* SURR_FAST_SIGMOID | SURR_SIGMOID                     */
+  int32_t surrogate;/* SURR_FAST_SIGMOID | SURR_SIGMOID | SURR_TRIANGLE     */
   int32_t smooth;   /* 1: S = sigmoid(beta (V - theta)) in the forward too  */
   double alpha;     /* leak per step; cast to REAL before use               */
   double theta;     /* threshold                                            */
@@ -96,6 +97,13 @@ static inline double surrogate_grad(const oracle_params* p, double x) {
   if (p->smooth || p->surrogate == SURR_SIGMOID) {
     double s = sigmoid_d(p->beta * x);
     return p->beta * s * (1.0 - s);
+  }
+  if (p->surrogate == SURR_TRIANGLE) {
+    /* An extension beyond the paper, which names no surrogate: the triangular pseudo-derivative
+     * beta * max(0, 1 - beta |x|), zero outside |x| < 1/beta, unit area.  With it only neurons near
+     * the threshold carry gradient, which is what an event-driven backward pass would exploit. */
+    double u = 1.0 - p->beta * fabs(x);
+    return u > 0.0 ? p->beta * u : 0.0;
   }
   double d = 1.0 + p->beta * fabs(x);
   return 1.0 / (d * d);

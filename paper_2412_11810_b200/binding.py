@@ -17,7 +17,7 @@ SNN_OK, SNN_ERR_INVALID_ARG, SNN_ERR_WORKSPACE_TOO_SMALL, SNN_ERR_EVENT_OVERFLOW
 SNN_ERR_DEVICE_TIMEOUT, SNN_ERR_CUDA, SNN_ERR_UNSUPPORTED = 4, 5, 6
 SNN_STANDARD, SNN_CHUNK, SNN_REMOTE, SNN_DOUBLE, SNN_HIERARCHICAL, SNN_DOUBLE_LOCAL = 0, 1, 2, 3, 4, 5
 SNN_CELL_LIF, SNN_CELL_GRADED = 0, 1
-SNN_SURR_FAST_SIGMOID, SNN_SURR_SIGMOID = 0, 1
+SNN_SURR_FAST_SIGMOID, SNN_SURR_SIGMOID, SNN_SURR_TRIANGLE = 0, 1, 2
 SNN_INPUT_BITS, SNN_INPUT_DENSE = 0, 1
 SNN_FLAG_INPUT_ON_HOST, SNN_FLAG_FORWARD_ONLY, SNN_FLAG_TIME_PHASES = 1, 2, 4
 SNN_FLAG_BACKWARD_LAYER_BY_LAYER, SNN_FLAG_BACKWARD_WAVEFRONT = 8, 16

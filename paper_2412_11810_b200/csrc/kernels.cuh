@@ -1231,6 +1231,10 @@ __device__ __forceinline__ float surrogate_grad(float v, float theta, float beta
     const float d = fmaf(beta, fabsf(x), 1.f);
     return 1.f / (d * d);
   }
+  if (surrogate == 2) {   // triangle with support |x| < 1 / beta
+    const float u = fmaf(-beta, fabsf(x), 1.f);
+    return u > 0.f ? beta * u : 0.f;
+  }
   const float s = 1.f / (1.f + expf(-beta * x));
   return beta * s * (1.f - s);
 }

@@ -146,7 +146,9 @@ extern "C" snn_status snn_create(const snn_config* cfg, snn_net** out) {
     if (cfg->sizes[l] % 4 != 0 || cfg->sizes[l] > SNN_MAX_NEURONS) return SNN_ERR_UNSUPPORTED;
   if (cfg->sizes[0] > SNN_MAX_NEURONS) return SNN_ERR_UNSUPPORTED;
   if (!(cfg->tau_mem > 0) || !(cfg->surrogate_beta > 0)) return SNN_ERR_INVALID_ARG;
-  if (cfg->surrogate != SNN_SURR_FAST_SIGMOID && cfg->surrogate != SNN_SURR_SIGMOID) return SNN_ERR_INVALID_ARG;
+  if (cfg->surrogate != SNN_SURR_FAST_SIGMOID && cfg->surrogate != SNN_SURR_SIGMOID &&
+      cfg->surrogate != SNN_SURR_TRIANGLE)
+    return SNN_ERR_INVALID_ARG;
   if (cfg->cell != SNN_CELL_LIF && cfg->cell != SNN_CELL_GRADED) return SNN_ERR_INVALID_ARG;
   snn_net* n = new snn_net();
   n->sizes.assign(cfg->sizes, cfg->sizes + cfg->n_sizes);

@@ -33,7 +33,7 @@ def test_binding_constants_match_the_header():
     assert len(flags) >= 9
     for name, value in flags.items():
         assert getattr(sb, name) == int(value), name
-    for name, value in re.findall(r"\b(SNN_(?:ERR_[A-Z_]+|OK|STANDARD|CHUNK|REMOTE|DOUBLE|HIERARCHICAL|DOUBLE_LOCAL|CELL_[A-Z]+))\s*=\s*(\d+)", header):
+    for name, value in re.findall(r"\b(SNN_(?:ERR_[A-Z_]+|OK|STANDARD|CHUNK|REMOTE|DOUBLE|HIERARCHICAL|DOUBLE_LOCAL|CELL_[A-Z]+|SURR_[A-Z_]+))\s*=\s*(\d+)", header):
         assert getattr(sb, name) == int(value), name
     m = re.search(r"#define\s+SNN_STATIC_WORKSPACE_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", header)
     assert m and sb.SNN_STATIC_WORKSPACE_BYTES == int(m.group(1)) << int(m.group(2))

@@ -212,6 +212,31 @@ def test_sigmoid_surrogate(orc32):
     s.close()
 
 
+def test_triangle_surrogate(orc32):
+    """The compact-support pseudo-derivative: most neurons get exactly zero, the rest must agree with the oracle,
+    on both backward paths and bit-identically across strategies."""
+    from oracle.oracle import SURR_TRIANGLE, NetSpec, leak_from_tau
+    from paper_2412_11810_b200 import Session
+    b = sb()
+    w = wl.small(sizes=(70, 700, 260, 7), T=41, B=5, p_in=0.05, g_ff=(2.5, 1.4), g_rec=(1.0, 1.0), seed=71)
+    d = wl.make(w)
+    spec = NetSpec(w.sizes, leak_from_tau(w.tau_mem), w.theta, 3.0, w.scale(), surrogate=SURR_TRIANGLE)
+    ref = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
+    assert all(np.abs(g).max() > 0 for g in ref["dW_rec"])
+    s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate=b.SNN_SURR_TRIANGLE, surrogate_beta=3.0,
+                readout_scale=w.scale())
+    s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    s.train_step(d["input_bits"], d["targets"], strategy=0, max_activity=1.0)
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R, flags in [(1, 6, 0, 0), (3, 4, 16, 0), (1, 6, 0, b.SNN_FLAG_BACKWARD_PER_STEP)]:
+        s.train_step(d["input_bits"], d["targets"], strategy=strat, chunk_size=K, remote_chunk_size=R,
+                     max_activity=1.0, extra_flags=flags)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R, flags)
+    s.close()
+
+
 def test_c1_gradients_all_strategies(orc32):
     w = wl.WORKLOADS["c1"]
     d = wl.make(w)

@@ -10,7 +10,7 @@ import torch
 
 import snn_workloads as wl
 from oracle import checkpointing as ck
-from oracle.oracle import (CELL_GRADED, CELL_LIF, SURR_FAST_SIGMOID, SURR_SIGMOID, NetSpec, Oracle,
+from oracle.oracle import (CELL_GRADED, CELL_LIF, SURR_FAST_SIGMOID, SURR_SIGMOID, SURR_TRIANGLE, NetSpec, Oracle,
                            leak_from_tau)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -139,8 +139,15 @@ class _SurrogateSpike(torch.autograd.Function):
         (v,) = ctx.saved_tensors
         x = (v - ctx.theta).detach().requires_grad_(True)
         with torch.enable_grad():
-            # fast sigmoid x / (1 + beta |x|) (SuperSpike) or logistic sigmoid(beta x)
-            f = x / (1 + ctx.beta * x.abs()) if ctx.kind == SURR_FAST_SIGMOID else torch.sigmoid(ctx.beta * x)
+            # fast sigmoid x / (1 + beta |x|) (SuperSpike), logistic sigmoid(beta x), or the piecewise
+            # quadratic whose derivative is the triangle beta max(0, 1 - beta |x|)
+            if ctx.kind == SURR_FAST_SIGMOID:
+                f = x / (1 + ctx.beta * x.abs())
+            elif ctx.kind == SURR_SIGMOID:
+                f = torch.sigmoid(ctx.beta * x)
+            else:
+                u = (ctx.beta * x).clamp(-1.0, 1.0)
+                f = u - 0.5 * u * u.abs()
             (d,) = torch.autograd.grad(f.sum(), x)
         return g * d, None, None, None
 
@@ -150,12 +157,13 @@ def _tiny(seed, sizes=(5, 7, 6, 3), T=6, B=2, **kw):
     return w, wl.make(w)
 
 
-@pytest.mark.parametrize("surr", [SURR_FAST_SIGMOID, SURR_SIGMOID])
+@pytest.mark.parametrize("surr", [SURR_FAST_SIGMOID, SURR_SIGMOID, SURR_TRIANGLE])
 def test_backward_matches_autograd_with_surrogate(orc64, surr):
     """Heaviside spikes, surrogate derivative in the backward: torch autograd with a custom
     spike function (derivative obtained by differentiating the smooth function itself)."""
     w, d = _tiny(3)
-    spec = spec_of(w, alpha=math.exp(-1 / 20.0), surrogate=surr, beta=4.0)
+    # the triangle has support |V - theta| < 1 / beta: a wide one here, so that the tiny case has neurons inside it
+    spec = spec_of(w, alpha=math.exp(-1 / 20.0), surrogate=surr, beta=1.0 if surr == SURR_TRIANGLE else 4.0)
     r = orc64.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
     assert 0.05 < np.mean([s[1:].mean() for s in r["S"]]) < 0.6       # the case is not degenerate
     fn = lambda v: _SurrogateSpike.apply(v, spec.theta, spec.beta, surr)
@@ -226,6 +234,20 @@ def test_surrogate_is_derivative_of_fast_sigmoid(orc64):
         fd = (f(x + h) - f(x - h)) / (2 * h) if x != 0 else 1.0
         if g_out[0, 0] != 0:
             assert abs(r["dW_ff"][0][0, 0] / g_out[0, 0] - fd) < 1e-6
+
+
+def test_triangle_surrogate_closed_form(orc64):
+    """The triangular pseudo-derivative read off a one-neuron network: beta at the threshold, half of it
+    half-way to the edge of its support, exactly zero from |V - theta| = 1 / beta on."""
+    beta, theta = 4.0, 1.0
+    for v, want in ((1.0, 4.0), (1.125, 2.0), (0.875, 2.0), (1.25, 0.0), (0.75, 0.0), (1.3, 0.0), (0.2, 0.0), (1.0625, 3.0)):
+        spec = NetSpec((1, 1, 2), 0.9, theta=theta, beta=beta, surrogate=SURR_TRIANGLE)
+        W_out = np.array([[0.8, -0.3]])
+        r = orc64.bptt_full(spec, np.ones((1, 1, 1)), [1], [np.array([[v]])], [np.zeros((1, 1))], W_out)
+        c = np.array([[1.0 if v > theta else 0.0]])
+        _, _, _, g_out, _ = orc64.readout(spec, c, np.array([1], np.int32), W_out)
+        assert g_out[0, 0] != 0
+        assert abs(r["dW_ff"][0][0, 0] / g_out[0, 0] - want) < 1e-12, v
 
 
 # ---------------------------------------------------------------- canonical fp32 order (pure Python)
