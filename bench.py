@@ -1,9 +1,11 @@
 #!/usr/bin/env python
 """Benchmark of the BPTT training step: sample-timesteps/s per checkpoint strategy.
 
-Default arm: the CUDA library on workload c2 (2 recurrent LIF layers 512-1024-1024-20, T = 1000,
-batch 32, Chunk checkpointing every 32 steps), one process per GPU; with several GPUs every rank
-runs an independent replica (the step does not shard: no collective).  One JSON line on rank 0.
+Default arm: the CUDA library on workload c4, the largest configuration of the benchmark definition
+(3 recurrent LIF layers 1024-8192-8192-8192-100, T = 2000, batch 8, Double checkpointing with
+remote checkpoints every 256 steps and local ones every 16), one process per GPU; with several GPUs
+every rank runs an independent replica (the step does not shard: no collective).  One JSON line on
+rank 0; the other workloads are timed briefly and reported under "workloads" of the same line.
 
 `--impl reference` times the CPU oracle as it stands on the host cores, each step a bounded
 sample (the first T' steps) of the same workload.
@@ -214,6 +216,61 @@ def dw_bytes(w, activity, B, n_steps):
     return total
 
 
+def host_link_probe(torch, device, nbytes=64 << 20, reps=5):
+    """Pinned-memory copy bandwidth of the host link, each way: one asynchronous copy of nbytes between a
+    page-locked host buffer and a device buffer, timed with CUDA events, best of reps (GB/s)."""
+    host = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    dev = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    st = torch.cuda.Stream(device=device)
+    best = {"h2d": 0.0, "d2h": 0.0}
+    with torch.cuda.stream(st):
+        for _ in range(reps + 1):
+            for name, dst, src in (("h2d", dev, host), ("d2h", host, dev)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(st)
+                dst.copy_(src, non_blocking=True)
+                e1.record(st)
+                e1.synchronize()
+                best[name] = max(best[name], nbytes / (e0.elapsed_time(e1) / 1e3) / 1e9)
+    return {"h2d_gbs": best["h2d"], "d2h_gbs": best["d2h"], "bytes": nbytes}
+
+
+def quick_measure(torch, name, device, flush, max_activity, steps=3):
+    """A few steps of another workload of the benchmark definition in its own strategy (CUDA events on the
+    library's stream, L2 flushed between steps): an entry of the "workloads" table, not the headline."""
+    from paper_2412_11810_b200 import Session
+    w = wl.WORKLOADS[name]
+    d = wl.make(w, dense_input=False)
+    s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate_beta=w.beta, cell=w.cell,
+                readout_scale=w.scale(), device=str(device))
+    s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    src = d["input_dense"] if w.cell == wl.CELL_GRADED else d["input_bits"].view(np.int32)
+    bits, targets = torch.from_numpy(src).to(device), torch.from_numpy(d["targets"]).to(device)
+    kw = dict(strategy=w.strategy, chunk_size=w.chunk_size, remote_chunk_size=w.remote_chunk_size,
+              max_activity=max_activity)
+    for _ in range(3):
+        s.train_step(bits, targets, **kw)
+    ms = []
+    for _ in range(steps):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(s.main):
+            e0.record(); s.train_step(bits, targets, **kw); e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    s.train_step(bits, targets, time_phases=True, **kw)
+    ph = s.phase_times()
+    dp, pp = s.peak_memory()
+    out = {"value": w.B * w.T / (float(np.median(ms)) / 1e3), "unit": UNIT, "ms_per_step": float(np.median(ms)),
+           "steps": steps, "strategy": STRATEGY_NAME[w.strategy], "chunk_size": w.chunk_size,
+           "remote_chunk_size": w.remote_chunk_size, "sizes": list(w.sizes), "T": w.T, "B": w.B,
+           "device_peak_bytes": dp, "pinned_peak_bytes": pp, "kernel_launches": int(s.stats().kernel_launches),
+           "phases_ms": {k: v[0] for k, v in ph.items()}}
+    s.close()
+    return out
+
+
 def run_ours(args, rank, world):
     import torch
     from paper_2412_11810_b200 import Session, binding as sb
@@ -270,10 +327,12 @@ def run_ours(args, rank, world):
     if rank == 0:
         clocks.start()
     wall0 = time.perf_counter()
-    ms, phases = timed_steps(args.steps, bits, targets, time_phases=True)
+    ms, _ = timed_steps(args.steps, bits, targets)
     barrier()
     wall = time.perf_counter() - wall0
     clk = clocks.stop() if rank == 0 else None
+    # the split into passes comes from separate steps: the events around every pass cost a few per cent
+    _, phases = timed_steps(min(3, args.steps), bits, targets, time_phases=True)
     stats = s.stats()
     dev_peak, pin_peak = s.peak_memory()
     total_ms = float(sum(ms))
@@ -361,6 +420,12 @@ def run_ours(args, rank, world):
                 "ms_per_step": float(np.median(tms)), "device_peak_bytes": dp, "pinned_peak_bytes": pp,
                 "local_state_slots": st.local_state_slots, "state_bytes": st.state_bytes,
                 "kernel_launches": st.kernel_launches}
+        link = host_link_probe(torch, s.device)
+        others = {}
+        if world == 1 and not args.no_other_workloads:
+            for name in sorted(wl.WORKLOADS):
+                if name != w.name:
+                    others[name] = quick_measure(torch, name, s.device, flush, args.max_activity)
         cpu = None
         if not args.no_cpu_baseline:
             from oracle.oracle import num_threads
@@ -393,11 +458,17 @@ def run_ours(args, rank, world):
                 "d2h_gbs": stats.state_bytes * stats.d2h_copies / (ph["d2h"][0] / 1e3) / 1e9 if ph["d2h"][0] > 0 else None,
                 "h2d_gbs": stats.state_bytes * stats.h2d_copies / (ph["h2d"][0] / 1e3) / 1e9 if ph["h2d"][0] > 0 else None,
                 "copy_ms_per_step": ph["d2h"][0] + ph["h2d"][0],
+                "peak": link, "peak_kind": "pinned 64 MiB copy each way, CUDA events, same run",
+                "d2h_frac": (stats.state_bytes * stats.d2h_copies / (ph["d2h"][0] / 1e3) / 1e9 / link["d2h_gbs"])
+                            if ph["d2h"][0] > 0 else None,
+                "h2d_frac": (stats.state_bytes * stats.h2d_copies / (ph["h2d"][0] / 1e3) / 1e9 / link["h2d_gbs"])
+                            if ph["h2d"][0] > 0 else None,
                 "note": "CUDA events on the side stream around every checkpoint copy; copies overlap the passes"},
             "peak_memory": {"device_bytes": dev_peak, "pinned_bytes": pin_peak,
                             "local_state_slots": stats.local_state_slots, "state_bytes": stats.state_bytes,
                             "event_bytes": stats.event_bytes},
             "strategies": per_strategy,
+            "workloads": others,
             "cpu_baseline": cpu,
             "wall_s_timed_region": wall,
         }
@@ -412,17 +483,27 @@ def run_ours(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--workload", default="c4", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--max-activity", type=float, default=0.25)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-strategies", action="store_true", help="skip the per-strategy table")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the brief runs of the other workloads")
     ap.add_argument("--flags", type=int, default=0,
                     help="extra SNN_FLAG_* bits for the timed strategy, e.g. 256 = backward with one launch per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # called as a plain script: start one replica rank per GPU and let rank 0 print the line
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":

@@ -118,7 +118,15 @@ snn_status snn_suggest_ckpt(const snn_net* net, int32_t T, int32_t B, int32_t st
 snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
                                float max_activity, size_t* device_bytes, size_t* pinned_bytes);
 
-#define SNN_INPUT_BITS 0  /* uint32 [T][B][ceil(N_0/32)], bit i%32 of word i/32 = spike of input i */
+/* The same for a step that will run with the given SNN_FLAG_* bits: SNN_FLAG_INPUT_ON_HOST adds a staging
+ * area for the input and the targets (T B N_0 values resp. T B ceil(N_0/32) words); snn_workspace_query
+ * is this call with flags = 0.  snn_train_step checks the workspace against the flags it is given. */
+snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
+                                     float max_activity, uint32_t flags, size_t* device_bytes,
+                                     size_t* pinned_bytes);
+
+#define SNN_INPUT_BITS 0  /* uint32 [T][B][ceil(N_0/32)], bit i%32 of word i/32 = spike of input i; bits at
+                             positions >= N_0 of a row's last word are ignored                          */
 #define SNN_INPUT_DENSE 1 /* fp32 [T][B][N_0], zero = no event (graded cell)                        */
 
 #define SNN_FLAG_INPUT_ON_HOST 1u /* input and targets are pinned host pointers; copied in the call */
@@ -155,7 +163,8 @@ typedef struct {
   int32_t T, B;
   const void* input;      /* device (or pinned host with SNN_FLAG_INPUT_ON_HOST), read-only       */
   int32_t input_format;   /* SNN_INPUT_BITS | SNN_INPUT_DENSE                                      */
-  const int32_t* targets; /* [B], same memory space as input                                      */
+  const int32_t* targets; /* [B], same memory space as input; each in [0, N_out), else the step
+                             returns SNN_ERR_INVALID_ARG (checked on the device, never used as an index) */
   const float* const* W_ff;  /* host array of L device pointers                                   */
   const float* const* W_rec; /* host array of L device pointers                                   */
   const float* W_out;        /* device                                                            */

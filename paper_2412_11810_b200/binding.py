@@ -30,7 +30,7 @@ SNN_OP_FWD, SNN_OP_REFWD1, SNN_OP_REFWD2, SNN_OP_BWD, SNN_OP_D2H, SNN_OP_H2D, SN
 STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "remote", SNN_DOUBLE: "double",
                   SNN_HIERARCHICAL: "hierarchical", SNN_DOUBLE_LOCAL: "double_local"}
 
-EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_train_step", "snn_peak_memory",
+EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_workspace_query_flags", "snn_train_step", "snn_peak_memory",
            "snn_memory_stats_get", "snn_last_error", "snn_plan", "snn_compact_spikes", "snn_get_event_layout",
            "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt", "snn_selftest_wait_timeout"]
 SNN_STATIC_WORKSPACE_BYTES = 32 << 20
@@ -89,6 +89,8 @@ def _load() -> C.CDLL:
     lib.snn_alpha.restype = C.c_float
     lib.snn_workspace_query.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(snn_ckpt), C.c_float,
                                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    lib.snn_workspace_query_flags.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(snn_ckpt), C.c_float,
+                                              C.c_uint32, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.snn_train_step.argtypes = [C.c_void_p, C.POINTER(snn_step_args), C.POINTER(C.c_float)]
     lib.snn_train_step_static.argtypes = [C.c_void_p, C.POINTER(snn_step_args), C.POINTER(C.c_float)]
     lib.snn_peak_memory.argtypes = [C.c_void_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
@@ -139,9 +141,9 @@ def snn_alpha(net) -> float:
     return float(lib.snn_alpha(net))
 
 
-def snn_workspace_query(net, T: int, B: int, ckpt: snn_ckpt, max_activity: float):
+def snn_workspace_query(net, T: int, B: int, ckpt: snn_ckpt, max_activity: float, flags: int = 0):
     d, p = C.c_size_t(), C.c_size_t()
-    _check(lib.snn_workspace_query(net, T, B, C.byref(ckpt), max_activity, C.byref(d), C.byref(p)), net)
+    _check(lib.snn_workspace_query_flags(net, T, B, C.byref(ckpt), max_activity, flags, C.byref(d), C.byref(p)), net)
     return d.value, p.value
 
 

@@ -21,6 +21,7 @@ constexpr int FWD_COLS = FWD_THREADS * 4;   // neurons per CTA
 constexpr int LIST_CHUNK = 1024;            // events staged in shared memory at a time
 constexpr int MAX_WORDS = 2048;             // 65536 neurons / 32
 constexpr uint32_t STATUS_EVENT_OVERFLOW = 1u;
+constexpr uint32_t STATUS_BAD_TARGET = 4u;   // a target outside [0, N_out)
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 
@@ -52,13 +53,21 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 constexpr uint32_t REC_TAG = 0x80000000u;  // list entry names a row of W_rec (else of W_ff)
 
+// Valid bits of the last spike word of a row of n neurons.
+__host__ __device__ __forceinline__ uint32_t last_word_mask(int n) {
+  return (n & 31) ? (1u << (n & 31)) - 1u : 0xffffffffu;
+}
+
 // A row of spike words made of two parts that is addressed as one: the feed-forward source
 // (layer below, this step) followed by the recurrent source (own layer, previous step).
 struct WordPair {
   const uint32_t* a; int n_a;
   const uint32_t* b; int n_b;
+  uint32_t a_last_mask = 0xffffffffu;   // valid bits of part a's last word (caller-owned input: its padding bits are ignored)
   __device__ __forceinline__ int size() const { return n_a + n_b; }
-  __device__ __forceinline__ uint32_t get(int w) const { return w < n_a ? a[w] : b[w - n_a]; }
+  __device__ __forceinline__ uint32_t get(int w) const {
+    return w < n_a ? (w == n_a - 1 ? a[w] & a_last_mask : a[w]) : b[w - n_a];
+  }
   __device__ __forceinline__ uint32_t first_index(int w) const {
     return w < n_a ? (uint32_t)w * 32u : ((uint32_t)(w - n_a) * 32u) | REC_TAG;
   }
@@ -305,7 +314,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   WordPair wp{nullptr, 0, nullptr, 0};
   if (GEN) {
     wp = WordPair{step ? L.ff_mask + (size_t)b * L.W_pre : nullptr, step ? L.W_pre : 0,
-                  L.rec_mask + (size_t)b * L.W, L.W};
+                  L.rec_mask + (size_t)b * L.W, L.W, last_word_mask(L.N_pre)};
     total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
     n_ff = s_pref[wp.n_a];
     if (tile0) {  // this CTA appends the lists to the event pools
@@ -765,8 +774,10 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
     {
       const uint32_t* ffw = L.ff_words + ((size_t)(t - L.ff_row0) * B + b) * L.W_pre;
       const uint32_t* recw = L.words + ((size_t)(t - 1) * B + b) * L.W;
-      for (int w = tid; w < L.W_pre + L.W; w += FWD_THREADS)
-        s_words[w] = __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre));
+      for (int w = tid; w < L.W_pre + L.W; w += FWD_THREADS) {
+        const uint32_t x = __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre));
+        s_words[w] = w == L.W_pre - 1 ? x & last_word_mask(L.N_pre) : x;
+      }
     }
     __syncthreads();
     const WordPair wp{s_words, L.W_pre, s_words + L.W_pre, L.W};
@@ -1008,6 +1019,7 @@ __global__ void __launch_bounds__(RS_THREADS, 1) fwd_resident_kernel(const __gri
           for (int j = 0; j < 4; ++j) {
             const int w = w0 + j * RS_COLS;
             r[j] = w < Wtot ? __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre)) : 0u;
+            if (w == L.W_pre - 1) r[j] &= last_word_mask(L.N_pre);
           }
 #pragma unroll
           for (int j = 0; j < 4; ++j)
@@ -2088,7 +2100,7 @@ readout_logits_kernel(const uint32_t* __restrict__ counts, int counts_are_float,
 
 __global__ void __launch_bounds__(256)
 softmax_loss_kernel(const float* __restrict__ logits, const int32_t* __restrict__ targets, int B, int N_out,
-                    float* __restrict__ dlogits, float* __restrict__ loss_out) {
+                    float* __restrict__ dlogits, float* __restrict__ loss_out, uint32_t* __restrict__ status) {
   extern __shared__ float s_loss[];  // [B]
   for (int b = threadIdx.x; b < B; b += 256) {
     const float* z = logits + (size_t)b * N_out;
@@ -2097,7 +2109,11 @@ softmax_loss_kernel(const float* __restrict__ logits, const int32_t* __restrict_
     float se = 0.f;
     for (int k = 0; k < N_out; ++k) se += expf(z[k] - m);
     const float lse = m + logf(se);
-    const int tg = targets[b];
+    int tg = targets[b];
+    if (tg < 0 || tg >= N_out) {   // never used as an index: the step reports it and its results are void
+      atomicOr(status, STATUS_BAD_TARGET);
+      tg = 0;
+    }
     s_loss[b] = lse - z[tg];
     for (int k = 0; k < N_out; ++k)
       dlogits[(size_t)b * N_out + k] = (expf(z[k] - lse) - (k == tg ? 1.f : 0.f)) / (float)B;

@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -28,8 +29,8 @@ struct snn_net {
   std::vector<cudaEvent_t> copy_events;    // one per checkpoint copy in flight, grown on demand
   std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
   snn_phase_times phases{};
+  int device = -1;                         // device the two figures below were asked of
   int coop_sms = -1;                       // SMs usable by a cooperative launch (-1: not asked yet)
-  size_t resident_smem_set = 0;            // dynamic shared memory fwd_resident_kernel is opted in for
   int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
 };
 
@@ -67,8 +68,8 @@ struct Layout {
   bool tier2_on_device;
 };
 
-bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float max_activity, Layout& lo,
-                    std::string& why) {
+bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float max_activity, uint32_t flags,
+                    Layout& lo, std::string& why) {
   const int L = net->L;
   const auto& sz = net->sizes;
   int n_ops = 0;
@@ -93,9 +94,11 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.vcarry = take(lo.state_bytes);   // last state of a re-forward run, start of the next
   lo.words[0] = (sz[0] + 31) / 32;
   const bool graded = net->cell == SNN_CELL_GRADED;
-  lo.in_stage = take(4 * (size_t)T * B * (graded ? sz[0] : lo.words[0]));
+  // staging of input and targets that arrive in host memory: only then
+  const bool host_input = (flags & SNN_FLAG_INPUT_ON_HOST) != 0;
+  lo.in_stage = host_input ? take(4 * (size_t)T * B * (graded ? sz[0] : lo.words[0])) : 0;
   lo.in_words = graded ? take(4 * (size_t)T * B * lo.words[0]) : 0;
-  lo.tg_stage = take(4 * (size_t)B);
+  lo.tg_stage = host_input ? take(4 * (size_t)B) : 0;
   const size_t ev0 = cur;
   for (int l = 0; l <= L; ++l) {
     lo.words[l] = (sz[l] + 31) / 32;
@@ -126,6 +129,8 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.total = cur;
   return true;
 }
+
+constexpr size_t RESIDENT_SMEM_MAX = (size_t)200 << 10;   // most dynamic shared memory fwd_resident_kernel is given
 
 #define CUDA_TRY(expr)                                                                         \
   do {                                                                                         \
@@ -174,10 +179,16 @@ extern "C" const char* snn_last_error(const snn_net* net) { return net ? net->er
 
 extern "C" snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
                                           float max_activity, size_t* device_bytes, size_t* pinned_bytes) {
+  return snn_workspace_query_flags(net, T, B, ckpt, max_activity, 0u, device_bytes, pinned_bytes);
+}
+
+extern "C" snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
+                                                float max_activity, uint32_t flags, size_t* device_bytes,
+                                                size_t* pinned_bytes) {
   if (!net || !ckpt || T < 1 || B < 1 || !(max_activity > 0.f) || max_activity > 1.f) return SNN_ERR_INVALID_ARG;
   Layout lo;
   std::string why;
-  if (!compute_layout(net, T, B, ckpt, max_activity, lo, why))
+  if (!compute_layout(net, T, B, ckpt, max_activity, flags, lo, why))
     return fail(const_cast<snn_net*>(net), SNN_ERR_INVALID_ARG, "%s", why.c_str());
   if (device_bytes) *device_bytes = lo.total;
   if (pinned_bytes) *pinned_bytes = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
@@ -446,7 +457,7 @@ struct Exec {
       ctas += (net->sizes[l] + RS_COLS - 1) / RS_COLS;
     }
     const size_t smem = resident_smem_max();
-    if (smem > (size_t)200 << 10) return false;
+    if (smem > RESIDENT_SMEM_MAX) return false;
     if (net->coop_sms < 0) {
       int dev = 0, sms = 0, coop = 0;
       if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -490,11 +501,7 @@ struct Exec {
       s.cta0 = ctas;
       ctas += s.tiles;
     }
-    const size_t smem = resident_smem_max();
-    if (smem > net->resident_smem_set) {
-      CUDA_TRY(cudaFuncSetAttribute(fwd_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      net->resident_smem_set = smem;
-    }
+    const size_t smem = resident_smem_max();   // at most RESIDENT_SMEM_MAX, which the kernel is opted in for
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L, main));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(RS_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = main;
@@ -611,7 +618,8 @@ struct Exec {
     readout_logits_kernel<<<B, 256, 8 * N_out * sizeof(float), main>>>(counts, cf, a->W_out, N_L, N_out, net->scale,
                                                                        at<float>(lo.logits));
     softmax_loss_kernel<<<1, 256, B * sizeof(float), main>>>(at<float>(lo.logits), targets, B, N_out,
-                                                             at<float>(lo.dlogits), at<float>(lo.status) + 1);
+                                                             at<float>(lo.dlogits), at<float>(lo.status) + 1,
+                                                             at<uint32_t>(lo.status));
     launches += 2;
     if (!(a->flags & SNN_FLAG_FORWARD_ONLY)) {
       readout_gout_kernel<<<(unsigned)(((size_t)B * N_L + 255) / 256), 256, 0, main>>>(
@@ -883,6 +891,43 @@ struct Exec {
 
 }  // namespace
 
+namespace {
+// Kernels that use more than 48 KB of dynamic shared memory are opted in once per device (the attribute belongs
+// to the function on one device); a mutex orders host threads that take their first step at the same time.
+constexpr int kMaxDevices = 64;
+std::mutex g_device_mutex;
+bool g_smem_opted_in[kMaxDevices] = {false};
+
+snn_status opt_in_shared_memory(snn_net* net, int dev) {
+  if (dev < 0 || dev >= kMaxDevices) return fail(net, SNN_ERR_UNSUPPORTED, "device index %d out of range", dev);
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  if (g_smem_opted_in[dev]) return SNN_OK;
+  const auto dyn = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, false>, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_resident_kernel, dyn, (int)RESIDENT_SMEM_MAX));
+  CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, dyn, (int)REFWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, dyn, (int)REFWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, dyn, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8)));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, dyn, (int)Exec::bwd_smem_bytes(16)));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, dyn, (int)Exec::bwd_smem_bytes(32)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, dyn, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, dyn, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, dyn, (int)dw_smem_bytes<4, false>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, false>, dyn, (int)dw_smem_bytes<8, false>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, dyn, (int)dw_smem_bytes<1, true>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, dyn, (int)dw_smem_bytes<2, true>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, true>, dyn, (int)dw_smem_bytes<4, true>(DW_WINDOW)));
+  CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, true>, dyn, (int)dw_smem_bytes<8, true>(DW_WINDOW)));
+  g_smem_opted_in[dev] = true;
+  return SNN_OK;
+}
+}  // namespace
+
 extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float* loss_host_out) {
   if (!net) return SNN_ERR_INVALID_ARG;
   if (!a || !loss_host_out) return fail(net, SNN_ERR_INVALID_ARG, "null argument");
@@ -914,7 +959,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   Exec ex;
   ex.net = net; ex.a = a; ex.L = L; ex.B = B; ex.T = T;
   std::string why;
-  if (!compute_layout(net, T, B, &a->ckpt, a->max_activity, ex.lo, why))
+  if (!compute_layout(net, T, B, &a->ckpt, a->max_activity, a->flags, ex.lo, why))
     return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
   const Layout& lo = ex.lo;
   const size_t pinned_need = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
@@ -939,34 +984,21 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     CUDA_TRY(cudaEventCreateWithFlags(&net->ev_main, cudaEventDisableTiming));
   }
   {
-    static bool smem_opt_in = false;   // kernels that use more than 48 KB of dynamic shared memory
-    if (!smem_opt_in) {
-
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFWD_DYN_SMEM));
-      CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(8)));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(16)));
-      CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Exec::bwd_smem_bytes(32)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<1, true>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<2, true>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<4, false>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<8, false>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<8, true>(DW_WINDOW)));
-      CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw_smem_bytes<4, true>(DW_WINDOW)));
-      smem_opt_in = true;
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (const snn_status os = opt_in_shared_memory(net, dev); os != SNN_OK) return os;
+    if (net->device != dev) {   // figures cached per net belong to the device they were asked of
+      net->device = dev;
+      net->coop_sms = -1;
+      net->fwd_segment_capacity = -1;
     }
   }
   cudaStream_t ms = ex.main;
   const auto& sz = net->sizes;
 
+  // Everything the step enqueues; an error ends the enqueueing, and the caller below still waits for both
+  // streams before it returns, so no work is in flight on the caller's buffers after any return.
+  auto enqueue = [&]() -> snn_status {
   // ---- start-of-step state: status, counts, delta carry, list offsets, spikes at t = 0, gradients
   CUDA_TRY(cudaMemsetAsync(ex.ws + lo.status, 0, 256, ms));
   CUDA_TRY(cudaMemsetAsync(ex.ws + lo.counts, 0, 4 * (size_t)B * sz[L], ms));
@@ -1031,6 +1063,9 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     }
     if (fwd_only && i == last_fwd) break;
   }
+  return st;
+  };
+  const snn_status st = enqueue();
   // ---- finish: everything on both streams, then status and loss
   cudaError_t e1 = cudaStreamSynchronize(ex.side);
   cudaError_t e2 = cudaStreamSynchronize(ex.main);
@@ -1057,6 +1092,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = lo.vals[l]; e.pool_capacity = lo.cap[l];
     e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];
   }
+  if (host_status[0] & STATUS_BAD_TARGET)
+    return fail(net, SNN_ERR_INVALID_ARG, "a target is outside [0, %d)", sz[L + 1]);
   if (host_status[0] & STATUS_SYNC_TIMEOUT)
     return fail(net, SNN_ERR_DEVICE_TIMEOUT, "a thread block gave up waiting for the spikes of another one");
   if (host_status[0] & STATUS_EVENT_OVERFLOW)
@@ -1090,8 +1127,7 @@ extern "C" snn_status snn_selftest_wait_timeout(void* device_scratch, uint32_t p
 static __device__ __align__(256) unsigned char g_static_workspace[SNN_STATIC_WORKSPACE_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
-void* g_static_workspace_addr[kMaxDevices] = {nullptr};
+void* g_static_workspace_addr[kMaxDevices] = {nullptr};   // guarded by g_device_mutex
 }  // namespace
 
 extern "C" snn_status snn_train_step_static(snn_net* net, const snn_step_args* args, float* loss_host_out) {
@@ -1103,7 +1139,7 @@ extern "C" snn_status snn_train_step_static(snn_net* net, const snn_step_args* a
   // size check first: nothing runs for a step that does not fit the built-in buffer
   Layout lo;
   std::string why;
-  if (!compute_layout(net, args->T, args->B, &args->ckpt, args->max_activity, lo, why))
+  if (!compute_layout(net, args->T, args->B, &args->ckpt, args->max_activity, args->flags, lo, why))
     return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
   if (lo.total > (size_t)SNN_STATIC_WORKSPACE_BYTES)
     return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL,
@@ -1113,14 +1149,19 @@ extern "C" snn_status snn_train_step_static(snn_net* net, const snn_step_args* a
   int dev = -1;
   CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return fail(net, SNN_ERR_UNSUPPORTED, "device index %d out of range", dev);
-  if (!g_static_workspace_addr[dev]) {  // first call on this device: resolve the buffer's device address
-    void* p = nullptr;
-    CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
-    if (!p) return fail(net, SNN_ERR_CUDA, "built-in workspace has no device address");
-    g_static_workspace_addr[dev] = p;
+  void* ws_addr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    if (!g_static_workspace_addr[dev]) {  // first call on this device: resolve the buffer's device address
+      void* p = nullptr;
+      CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
+      if (!p) return fail(net, SNN_ERR_CUDA, "built-in workspace has no device address");
+      g_static_workspace_addr[dev] = p;
+    }
+    ws_addr = g_static_workspace_addr[dev];
   }
   snn_step_args a = *args;
-  a.device_ws = g_static_workspace_addr[dev];
+  a.device_ws = ws_addr;
   a.device_ws_bytes = (size_t)SNN_STATIC_WORKSPACE_BYTES;
   return snn_train_step(net, &a, loss_host_out);
 }

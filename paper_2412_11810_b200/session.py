@@ -68,8 +68,8 @@ class Session:
     def ckpt(self, strategy: int, chunk_size: int = 0, remote_chunk_size: int = 0, nb_local: int = 0) -> sb.snn_ckpt:
         return sb.snn_ckpt(strategy, chunk_size, remote_chunk_size, nb_local)
 
-    def ensure_workspace(self, T: int, B: int, ck: sb.snn_ckpt, max_activity: float):
-        d, p = sb.snn_workspace_query(self.net, T, B, ck, max_activity)
+    def ensure_workspace(self, T: int, B: int, ck: sb.snn_ckpt, max_activity: float, flags: int = 0):
+        d, p = sb.snn_workspace_query(self.net, T, B, ck, max_activity, flags)
         if self.device_ws is None or self.device_ws.numel() < d:
             self.device_ws = None
             self.device_ws = torch.empty(d, dtype=torch.uint8, device=self.device)
@@ -96,9 +96,9 @@ class Session:
                 targets = torch.from_numpy(np.ascontiguousarray(targets, np.int32)).pin_memory()
         T, B = int(input_bits.shape[0]), int(input_bits.shape[1])
         ck = self.ckpt(strategy, chunk_size, remote_chunk_size, nb_local)
-        self.ensure_workspace(T, B, ck, max_activity)
         flags = (sb.SNN_FLAG_INPUT_ON_HOST if on_host else 0) | (sb.SNN_FLAG_FORWARD_ONLY if forward_only else 0) \
             | (sb.SNN_FLAG_TIME_PHASES if time_phases else 0) | extra_flags
+        self.ensure_workspace(T, B, ck, max_activity, flags)
         dbg = None
         if keep_V:
             self.debug_V = [torch.zeros((T + 1, B, self.sizes[l + 1]), dtype=torch.float32, device=self.device)

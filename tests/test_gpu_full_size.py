@@ -67,6 +67,26 @@ def test_truncated_sequence_at_full_width(orc32, name, T_short, K, R):
     s.close()
 
 
+def test_c5_at_its_own_gains_against_oracle(orc32):
+    """The graded workload with the benchmark's own weights, truncated to 400 steps at full width (the
+    network needs about 150 steps to reach its stationary 10 % activity), DOUBLE with K = 16 and R = 64:
+    loss, every event mask and every gradient against the oracle."""
+    w_full = wl.WORKLOADS["c5"]
+    T_short = 400
+    w = w_full.with_T(T_short)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    for x in ref["S"]:      # both hidden layers are busy over the second half: the case is not vacuous
+        assert 0.03 < float((x[T_short // 2:] != 0).mean()) < 0.3
+    s, bits, targets = make_session(w, d)
+    loss = s.train_step(bits, targets, strategy=w_full.strategy, chunk_size=16, remote_chunk_size=64,
+                        max_activity=0.25)
+    assert abs(loss - ref["loss"]) <= 1e-5 * max(1.0, abs(ref["loss"]))
+    _check_prefix_spikes(s, w, ref, T_short)
+    assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
 @pytest.mark.parametrize("name,T_prefix", [("c3", 60), ("c4", 12), ("c5", 100)])
 def test_full_length_properties(orc32, name, T_prefix):
     w = wl.WORKLOADS[name]

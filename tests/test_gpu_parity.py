@@ -315,6 +315,41 @@ def test_errors_are_reported(orc32):
     s.close()
 
 
+def test_bad_targets_and_input_padding_bits_are_guarded(orc32):
+    """Caller data never becomes an unchecked index: a target outside [0, N_out) is reported as an invalid
+    argument (and not read through), and stray bits beyond N_0 in the last input word of a row change nothing,
+    on every forward path."""
+    b = sb()
+    w = wl.small(sizes=(40, 260, 132, 6), T=21, B=5, p_in=0.1, g_ff=(2.5, 1.6), seed=17)   # 40 inputs: 8 valid bits in word 1
+    d = wl.make(w)
+    s, bits, targets = make_session(w, d)
+    for bad in (-1, w.sizes[-1], 2 ** 30):
+        t_bad = targets.clone()
+        t_bad[2] = bad
+        with pytest.raises(b.SnnError) as e:
+            s.train_step(bits, t_bad, strategy=0, max_activity=1.0)
+        assert e.value.status == b.SNN_ERR_INVALID_ARG and "target" in str(e.value)
+    dirty = bits.clone()
+    dirty[:, :, 1] |= torch.tensor(np.array(0xFFFFFF00, np.uint32).view(np.int32).item(), dtype=torch.int32)
+    for flags in (0, b.SNN_FLAG_FORWARD_STREAM_WEIGHTS, b.SNN_FLAG_FORWARD_PER_STEP):
+        loss0 = s.train_step(bits, targets, strategy=3, chunk_size=2, remote_chunk_size=8, max_activity=1.0,
+                             extra_flags=flags)
+        clean = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+        ev_clean = [s.events(l) for l in range(w.L + 1)]
+        loss1 = s.train_step(dirty, targets, strategy=3, chunk_size=2, remote_chunk_size=8, max_activity=1.0,
+                             extra_flags=flags)
+        assert loss0 == loss1
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), clean):
+            assert np.array_equal(x, y), flags
+        for l in range(w.L + 1):
+            off, pool = s.events(l)
+            assert np.array_equal(off[1:w.T + 2], ev_clean[l][0][1:w.T + 2])
+            for bb in range(w.B):
+                used = pool[bb][:int(off[w.T + 1][bb])]
+                assert used.size == 0 or int(used.max()) < w.sizes[l]
+    s.close()
+
+
 # ---------------------------------------------------------------- graded (thresholded-ReLU) cell
 def _graded(**kw):
     a = dict(cell=wl.CELL_GRADED, theta=0.3, g_ff=(1.2, 0.8), g_rec=(0.3, 0.3), p_in=0.3)

@@ -3,6 +3,7 @@ closed forms, library routines (matmul, autograd, cross-entropy), finite differe
 brute force in pure Python, and the traces and cost models the paper prints."""
 import math
 import os
+from fractions import Fraction
 
 import numpy as np
 import pytest
@@ -281,6 +282,54 @@ def test_fp32_forward_order_matches_scalar_python_loops(orc32):
         V, S = Vn, Sn
         assert np.array_equal(V, r["V"][0][t]) and np.array_equal(S, r["S"][0][t])
     assert r["S"][0].sum() > 0
+
+
+def test_fp32_graded_forward_order_matches_scalar_python_loops(orc32):
+    """The graded cell in the same style: every event contributes one fused multiply-add
+    fma(value, w, acc) in list order (feed-forward, then recurrent, ascending j); the leak is one more
+    fused multiply-add; there is no reset; the event value is V where V > theta.  The fused multiply-add
+    is evaluated exactly in rational arithmetic and rounded once to the nearest fp32 (ties to even)."""
+    w = wl.small(sizes=(6, 8, 4), T=9, B=2, seed=5, p_in=0.5, cell=CELL_GRADED, g_ff=(1.5,), g_rec=(0.6,),
+                 theta=0.3)
+    d = wl.make(w)
+    spec = spec_of(w)
+    r = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"],
+                        do_backward=False)
+    f32, f64 = np.float32, np.float64
+    alpha, theta = f32(spec.alpha), f32(spec.theta)
+    N = w.sizes[1]
+
+    def fma(a, b, c):
+        exact = Fraction(float(a)) * Fraction(float(b)) + Fraction(float(c))
+        near = f32(float(exact))                  # within one ulp of the answer: test it and its neighbours
+        cands = [near, np.nextafter(near, f32(np.inf)), np.nextafter(near, f32(-np.inf))]
+        dist = [abs(Fraction(float(x)) - exact) for x in cands]
+        best = min(dist)
+        winners = [x for x, e in zip(cands, dist) if e == best]
+        if len(winners) > 1:                      # a tie: the even mantissa wins
+            winners = [x for x in winners if (int(np.array(x, f32).view(np.uint32)) & 1) == 0]
+        return winners[0]
+
+    V = np.zeros((w.B, N), f32); A = np.zeros((w.B, N), f32)
+    n_rec_events = 0
+    for t in range(1, w.T + 1):
+        Vn = np.zeros_like(V); An = np.zeros_like(A)
+        for b in range(w.B):
+            for i in range(N):
+                acc = f32(0)
+                for j in range(w.sizes[0]):
+                    x = d["input_dense"][t - 1, b, j]
+                    if x != 0:
+                        acc = fma(x, d["W_ff"][0][j, i], acc)
+                for j in range(N):
+                    if A[b, j] != 0:
+                        acc = fma(A[b, j], d["W_rec"][0][j, i], acc)
+                        n_rec_events += 1
+                v = fma(alpha, V[b, i], acc)
+                Vn[b, i] = v; An[b, i] = v if v > theta else f32(0)
+        V, A = Vn, An
+        assert np.array_equal(V, r["V"][0][t]) and np.array_equal(A, r["S"][0][t]), t
+    assert n_rec_events > 50 and (r["S"][0] != 0).mean() > 0.05
 
 
 def test_fp32_and_fp64_forward_agree(orc32, orc64):
