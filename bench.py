@@ -327,19 +327,23 @@ def run_ours(args, rank, world):
     if rank == 0:
         clocks.start()
     wall0 = time.perf_counter()
-    ms, _ = timed_steps(args.steps, bits, targets)
+    ms, phases = timed_steps(args.steps, bits, targets, **({"time_phases": True} if args.profile else {}))
     barrier()
     wall = time.perf_counter() - wall0
     clk = clocks.stop() if rank == 0 else None
     # the split into passes comes from separate steps: the events around every pass cost a few per cent
-    _, phases = timed_steps(min(3, args.steps), bits, targets, time_phases=True)
+    if not args.profile:
+        _, phases = timed_steps(min(3, args.steps), bits, targets, time_phases=True)
     stats = s.stats()
     dev_peak, pin_peak = s.peak_memory()
     total_ms = float(sum(ms))
     # end to end: inputs start in pinned host memory, the loss comes back to the host
-    timed_steps(1, bits_host, tg_host)
-    e2e_ms, _ = timed_steps(max(3, args.steps // 4), bits_host, tg_host)
-    e2e_total = float(sum(e2e_ms)) / len(e2e_ms) * args.steps
+    if args.profile:
+        e2e_total = total_ms
+    else:
+        timed_steps(1, bits_host, tg_host)
+        e2e_ms, _ = timed_steps(max(3, args.steps // 4), bits_host, tg_host)
+        e2e_total = float(sum(e2e_ms)) / len(e2e_ms) * args.steps
     (total_ms, e2e_total), (value, e2e_value) = aggregate_replicas(
         [total_ms, e2e_total], w.B * w.T * args.steps, world, dist, s.device)
 
@@ -491,10 +495,17 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-strategies", action="store_true", help="skip the per-strategy table")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the brief runs of the other workloads")
+    ap.add_argument("--profile", action="store_true",
+                    help="for a profiler: one warm-up step and one timed step of the workload, nothing else "
+                         "(no end-to-end steps, strategy table, other workloads or CPU baseline); the printed "
+                         "numbers are not benchmark values")
     ap.add_argument("--flags", type=int, default=0,
                     help="extra SNN_FLAG_* bits for the timed strategy, e.g. 256 = backward with one launch per step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.profile:
+        args.warmup, args.steps = 1, 1
+        args.no_cpu_baseline = args.no_strategies = args.no_other_workloads = True
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         # called as a plain script: start one replica rank per GPU and let rank 0 print the line
         import socket

@@ -143,6 +143,11 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
  * currents of all its steps from the stored events at once, then the leak/reset recurrence); this flag
  * forces one launch per step, the order used for larger networks.  Results are bit-identical either way. */
 #define SNN_FLAG_REFORWARD_PER_STEP 32u
+/* Networks whose weights exceed L2 compute those input currents with the weight rows as the stationary
+ * operand instead: a thread block reads each row of its column slab once per run and adds it to every
+ * (step, sample) of the run in which that neuron fired (spiking cell).  This flag forces that order for
+ * smaller networks too.  Results are bit-identical either way. */
+#define SNN_FLAG_REFORWARD_ROWS 512u
 /* The forward pass of a spiking (LIF) network whose weights fit in L2 runs as one cooperative launch per
  * forward operation of the plan when the device can hold all its thread blocks at once: blocks wait for
  * each other's spike words sample by sample instead of once per launch.  This flag forces one launch per

@@ -11,6 +11,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "tma.cuh"
+
 namespace snnk {
 
 namespace cg = cooperative_groups;
@@ -21,6 +23,7 @@ constexpr int FWD_COLS = FWD_THREADS * 4;   // neurons per CTA
 constexpr int LIST_CHUNK = 1024;            // events staged in shared memory at a time
 constexpr int MAX_WORDS = 2048;             // 65536 neurons / 32
 constexpr uint32_t STATUS_EVENT_OVERFLOW = 1u;
+constexpr uint32_t STATUS_SYNC_TIMEOUT = 2u;     // a bounded wait (on a counter or an mbarrier) ran out
 constexpr uint32_t STATUS_BAD_TARGET = 4u;   // a target outside [0, N_out)
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
@@ -648,6 +651,225 @@ __global__ void __launch_bounds__(128) refwd_scan_kernel(const __grid_constant__
 }
 
 // ------------------------------------------------------------------------------------------
+// Input currents of a run of steps with the weight rows as the stationary operand (recomputation passes
+// of networks whose weights do not stay in L2).
+//
+// The gather above reads, for every (step, sample), each active weight row again: 16 steps x 8 samples at
+// 5 % activity touch every row about six times.  Here a CTA owns a slab of RR_COLS columns and a block of
+// (step, sample) pairs of the run, walks through the presynaptic rows in ascending order (feed-forward rows,
+// then recurrent ones), reads each row ONCE, and adds it to the accumulators of exactly those pairs in which
+// that neuron fired.  Per accumulator this is the sequence of additions of fwd_step_kernel (feed-forward
+// events ascending, then recurrent events ascending, starting from zero), hence the same bits.
+//
+// Two launches.  rows_events_kernel turns the stored spike words of the run into two 32-bit words per
+// (block of 32 rows, pair): the number of firing rows of that block, and up to four row numbers, one per byte
+// (a block with more keeps its raw spike word instead).  refwd_rows_kernel then streams the rows: one
+// elected thread issues, per block of 32 rows, one tiled bulk copy (TMA) of the [32 rows][128 columns] tile
+// and one bulk copy of the pairs' event words into a ring of RR_STAGES stages guarded by full / empty
+// mbarriers; the other warps consume: a warp owns 8 pairs, a lane four adjacent columns (8 float4
+// accumulators per thread, named statically), and an event is one 16-byte shared-memory read and two packed
+// fp32 additions.
+struct RowsLayer {
+  const uint32_t* ff_words;   // spike words of the layer below; row of step t at (t - ff_row0) * B * W_pre
+  const uint32_t* words;      // own spike words [T+1][B][W]
+  size_t state_off;           // offset of this layer inside a state slot, in floats
+  size_t ev_off;              // this layer's event words inside `events`, in words: [W_pre + W][ev_stride]
+  int N_pre, N, W_pre, W;
+  int ff_row0;                // 1 for the input (its rows start at step 1), 0 for hidden layers
+};
+
+struct RowsParams {
+  CUtensorMap map_ff[MAXL];   // W_ff^l [N_pre][N], box 32 rows x 128 columns
+  CUtensorMap map_rec[MAXL];  // W_rec^l [N][N]
+  RowsLayer lay[MAXL];
+  float* slots;               // state slot s starts at slots + s * slot_stride
+  size_t slot_stride;         // floats
+  uint32_t* events;           // event counts of the run; the row-number words follow at + raw_off
+  size_t raw_off;             // words
+  uint32_t* status;
+  int ev_stride;              // pairs rounded up to whole CTA blocks
+  int B;
+  int t0;                     // the operation computes steps t0+1 .. from the state of step t0
+  int d0, n;                  // this run: steps t0+d0+1 .. t0+d0+n
+  int buf_slot, buf_len;      // step t0+d goes to slot buf_slot + (d-1) % buf_len (as in snn_op)
+  int pb;                     // (step, sample) pairs per CTA: 16, 32, 64 or 128, one consumer warp per 8
+};
+
+constexpr int RR_COLS = 128;     // columns per CTA (32 lanes x 4)
+constexpr int RR_ROWS = 32;      // rows per tile: one spike word
+constexpr int RR_STAGES = 4;     // tiles in flight per CTA
+constexpr int RR_PPW = 8;        // pairs per consumer warp (32 accumulator registers per thread: many warps per SM
+                                 // hide the shared-memory latency of the data-dependent row reads)
+constexpr int RR_MAX_PB = 128;   // at most 16 consumer warps
+constexpr uint32_t RR_TILE_BYTES = RR_ROWS * RR_COLS * sizeof(float);
+constexpr uint32_t RR_EV_MANY = 7u;   // count field of an event word whose block has more than four firing rows
+__host__ __device__ inline size_t refwd_rows_smem_bytes(int pb) {
+  return (size_t)RR_STAGES * (RR_TILE_BYTES + 2 * (size_t)pb * sizeof(uint32_t)) + 2 * RR_STAGES * sizeof(uint64_t);
+}
+
+// Event words of the run: thread = (pair, block of 32 rows, layer).
+__global__ void __launch_bounds__(128) rows_events_kernel(const __grid_constant__ RowsParams p) {
+  pdl_launch_dependents();
+  const RowsLayer& L = p.lay[blockIdx.z];
+  const int rb = blockIdx.y, pair = blockIdx.x * 128 + threadIdx.x;
+  if (rb >= L.W_pre + L.W || pair >= p.ev_stride) return;
+  pdl_wait();
+  uint32_t bits = 0;
+  if (pair < p.n * p.B) {
+    const int t = p.t0 + p.d0 + 1 + pair / p.B, b = pair % p.B;
+    if (rb < L.W_pre) {
+      bits = L.ff_words[((size_t)(t - L.ff_row0) * p.B + b) * L.W_pre + rb];
+      if (rb == L.W_pre - 1) bits &= last_word_mask(L.N_pre);   // the input's padding bits are ignored
+    } else {
+      bits = L.words[((size_t)(t - 1) * p.B + b) * L.W + (rb - L.W_pre)];
+    }
+  }
+  // first word: the number of firing rows (RR_EV_MANY if more than four); second word: up to four row
+  // numbers, ascending, one per byte -- or the raw spike word when there are more
+  const uint32_t cnt = __popc(bits);
+  uint32_t w = RR_EV_MANY, rows = bits;
+  if (cnt <= 4) {
+    w = cnt;
+    rows = 0;
+    uint32_t rest = bits;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (rest) {
+        rows |= (uint32_t)(__ffs(rest) - 1) << (8 * k);
+        rest &= rest - 1;
+      }
+    }
+  }
+  const size_t at = L.ev_off + (size_t)rb * p.ev_stride + pair;
+  p.events[at] = w;
+  p.events[p.raw_off + at] = rows;
+}
+
+__device__ __forceinline__ void lds_2x64(uint32_t saddr, unsigned long long& a, unsigned long long& b) {
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(saddr));
+}
+// two fp32 lanes per register pair: a += w, each element rounded to nearest even (as __fadd_rn)
+__device__ __forceinline__ void add_f32x2(unsigned long long& a, const unsigned long long w) {
+  asm("add.rn.f32x2 %0, %0, %1;" : "+l"(a) : "l"(w));
+}
+
+__global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kernel(const __grid_constant__ RowsParams p) {
+  pdl_launch_dependents();
+  const int l = blockIdx.z;
+  const RowsLayer& L = p.lay[l];
+  const int col0 = blockIdx.y * RR_COLS;
+  const int pairs = p.n * p.B, pair0 = blockIdx.x * p.pb;
+  if (col0 >= L.N || pair0 >= pairs) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_consumers = p.pb / RR_PPW;            // consumer warps 0 .. n_consumers-1, then the producer warp
+  extern __shared__ __align__(128) unsigned char s_raw_bytes[];
+  float4* const s_tiles = reinterpret_cast<float4*>(s_raw_bytes);                                 // [RR_STAGES][32][32]
+  uint32_t* const s_ev = reinterpret_cast<uint32_t*>(s_raw_bytes + (size_t)RR_STAGES * RR_TILE_BYTES);   // [RR_STAGES][2][pb]
+  uint64_t* const s_full = reinterpret_cast<uint64_t*>(s_ev + (size_t)RR_STAGES * 2 * p.pb);       // [RR_STAGES]
+  uint64_t* const s_empty = s_full + RR_STAGES;
+  const int n_blocks = L.W_pre + L.W;
+  if (tid == 0) {
+    for (int s = 0; s < RR_STAGES; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, n_consumers); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  const uint32_t ev_bytes = (uint32_t)p.pb * sizeof(uint32_t);
+  if (warp == n_consumers) {
+    // ---- producer: one thread keeps the ring full
+    if (lane == 0) {
+      const uint32_t* ev_src = p.events + L.ev_off + pair0;
+      for (int rb = 0; rb < n_blocks; ++rb) {
+        const int stage = rb % RR_STAGES;
+        if (rb >= RR_STAGES && !mbar_wait(s_empty + stage, (uint32_t)(rb / RR_STAGES - 1) & 1u)) {
+          atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+          break;
+        }
+        mbar_arrive_expect_tx(s_full + stage, RR_TILE_BYTES + 2 * ev_bytes);
+        const bool ff = rb < L.W_pre;
+        tma_load_2d(s_tiles + (size_t)stage * (RR_TILE_BYTES / 16), ff ? &p.map_ff[l] : &p.map_rec[l], col0,
+                    (ff ? rb : rb - L.W_pre) * RR_ROWS, s_full + stage);
+        uint32_t* const dst = s_ev + (size_t)stage * 2 * p.pb;
+        bulk_load(dst, ev_src + (size_t)rb * p.ev_stride, ev_bytes, s_full + stage);
+        bulk_load(dst + p.pb, ev_src + p.raw_off + (size_t)rb * p.ev_stride, ev_bytes, s_full + stage);
+      }
+    }
+    return;   // copies still in flight complete on barriers the consumers wait for before they leave
+  }
+  // ---- consumers
+  unsigned long long acc01[RR_PPW], acc23[RR_PPW];
+#pragma unroll
+  for (int i = 0; i < RR_PPW; ++i) acc01[i] = acc23[i] = 0ull;   // +0.0f in both halves
+  const uint32_t lane_off = smem_u32(s_tiles) + (uint32_t)lane * 16u;
+  for (int rb = 0; rb < n_blocks; ++rb) {
+    const int stage = rb % RR_STAGES;
+    if (!mbar_wait(s_full + stage, (uint32_t)(rb / RR_STAGES) & 1u)) {
+      if (lane == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+      return;
+    }
+    const uint32_t tile = lane_off + (uint32_t)stage * RR_TILE_BYTES;
+    const uint32_t* const evs = s_ev + (size_t)stage * 2 * p.pb + warp * RR_PPW;
+    uint32_t e[RR_PPW];
+#pragma unroll
+    for (int i = 0; i < RR_PPW / 4; ++i) {
+      const uint4 x = reinterpret_cast<const uint4*>(evs)[i];
+      e[4 * i] = x.x; e[4 * i + 1] = x.y; e[4 * i + 2] = x.z; e[4 * i + 3] = x.w;
+    }
+    uint32_t rw[RR_PPW];
+#pragma unroll
+    for (int i = 0; i < RR_PPW / 4; ++i) {
+      const uint4 x = reinterpret_cast<const uint4*>(evs + p.pb)[i];
+      rw[4 * i] = x.x; rw[4 * i + 1] = x.y; rw[4 * i + 2] = x.z; rw[4 * i + 3] = x.w;
+    }
+    // one event: the row's 16 bytes of this lane, two packed additions
+    auto add_row = [&](int i, uint32_t r) {
+      unsigned long long w01, w23;
+      lds_2x64(tile + r * (RR_COLS * 4u), w01, w23);
+      add_f32x2(acc01[i], w01); add_f32x2(acc23[i], w23);
+    };
+#pragma unroll
+    for (int i = 0; i < RR_PPW; ++i) {
+      // the count is the same for the whole warp: real branches, the common counts first, straight-line
+      // code for each (independent reads, additions in ascending row order)
+      const uint32_t cnt = e[i], r = rw[i];
+      if (cnt == 0) {
+      } else if (cnt == 1) {
+        add_row(i, r & 0xffu);
+      } else if (cnt == 2) {
+        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu);
+      } else if (cnt == 3) {
+        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu); add_row(i, (r >> 16) & 0xffu);
+      } else if (cnt == 4) {
+        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu); add_row(i, (r >> 16) & 0xffu); add_row(i, r >> 24);
+      } else {
+        uint32_t bits = r;
+        while (bits) {
+          add_row(i, (uint32_t)__ffs(bits) - 1u);
+          bits &= bits - 1;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(s_empty + stage);
+  }
+  const int col = col0 + lane * 4;
+  if (col < L.N) {
+#pragma unroll
+    for (int i = 0; i < RR_PPW; ++i) {
+      const int pair = pair0 + warp * RR_PPW + i;
+      if (pair < pairs) {
+        const int d = p.d0 + 1 + pair / p.B, b = pair % p.B;
+        float4 v;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(v.x), "=f"(v.y) : "l"(acc01[i]));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(v.z), "=f"(v.w) : "l"(acc23[i]));
+        *reinterpret_cast<float4*>(p.slots + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride + L.state_off +
+                                   (size_t)b * L.N + col) = v;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Forward pass over a whole segment of steps in one cooperative launch (LIF cell).
 //
 // Unlike the recomputation above the spikes are not known yet, so a CTA (column tile, sample b,
@@ -659,7 +881,6 @@ __global__ void __launch_bounds__(128) refwd_scan_kernel(const __grid_constant__
 // step or owned by the writing thread, so running ahead overwrites nothing that is still needed.
 // All CTAs must be resident together (cooperative launch); a wait that does not end within
 // SYNC_POLL_LIMIT polls raises STATUS_SYNC_TIMEOUT and the CTA returns.
-constexpr uint32_t STATUS_SYNC_TIMEOUT = 2u;
 constexpr uint32_t SYNC_POLL_LIMIT = 1u << 22;   // a few seconds
 constexpr int SEG_WORDS = 1024;                  // spike words of both sources of a layer, staged per step
 

@@ -63,6 +63,9 @@ struct Layout {
   size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets)
   bool layer_major;      // backward goes layer by layer over runs of steps, with that product batched over time
   bool weights_resident; // all weight matrices together stay in L2
+  size_t rows_ev;        // event words of a run of recomputed steps (refwd_rows_kernel), then the raw words
+  size_t rows_ev_words;  // words of each of the two halves
+  size_t rows_ev_stride; // words per block of 32 rows: the pairs of the longest run, rounded up
   size_t tier2;          // DOUBLE_LOCAL: the second checkpoint tier, in device memory
   int n_local, n_remote;
   bool tier2_on_device;
@@ -122,6 +125,17 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     lo.weights_resident = wbytes <= ((size_t)96 << 20);
     lo.layer_major = L > 1 && !lo.weights_resident;
     lo.gff = L > 1 ? take(4 * (size_t)BWD_RUN * B * maxN) : 0;
+  }
+  lo.rows_ev = 0; lo.rows_ev_words = 0; lo.rows_ev_stride = 0;
+  if (!graded && ck->strategy != SNN_STANDARD) {
+    // one word per (32 presynaptic rows, pair) for the pairs of a run (at most chunk_size steps), twice
+    const int Kc = std::min(std::max(ck->chunk_size, 1), T);
+    const size_t stride = ((size_t)Kc * B + RR_MAX_PB - 1) / RR_MAX_PB * RR_MAX_PB;
+    size_t blocks = 0;
+    for (int l = 1; l <= L; ++l) blocks += (size_t)lo.words[l - 1] + lo.words[l];
+    lo.rows_ev_stride = stride;
+    lo.rows_ev_words = stride * blocks;
+    lo.rows_ev = take(2 * 4 * lo.rows_ev_words);
   }
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
   lo.tier2_on_device = ck->strategy == SNN_DOUBLE_LOCAL;
@@ -378,8 +392,65 @@ struct Exec {
   // state slots the operation writes to.  Used while the weights stay in L2; beyond that the per-step
   // launches keep the samples in step, and the rows they share are read from HBM once.
   bool reforward_runs_possible(const snn_op& op) const {
-    if (!lo.weights_resident || (a->flags & SNN_FLAG_REFORWARD_PER_STEP)) return false;
+    if (a->flags & SNN_FLAG_REFORWARD_PER_STEP) return false;
+    if (reforward_rows()) return true;
+    if (!lo.weights_resident) return false;
     return (long long)L * std::min(op.buf_len, op.t1 - op.t0) <= 65535;
+  }
+  // the currents of a run come from refwd_rows_kernel (weight rows stationary) rather than refwd_gather_kernel
+  bool reforward_rows() const {
+    return !graded() && (!lo.weights_resident || (a->flags & SNN_FLAG_REFORWARD_ROWS));
+  }
+
+  // Input currents of steps t0+d0+1 .. t0+d0+n with the weight rows stationary (weights beyond L2).
+  RowsParams rows_params;        // tensor maps and per-layer constants, filled on first use in a step
+  bool rows_params_ready = false;
+  snn_status launch_reforward_rows(const snn_op& op, int d0, int n) {
+    RowsParams& r = rows_params;
+    int slabs_all = 0, slabs_max = 0, blocks_max = 0;
+    for (int l = 1; l <= L; ++l) {
+      const int slabs = (net->sizes[l] + RR_COLS - 1) / RR_COLS;
+      slabs_all += slabs; slabs_max = std::max(slabs_max, slabs);
+      blocks_max = std::max(blocks_max, lo.words[l - 1] + lo.words[l]);
+    }
+    // pairs per CTA: as many as a CTA can hold, halved while the grid would leave SMs without two CTAs
+    // (every block of pairs streams the rows again; blocks of one slab are neighbours in launch order and
+    // share the rows through L2)
+    const int pairs = n * B;
+    int pb = RR_MAX_PB;
+    while (pb > 16 && (pb / 2 >= pairs || (long long)slabs_all * ((pairs + pb - 1) / pb) < 2 * 148)) pb /= 2;
+    const int n_pb = (pairs + pb - 1) / pb;
+    if (!rows_params_ready) {
+      std::memset(&r, 0, sizeof r);
+      size_t ev_off = 0;
+      const size_t stride_max = lo.rows_ev_stride;
+      for (int l = 1; l <= L; ++l) {
+        RowsLayer& s = r.lay[l - 1];
+        s.ff_words = l == 1 ? in_mask(1) : mask(l - 1, 0);
+        s.ff_row0 = l == 1 ? 1 : 0;
+        s.words = mask(l, 0);
+        s.state_off = lo.layer_off[l];
+        s.N_pre = net->sizes[l - 1]; s.N = net->sizes[l]; s.W_pre = lo.words[l - 1]; s.W = lo.words[l];
+        s.ev_off = ev_off;
+        ev_off += stride_max * ((size_t)s.W_pre + s.W);
+        if (!make_tensor_map_2d(&r.map_ff[l - 1], a->W_ff[l - 1], (uint64_t)s.N_pre, (uint64_t)s.N, (uint64_t)s.N, RR_ROWS, RR_COLS, false) ||
+            !make_tensor_map_2d(&r.map_rec[l - 1], a->W_rec[l - 1], (uint64_t)s.N, (uint64_t)s.N, (uint64_t)s.N, RR_ROWS, RR_COLS, false))
+          return fail(net, SNN_ERR_CUDA, "tensor map of a weight matrix could not be encoded");
+      }
+      r.slots = at<float>(lo.slots); r.slot_stride = lo.state_bytes / 4;
+      r.events = at<uint32_t>(lo.rows_ev); r.raw_off = lo.rows_ev_words;
+      r.status = at<uint32_t>(lo.status);
+      r.B = B;
+      rows_params_ready = true;
+    }
+    r.t0 = op.t0; r.d0 = d0; r.n = n; r.buf_slot = op.buf_slot; r.buf_len = op.buf_len;
+    r.pb = pb; r.ev_stride = n_pb * pb;
+    CUDA_TRY(launch_pdl(rows_events_kernel, dim3((unsigned)((r.ev_stride + 127) / 128), (unsigned)blocks_max, (unsigned)L),
+                        dim3(128), 0, r));
+    CUDA_TRY(launch_pdl(refwd_rows_kernel, dim3((unsigned)n_pb, (unsigned)slabs_max, (unsigned)L),
+                        dim3(32 * (pb / RR_PPW + 1)), refwd_rows_smem_bytes(pb), r));
+    launches += 2;
+    return SNN_OK;
   }
 
   snn_status run_reforward_runs(const snn_op& op) {
@@ -411,9 +482,14 @@ struct Exec {
       const int n = std::min(op.buf_len, n_all - d0);
       g.d0 = c.d0 = d0; g.n = c.n = n;
       c.v_start = d0 == 0 ? at<float>(lo.slots) + (size_t)op.in_slot * g.slot_stride : c.carry;
-      CUDA_TRY(launch_pdl(kg, dim3(fg.x, fg.y, (unsigned)(L * n)), dim3(FWD_THREADS), REFWD_DYN_SMEM, g));
+      if (!reforward_rows()) {
+        CUDA_TRY(launch_pdl(kg, dim3(fg.x, fg.y, (unsigned)(L * n)), dim3(FWD_THREADS), REFWD_DYN_SMEM, g));
+        ++launches;
+      } else if (const snn_status st = launch_reforward_rows(op, d0, n); st != SNN_OK) {
+        return st;
+      }
       CUDA_TRY(launch_pdl(kc, dim3((unsigned)((c.n_quads + 127) / 128)), dim3(128), 0, c));
-      launches += 2;
+      ++launches;
     }
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
@@ -911,6 +987,7 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(fwd_resident_kernel, dyn, (int)RESIDENT_SMEM_MAX));
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, dyn, (int)REFWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, dyn, (int)REFWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(refwd_rows_kernel, dyn, (int)refwd_rows_smem_bytes(RR_MAX_PB)));
   CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, dyn, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8)));
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, dyn, (int)Exec::bwd_smem_bytes(16)));

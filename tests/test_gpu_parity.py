@@ -486,8 +486,9 @@ def test_layer_by_layer_backward_order(orc32):
 
 def test_reforward_as_one_launch_per_segment(orc32):
     """The recomputation passes walk through a whole segment inside one launch (small networks: the
-    default).  Gradients must be bit-identical to STANDARD, which recomputes nothing, and to the same
-    strategy with one launch per step; sizes that are no multiple of the column tile, segments longer
+    default), with the input currents gathered per (step, sample) or accumulated with the weight rows
+    stationary (the order of large networks, forced here).  Gradients must be bit-identical to STANDARD, which
+    recomputes nothing, and to the same strategy with one launch per step; sizes that are no multiple of the column tile, segments longer
     than the 32 steps staged at a time, steps with no events at all and steps with more events than
     one window of the merged list (1024) holds."""
     b = sb()
@@ -495,6 +496,7 @@ def test_reforward_as_one_launch_per_segment(orc32):
         wl.small(sizes=(70, 700, 1300, 7), T=83, B=5, p_in=0.05, g_ff=(2.5, 1.4), g_rec=(1.0, 1.0), seed=51),
         wl.small(sizes=(40, 4000, 6), T=12, B=2, p_in=0.5, g_ff=(6.0,), g_rec=(3.0,), seed=52),     # > 1024 events per step
         wl.small(sizes=(64, 96, 5), T=90, B=3, p_in=0.01, g_ff=(1.5,), g_rec=(0.5,), seed=53),      # mostly silent steps
+        wl.small(sizes=(33, 260, 136, 7), T=50, B=20, p_in=0.1, g_ff=(2.5, 1.6), seed=55),          # 800 (step, sample) pairs per run
     ]
     for w in cases:
         d = wl.make(w)
@@ -505,7 +507,7 @@ def test_reforward_as_one_launch_per_segment(orc32):
         base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
         for strat, K, R, P in [(1, 40, 0, 0), (1, 7, 0, 0), (2, 11, 0, 0), (3, 4, 16, 0), (3, 3, 9, 0), (4, 5, 0, 3), (5, 2, 8, 0)]:
             for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_REFORWARD_PER_STEP | b.SNN_FLAG_FORWARD_PER_STEP,
-                          b.SNN_FLAG_FORWARD_STREAM_WEIGHTS):
+                          b.SNN_FLAG_FORWARD_STREAM_WEIGHTS, b.SNN_FLAG_REFORWARD_ROWS):
                 for g in s.dW_ff + s.dW_rec + [s.dW_out]:
                     g.fill_(float("nan"))
                 s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, nb_local=P,
