@@ -47,8 +47,7 @@ def read_peaks():
 # the kernel still has that text.  The backward pass of c2 now runs in bwd_segment_kernel, a cooperative launch
 # of thread-block clusters that the profiler cannot launch: no counters, hence no entry.
 NCU_TRAFFIC = {
-    ("c4", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
-                    269405952 + 3885312),
+    ("c4", "bwd"): ("bwd_stream_kernel", "", 0),
     ("c3", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
                     51018240 + 43264),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
@@ -373,7 +372,11 @@ def run_ours(args, rank, world):
                 # small spiking networks: one cooperative launch per forward operation, T steps in all;
                 # the bytes are per step, so the launch count is replaced by the step count
                 kernel, units = "fwd_resident_kernel / fwd_segment_kernel (per step)", w.T
-            if dominant == "bwd" and ph["bwd"][1] < w.T:
+            if dominant == "bwd" and ph["ffgemm"][1] > 0 and ph["bwd"][1] < w.T * w.L:
+                # large networks: one cooperative launch per layer and run of 32 steps that keeps W_rec streaming;
+                # the bytes are per step of one layer
+                kernel, units = "bwd_stream_kernel (per layer and step)", w.T * w.L
+            elif dominant == "bwd" and ph["bwd"][1] < w.T:
                 # small networks: one cooperative launch per segment with the weights resident
                 kernel, units = "bwd_segment_kernel (per step)", w.T
             avg_s = ph[dominant][0] / 1e3 / units

@@ -163,6 +163,10 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
  * cooperative launch with those weights resident.  This flag forces one launch per step.  Results are
  * bit-identical either way. */
 #define SNN_FLAG_BACKWARD_PER_STEP 256u
+/* The feed-forward product of the layer-by-layer order runs on the tcgen05 tensor cores (accumulator in tensor
+ * memory).  This flag selects the older mma.sync kernel instead; the two agree to rounding (both are three-pass
+ * tf32 products with fp32 accumulation), not bit for bit. */
+#define SNN_FLAG_FF_PRODUCT_MMA_SYNC 1024u
 
 typedef struct {
   int32_t T, B;

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SOURCES = [os.path.join(CSRC, "snn_api.cu"), os.path.join(CSRC, "schedule.cpp")]
-HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(HERE, "..", "include", "snn.h")]
+HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "tma.cuh"), os.path.join(CSRC, "tc_gemm.cuh"), os.path.join(HERE, "..", "include", "snn.h")]
 LIB = os.path.join(HERE, "libsnnckpt.so")
 # -fmad=false: nothing is fused unless the source says fmaf; the forward arithmetic that decides
 # spikes is written with explicit intrinsics anyway.

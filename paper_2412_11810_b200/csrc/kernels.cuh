@@ -1528,15 +1528,13 @@ __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer&
 // accumulation, which keeps the result at fp32 accuracy (the dropped lo*lo term is ~2^-22 relative).
 constexpr int BWD_LD = 132;   // padded row length (floats) of the staged tiles: fragment loads hit 32 banks
 
-// fp32 -> tf32 (10 mantissa bits), round to nearest with ties away from zero: half an ulp added to the
-// magnitude, then the 13 low bits cleared.  Two integer operations at full rate instead of a conversion
-// instruction, which runs at an eighth of it and would cost as much as the tensor-core work it feeds.
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-  return (__float_as_uint(x) + 0x1000u) & 0xffffe000u;
-}
+// fp32 -> two tf32 pieces (10 mantissa bits each): hi = x with its 13 low mantissa bits cleared, lo = x - hi (exact
+// in fp32: the cleared bits) cut to tf32 the same way.  Three integer / floating-point operations at full rate per
+// value; conversion instructions run at an eighth of it and would cost as much as the tensor-core work they feed.
+// hi + lo differs from x by less than 2^-20 |x|.
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
-  hi = to_tf32(x);
-  lo = to_tf32(x - __uint_as_float(hi));
+  hi = __float_as_uint(x) & 0xffffe000u;
+  lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
 }
 // D(16x8) += A(16x8, row) * B(8x8, col); lane = 4 g + t holds A[g][t], A[g+8][t], A[g][t+4], A[g+8][t+4],
 // B[t][g], B[t+4][g] and D[g][2t], D[g][2t+1], D[g+8][2t], D[g+8][2t+1].
@@ -1547,6 +1545,83 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
+// Row length (floats) of the staged W and delta tiles of the step kernels.  A lane reads 2 KS adjacent values
+// of a row with one 64- or 128-bit load (KS = 16 / NWARP k-steps per warp and chunk); rows 8 (KS = 1) or 16
+// (KS = 2) banks apart make those loads conflict-free.
+__host__ __device__ constexpr int bwd_ld(int nwarp) { return nwarp == 8 ? 144 : 136; }
+
+// One warp's share of a chunk of 128 contraction values: KS consecutive k-steps of 8, i.e. the 8 KS values from
+// warp * 8 KS on.  Lane (g, t) loads, from each of its rows, the 2 KS adjacent values at 2 KS t with one vector
+// load and splits each once; within k-step j the hardware's k slots t and t + 4 take values 2 j and 2 j + 1 of
+// that group, for W and delta alike (the contraction does not care which k sits in which slot as long as both
+// operands agree).  Wl / Dl: this lane's first value in row g of the W tile / the delta tile; further rows of W
+// at multiples of 8 ldw, further sample tiles at multiples of 8 ldd.  Per k-step three passes, small terms
+// first; `between(phase)` runs after each pass (phases 0, 1, 2 of the first k-step are where callers issue the
+// copies that refill a stage).
+template <int NTN, int KS, class Between>
+__device__ __forceinline__ void warp_chunk_mma(float (&acc)[2][NTN][4], const float* Wl, int ldw, const float* Dl,
+                                               int ldd, Between&& between) {
+  static_assert(KS == 1 || KS == 2, "one or two k-steps per warp and chunk");
+  uint32_t wh[4][2 * KS], wlo[4][2 * KS], dh[NTN][2 * KS], dlo[NTN][2 * KS];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    float v[2 * KS];
+    if (KS == 2) {
+      const float4 x = *reinterpret_cast<const float4*>(Wl + (size_t)r * 8 * ldw);
+      v[0] = x.x; v[1] = x.y; v[2 * KS - 2] = x.z; v[2 * KS - 1] = x.w;
+    } else {
+      const float2 x = *reinterpret_cast<const float2*>(Wl + (size_t)r * 8 * ldw);
+      v[0] = x.x; v[1] = x.y;
+    }
+#pragma unroll
+    for (int i = 0; i < 2 * KS; ++i) split_tf32(v[i], wh[r][i], wlo[r][i]);
+  }
+#pragma unroll
+  for (int nt = 0; nt < NTN; ++nt) {
+    float v[2 * KS];
+    if (KS == 2) {
+      const float4 x = *reinterpret_cast<const float4*>(Dl + (size_t)nt * 8 * ldd);
+      v[0] = x.x; v[1] = x.y; v[2 * KS - 2] = x.z; v[2 * KS - 1] = x.w;
+    } else {
+      const float2 x = *reinterpret_cast<const float2*>(Dl + (size_t)nt * 8 * ldd);
+      v[0] = x.x; v[1] = x.y;
+    }
+#pragma unroll
+    for (int i = 0; i < 2 * KS; ++i) split_tf32(v[i], dh[nt][i], dlo[nt][i]);
+  }
+#pragma unroll
+  for (int j = 0; j < KS; ++j) {
+    uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {   // rows mt 16 + g (loaded row 2 mt) and mt 16 + g + 8 (loaded row 2 mt + 1)
+      a_hi[mt][0] = wh[2 * mt][2 * j];     a_hi[mt][1] = wh[2 * mt + 1][2 * j];
+      a_hi[mt][2] = wh[2 * mt][2 * j + 1]; a_hi[mt][3] = wh[2 * mt + 1][2 * j + 1];
+      a_lo[mt][0] = wlo[2 * mt][2 * j];     a_lo[mt][1] = wlo[2 * mt + 1][2 * j];
+      a_lo[mt][2] = wlo[2 * mt][2 * j + 1]; a_lo[mt][3] = wlo[2 * mt + 1][2 * j + 1];
+    }
+#pragma unroll
+    for (int nt = 0; nt < NTN; ++nt) {
+      b_hi[nt][0] = dh[nt][2 * j]; b_hi[nt][1] = dh[nt][2 * j + 1];
+      b_lo[nt][0] = dlo[nt][2 * j]; b_lo[nt][1] = dlo[nt][2 * j + 1];
+    }
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
+    between(3 * j);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
+    between(3 * j + 1);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
+    between(3 * j + 2);
+  }
+}
+
 // NTN = sample tiles of 8 per pass (BP = 8 NTN samples), NWARP warps per CTA; launched with cluster
 // size CS along x: blockIdx.x = row_tile * CS + rank.  A CTA owns 32 rows x BP samples.  Chunks of
 // 128 k of W [32][128] and delta [BP][128] stream through a BWD_STAGES-deep cp.async pipeline; within
@@ -1555,7 +1630,8 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
 // across the cluster in rank order.
 template <int NTN, int NWARP>
 __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kernel(const __grid_constant__ BwdParams p) {
-  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * BWD_LD, TILE = BWD_TM * BP;
+  constexpr int LD = bwd_ld(NWARP), KS = 16 / NWARP;
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * LD, TILE = BWD_TM * BP;
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;   // padded rows of the warps' partial tiles: 64-bit stores without bank conflicts
   constexpr int EPI = TILE / NT;                    // output elements a thread finishes at most (cluster of one)
   static_assert(TILE % NT == 0 && NWARP * TILEP <= BWD_STAGES * STAGE_F, "partial tiles fit the stages");
@@ -1569,7 +1645,7 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   __shared__ float s_part[TILE];
   extern __shared__ float4 s_dyn[];
-  float* const s_tiles = reinterpret_cast<float*>(s_dyn);   // [BWD_STAGES][ROWS][BWD_LD]; later [NWARP][32][BP]
+  float* const s_tiles = reinterpret_cast<float*>(s_dyn);   // [BWD_STAGES][ROWS][LD]; later [NWARP][32][BP]
   // this rank's slice of each contraction range, in units of 4 floats
   const int q_rec = L.N / 4, q_ff = L.W_ffa ? L.N_post / 4 : 0;
   const int lo_rec = (int)((long long)q_rec * rank / CS) * 4, hi_rec = (int)((long long)q_rec * (rank + 1) / CS) * 4;
@@ -1597,7 +1673,7 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
     for (int j = 0; j < ITER; ++j) {
       const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
       kcol[j] = 4 * c4;
-      dst_off[j] = rr * BWD_LD + 4 * c4;
+      dst_off[j] = rr * LD + 4 * c4;
       if (rr < BWD_TM) {   // rows and samples past the end are clamped to the last valid one; never used
         const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;
         src_rec[j] = L.W_rec + row * L.N + 4 * c4;
@@ -1643,46 +1719,13 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
       // order one after the other they would take turns instead of overlapping.
       const int it_refill = it + BWD_STAGES - 1;
       const float* Ws = s_tiles + (size_t)(it % BWD_STAGES) * STAGE_F;
-      const float* Ds = Ws + BWD_TM * BWD_LD;
-#pragma unroll
-      for (int ksl = 0; ksl < 16 / NWARP; ++ksl) {   // this warp's k-steps of the chunk: warp, warp + NWARP, ...
-        const bool refill = ksl == 0;
-        const int kk = (warp + ksl * NWARP) * 8 + t;
-        uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          const float* r0 = Ws + (mt * 16 + g) * BWD_LD + kk;
-          split_tf32(r0[0], a_hi[mt][0], a_lo[mt][0]);
-          split_tf32(r0[8 * BWD_LD], a_hi[mt][1], a_lo[mt][1]);
-          split_tf32(r0[4], a_hi[mt][2], a_lo[mt][2]);
-          split_tf32(r0[8 * BWD_LD + 4], a_hi[mt][3], a_lo[mt][3]);
-        }
-#pragma unroll
-        for (int nt = 0; nt < NTN; ++nt) {
-          const float* r0 = Ds + (nt * 8 + g) * BWD_LD + kk;
-          split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
-          split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
-        }
-        // small terms first; consecutive instructions go to different accumulators
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
-        if (refill) issue_part(it_refill, 0, ITER / 3);
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
-        if (refill) issue_part(it_refill, ITER / 3, 2 * ITER / 3);
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
-        if (refill) {
-          issue_part(it_refill, 2 * ITER / 3, ITER);
-          cp_async_commit();
-        }
-      }
+      const float* Ds = Ws + BWD_TM * LD;
+      const int kl = warp * 8 * KS + 2 * KS * t;   // this lane's values of the chunk
+      warp_chunk_mma<NTN, KS>(acc, Ws + g * LD + kl, LD, Ds + g * LD + kl, LD, [&](int phase) {
+        if (phase == 0) issue_part(it_refill, 0, ITER / 3);
+        else if (phase == 1) issue_part(it_refill, ITER / 3, 2 * ITER / 3);
+        else if (phase == 2) { issue_part(it_refill, 2 * ITER / 3, ITER); cp_async_commit(); }
+      });
     }
     cp_async_wait<0>();
     __syncthreads();   // the stages are free: they now hold the warps' partial tiles [NWARP][32][TS]
@@ -1738,6 +1781,205 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
 }
 
 // ------------------------------------------------------------------------------------------
+// Backward steps of ONE layer over a run of steps in one cooperative launch, the recurrent matrix streaming
+// from HBM without a pause (networks whose weights exceed L2: the layer-by-layer order).
+//
+// With one launch per step the HBM stream of W_rec stops at every step boundary: the next launch cannot start
+// its copies before delta_t is complete.  But the weights do not depend on the step.  Here a CTA (32 rows of
+// W_rec, all samples, the whole contraction range: no cluster) walks through the steps itself and keeps its
+// copy ring busy across the boundary: while the last chunks of step t are multiplied, the W parts of the first
+// chunks of step t-1 are already on their way; only their delta parts wait until every CTA has published
+// its rows of delta_t (one counter of finished (CTA, step) pairs, release add / acquire poll; delta is read
+// past L1).  Tiling, arithmetic and order of additions are those of bwd_step_kernel with a cluster of one:
+// bit-identical results.  Cooperative launch (all CTAs resident); bounded waits.
+struct BwdStreamParams {
+  const float* W_rec;       // [N][N]
+  const float* g_out;       // [B][N] (last layer) or null
+  const float* g_ff;        // feed-forward term of the run [n_steps][B][N] (first row: step t0 + ts_lo + 1), or null
+  const float* d_first;     // [B][N] delta_{t+1} of the run's latest step
+  float* carry_out;         // [B][N] receives delta of the step with ts == 0, or null
+  float* slots;             // state slot s starts at slots + s * slot_stride
+  size_t slot_stride;       // floats
+  size_t state_off;         // offset of this layer inside a state slot, in floats
+  uint32_t* status;
+  uint32_t* progress;       // finished (CTA, step) pairs, zero at launch
+  int N, B;
+  int buf_slot, ts_lo, ts_hi;   // steps ts = ts_hi-1 .. ts_lo; slot buf_slot + ts holds V on entry, delta on exit
+  float alpha, theta, beta;
+  int surrogate, cell;
+};
+
+template <int NTN, int NWARP>
+__host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
+  return ((size_t)BWD_STAGES * (BWD_TM + 8 * NTN) * bwd_ld(NWARP) + (size_t)NWARP * BWD_TM * (8 * NTN + 8)) * sizeof(float);
+}
+
+template <int NTN, int NWARP>
+__global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
+  constexpr int LD = bwd_ld(NWARP), KS = 16 / NWARP;
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * LD, TILE = BWD_TM * BP;
+  constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
+  constexpr int EPI = TILE / NT;
+  constexpr int ITER = ROWS * 32 / NT;      // 16-byte positions of a staged chunk per thread
+  constexpr int JW = BWD_TM * 32 / NT;      // the first JW of them are rows of W, the others rows of delta
+  static_assert(TILE % NT == 0 && ROWS * 32 % NT == 0 && BWD_TM * 32 % NT == 0, "tiles divide evenly among the threads");
+  const int tile_row0 = blockIdx.x * BWD_TM;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  __shared__ int s_ok;
+  extern __shared__ float4 s_dyn[];
+  float* const s_tiles = reinterpret_cast<float*>(s_dyn);            // [BWD_STAGES][ROWS][LD]
+  float* const s_parts = s_tiles + (size_t)BWD_STAGES * STAGE_F;     // [NWARP][32][TS] partial tiles of the warps
+  const int N = p.N, it_all = (N + 127) / 128, n_steps = p.ts_hi - p.ts_lo;
+  const int total = n_steps * it_all;                                 // chunks of the whole run
+  const int rlast = N - 1, blast = p.B - 1;
+  // fixed copy positions of this thread
+  const float* src_w[JW];
+  int d_row[ITER - JW], dst_off[ITER], kcol[ITER];
+#pragma unroll
+  for (int j = 0; j < ITER; ++j) {
+    const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
+    kcol[j] = 4 * c4;
+    dst_off[j] = rr * LD + 4 * c4;
+    if (j < JW) {   // rows and samples past the end are clamped to the last valid one; never used
+      const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;
+      src_w[j] = p.W_rec + row * N + 4 * c4;
+    } else {
+      d_row[j - JW] = rr - BWD_TM < blast ? rr - BWD_TM : blast;
+    }
+  }
+  // delta_{t+1} of the s-th step of the run (s = 0: the latest)
+  auto dn_of = [&](int s) -> const float* {
+    return s == 0 ? p.d_first : p.slots + (size_t)(p.buf_slot + p.ts_hi - s) * p.slot_stride + p.state_off;
+  };
+  // W part of chunk c (the `it`-th of its step), positions [j0, j1) among the W positions
+  auto issue_w = [&](int c, int it, int j0, int j1) {
+    if (c < total) {
+      const int k0 = it * 128;
+      float* st = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
+#pragma unroll
+      for (int j = 0; j < JW; ++j) {
+        if (j < j0 || j >= j1) continue;
+        if (k0 + kcol[j] < N) cp_async16(st + dst_off[j], src_w[j] + k0);
+        else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  };
+  // delta part of chunk c (the `it`-th of its step)
+  auto issue_d = [&](int c, int it, const float* dn) {
+    const int k0 = it * 128;
+    float* st = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
+#pragma unroll
+    for (int j = JW; j < ITER; ++j) {
+      if (k0 + kcol[j] < N) cp_async16(st + dst_off[j], dn + (size_t)d_row[j - JW] * N + kcol[j] + k0);
+      else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  // the W parts of the first chunks: they do not depend on anything this launch computes
+  int it_pre = 0;   // index within its step of the next chunk whose W part is issued (chunks wrap around the steps)
+  for (int c = 0; c < BWD_STAGES - 1; ++c) {
+    issue_w(c, it_pre, 0, JW);
+    cp_async_commit();
+    if (++it_pre == it_all) it_pre = 0;
+  }
+
+  for (int s = 0; s < n_steps; ++s) {
+    const int ts = p.ts_hi - 1 - s;
+    if (s > 0) {   // every CTA has written its rows of delta_{t+1}
+      if (tid == 0) {
+        const bool ok = wait_progress(p.progress, (uint32_t)gridDim.x * (uint32_t)s);
+        if (!ok) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+        s_ok = ok ? 1 : 0;
+      }
+      __syncthreads();
+      if (!s_ok) { cp_async_wait<0>(); return; }
+    }
+    const float* const dn = dn_of(s);
+    float* const Vd = p.slots + (size_t)(p.buf_slot + ts) * p.slot_stride + p.state_off;
+    const float* const gff = p.g_ff ? p.g_ff + (size_t)(ts - p.ts_lo) * p.B * N : nullptr;
+    // what the epilogue needs, fetched now (delta_{t+1} may come from another CTA of this launch: past L1)
+    float pre_dn[EPI], pre_go[EPI], pre_gf[EPI], pre_v[EPI];
+#pragma unroll
+    for (int j = 0; j < EPI; ++j) {
+      const int e = tid + j * NT, i = tile_row0 + e / BP, b = e % BP;
+      pre_dn[j] = pre_go[j] = pre_gf[j] = pre_v[j] = 0.f;
+      if (i < N && b < p.B) {
+        const size_t k = (size_t)b * N + i;
+        pre_dn[j] = __ldcg(dn + k);
+        pre_go[j] = p.g_out ? p.g_out[k] : 0.f;
+        pre_gf[j] = gff ? gff[k] : 0.f;
+        pre_v[j] = Vd[k];
+      }
+    }
+    // delta parts of the chunks of this step whose W part is already in flight
+    const int c0 = s * it_all;
+    for (int cc = 0; cc < BWD_STAGES - 1 && cc < it_all; ++cc) issue_d(c0 + cc, cc, dn);
+    cp_async_commit();
+    float acc[2][NTN][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+    for (int it = 0; it < it_all; ++it) {
+      const int c = c0 + it;
+      if (it == 0) cp_async_wait<0>();          // the delta parts issued just above are the latest group
+      else cp_async_wait<BWD_STAGES - 2>();     // this thread's copies of chunk c have landed
+      __syncthreads();                               // ... everybody's have, and chunk c-1 has been consumed
+      // refill of the stage chunk c-1 used: chunk c + BWD_STAGES - 1, its delta part only if it is of this step
+      const int c_refill = c + BWD_STAGES - 1;
+      const bool refill_d = it + BWD_STAGES - 1 < it_all;
+      const float* Ws = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
+      const float* Ds = Ws + BWD_TM * LD;
+      const int kl = warp * 8 * KS + 2 * KS * t;   // this lane's values of the chunk
+      // the copies that refill a stage are issued between the tensor-core passes
+      warp_chunk_mma<NTN, KS>(acc, Ws + g * LD + kl, LD, Ds + g * LD + kl, LD, [&](int phase) {
+        if (phase == 0) issue_w(c_refill, it_pre, 0, JW / 2);
+        else if (phase == 1) issue_w(c_refill, it_pre, JW / 2, JW);
+        else if (phase == 2) {
+          if (refill_d) issue_d(c_refill, it_pre, dn);
+          cp_async_commit();
+        }
+      });
+      if (++it_pre == it_all) it_pre = 0;
+    }
+    // the warps' partial tiles, summed in warp order
+    {
+      float* mine = s_parts + (size_t)warp * TILEP;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) {
+          const int r = mt * 16 + g, cc = nt * 8 + 2 * t;
+          *reinterpret_cast<float2*>(mine + r * TS + cc) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+          *reinterpret_cast<float2*>(mine + (r + 8) * TS + cc) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < EPI; ++j) {
+      const int e = tid + j * NT, i = tile_row0 + e / BP, b = e % BP;
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) sum += s_parts[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+      if (i < N && b < p.B) {
+        const size_t k = (size_t)b * N + i;
+        float gs = sum + pre_go[j];
+        if (gff) gs += pre_gf[j];
+        if (p.cell == 0) gs = fmaf(-p.theta, pre_dn[j], gs);
+        const float sp = surrogate_grad(pre_v[j], p.theta, p.beta, p.surrogate, p.cell);
+        const float dl = fmaf(gs, sp, p.alpha * pre_dn[j]);
+        Vd[k] = dl;
+        if (ts == 0 && p.carry_out) p.carry_out[k] = dl;
+      }
+    }
+    __syncthreads();   // delta_t of this CTA is written, and the partial tiles are free again
+    if (tid == 0) publish_progress(p.progress);
+  }
+  cp_async_wait<0>();
+}
+
+// ------------------------------------------------------------------------------------------
 // Backward pass over a whole segment in one cooperative launch, the weights resident in shared memory
 // (networks small enough that a CTA's slice of both matrices, 32 rows x its share of the contraction
 // index, fits beside the staging ring).
@@ -1777,17 +2019,17 @@ struct BwdSegParams {
 };
 
 constexpr int BSEG_STAGES = 3;   // chunks of delta in flight per warp
-constexpr int BSEG_LD = 12;      // floats per (k-step, sample) row of a warp's delta stage: 8 k + 4, fragment loads hit 32 banks
 
 // floats of the resident slice per row: every chunk of 128 k (feed-forward part first, each part padded to
-// whole chunks with zeros) plus 4 so that fragment loads hit 32 banks
-__host__ __device__ inline int bwd_resident_ld(int k_ff, int k_rec) {
-  return ((k_ff + 127) / 128 + (k_rec + 127) / 128) * 128 + 4;
+// whole chunks with zeros) plus the padding that makes the lanes' vector loads conflict-free (bwd_ld)
+__host__ __device__ inline int bwd_resident_ld(int k_ff, int k_rec, int nwarp) {
+  return ((k_ff + 127) / 128 + (k_rec + 127) / 128) * 128 + (bwd_ld(nwarp) - 128);
 }
 template <int NTN, int NWARP> __host__ __device__ constexpr size_t bwd_segment_region_floats() {
-  // the warps' delta rings (16 k-steps of a chunk x BP samples x BSEG_LD per stage), reused for their partial tiles
-  return (size_t)(BSEG_STAGES * 16 * 8 * NTN * BSEG_LD) > (size_t)(NWARP * BWD_TM * (8 * NTN + 8))
-             ? (size_t)(BSEG_STAGES * 16 * 8 * NTN * BSEG_LD) : (size_t)(NWARP * BWD_TM * (8 * NTN + 8));
+  // the warps' delta rings (per stage the warp's 8 KS values of a chunk for BP samples: 128 BP floats over all
+  // warps), reused for their partial tiles
+  return (size_t)(BSEG_STAGES * 128 * 8 * NTN) > (size_t)(NWARP * BWD_TM * (8 * NTN + 8))
+             ? (size_t)(BSEG_STAGES * 128 * 8 * NTN) : (size_t)(NWARP * BWD_TM * (8 * NTN + 8));
 }
 
 template <int NTN, int NWARP>
@@ -1796,8 +2038,9 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
   constexpr int EPI = TILE / NT;
   constexpr int KS = 16 / NWARP;                 // k-steps of a chunk per warp
-  constexpr int WSTAGE_F = KS * BP * BSEG_LD;    // floats of one warp's stage: its k-steps x BP samples x 8 k (padded)
-  constexpr int PIECES = KS * BP * 2;            // 16-byte pieces of it
+  constexpr int KW = 8 * KS;                     // its contraction values per chunk, adjacent
+  constexpr int WSTAGE_F = BP * KW;              // floats of one warp's stage: BP samples x KW values
+  constexpr int PIECES = BP * KW / 4;            // 16-byte pieces of it
   constexpr int ITER = (PIECES + 31) / 32;       // per lane
   static_assert(TILE % NT == 0 && 16 % NWARP == 0, "tiles divide evenly among the threads");
   cg::cluster_group cluster = cg::this_cluster();
@@ -1816,9 +2059,9 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
   const int lo_rec = (int)((long long)q_rec * rank / CS) * 4, hi_rec = (int)((long long)q_rec * (rank + 1) / CS) * 4;
   const int lo_ff = (int)((long long)q_ff * rank / CS) * 4, hi_ff = (int)((long long)q_ff * (rank + 1) / CS) * 4;
   const int it_ff = (hi_ff - lo_ff + 127) / 128, it_all = it_ff + (hi_rec - lo_rec + 127) / 128;
-  const int LDW = it_all * 128 + 4;
+  const int LDW = it_all * 128 + (bwd_ld(NWARP) - 128);
   float* const Wres = reinterpret_cast<float*>(s_dyn);             // [32][LDW]
-  float* const s_reg = Wres + (size_t)BWD_TM * LDW;                // per-warp delta rings [NWARP][BSEG_STAGES][KS][BP][BSEG_LD]; later partial tiles
+  float* const s_reg = Wres + (size_t)BWD_TM * LDW;                // per-warp delta rings [NWARP][BSEG_STAGES][BP][KW]; later partial tiles
   float* const ring = s_reg + (size_t)warp * BSEG_STAGES * WSTAGE_F;
   const int rlast = L.N - 1, blast = p.B - 1;
 
@@ -1871,18 +2114,18 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
           pre_v[j] = Vd[k];
         }
       }
-      // Every warp stages the delta values of its own k-steps (8 k x BP samples each: two 16-byte pieces per
-      // sample) in a ring of its own, so that no warp waits for another one inside the contraction and the
+      // Every warp stages the delta values of its own k-steps (KW adjacent values x BP samples: KW / 4 16-byte
+      // pieces per sample) in a ring of its own, so that no warp waits for another one inside the contraction and the
       // loads, splits and tensor-core passes of different warps overlap.  A lane copies fixed pieces.
       const float* src_rec[ITER];
       const float* src_ff[ITER];
       int dst_off[ITER], kofs[ITER];
 #pragma unroll
       for (int j = 0; j < ITER; ++j) {
-        const int q = lane + j * 32;                                   // piece: (k-step of the warp, sample, half)
-        const int ksl = q / (BP * 2), sm = (q / 2) % BP, half = q & 1;
-        kofs[j] = q < PIECES ? (warp + ksl * NWARP) * 8 + half * 4 : -1;   // k inside the chunk
-        dst_off[j] = (ksl * BP + sm) * BSEG_LD + half * 4;
+        const int q = lane + j * 32;                                   // piece: (sample, quarter of the warp's values)
+        const int sm = q / (KW / 4), part = q % (KW / 4);
+        kofs[j] = q < PIECES ? warp * KW + part * 4 : -1;              // k inside the chunk
+        dst_off[j] = sm * KW + part * 4;
         const size_t b = bp0 + sm < blast ? bp0 + sm : blast;           // samples past the batch: a valid row, never used
         src_rec[j] = dn + b * L.N;
         src_ff[j] = above ? da + b * L.N_post : nullptr;
@@ -1916,38 +2159,8 @@ __global__ void __launch_bounds__(32 * NWARP, 1) bwd_segment_kernel(const __grid
         issue(it + BSEG_STAGES - 1);        // refills the stage chunk it-1 used
         const float* Wc = Wres + it * 128;
         const float* Ds = ring + (size_t)(it % BSEG_STAGES) * WSTAGE_F;
-#pragma unroll
-        for (int ksl = 0; ksl < KS; ++ksl) {
-          const int kk = (warp + ksl * NWARP) * 8 + t4;
-          uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            const float* r0 = Wc + (size_t)(mt * 16 + g) * LDW + kk;
-            split_tf32(r0[0], a_hi[mt][0], a_lo[mt][0]);
-            split_tf32(r0[(size_t)8 * LDW], a_hi[mt][1], a_lo[mt][1]);
-            split_tf32(r0[4], a_hi[mt][2], a_lo[mt][2]);
-            split_tf32(r0[(size_t)8 * LDW + 4], a_hi[mt][3], a_lo[mt][3]);
-          }
-#pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) {
-            const float* r0 = Ds + (ksl * BP + nt * 8 + g) * BSEG_LD + t4;
-            split_tf32(r0[0], b_hi[nt][0], b_lo[nt][0]);
-            split_tf32(r0[4], b_hi[nt][1], b_lo[nt][1]);
-          }
-          // small terms first; consecutive instructions go to different accumulators
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
-        }
+        warp_chunk_mma<NTN, KS>(acc, Wc + (size_t)g * LDW + warp * KW + 2 * KS * t4, LDW, Ds + g * KW + 2 * KS * t4, KW,
+                                [](int) {});
       }
       cp_async_wait<0>();
       __syncthreads();   // the ring is free: it now holds the warps' partial tiles [NWARP][32][TS]

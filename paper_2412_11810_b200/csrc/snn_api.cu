@@ -12,6 +12,7 @@
 
 #include "../../include/snn.h"
 #include "kernels.cuh"
+#include "tc_gemm.cuh"
 
 using namespace snnk;
 
@@ -32,6 +33,7 @@ struct snn_net {
   int device = -1;                         // device the two figures below were asked of
   int coop_sms = -1;                       // SMs usable by a cooperative launch (-1: not asked yet)
   int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
+  int bwd_stream_capacity[3] = {-1, -1, -1};   // the same for the three instances of bwd_stream_kernel
 };
 
 namespace {
@@ -402,6 +404,10 @@ struct Exec {
     return !graded() && (!lo.weights_resident || (a->flags & SNN_FLAG_REFORWARD_ROWS));
   }
 
+  // tensor maps of the feed-forward matrices for ff_gemm_tc_kernel: 0 not tried yet, 1 ready, -1 not encodable
+  CUtensorMap ffw_map[MAXL];
+  int ffw_map_ready[MAXL] = {0};
+
   // Input currents of steps t0+d0+1 .. t0+d0+n with the weight rows stationary (weights beyond L2).
   RowsParams rows_params;        // tensor maps and per-layer constants, filled on first use in a step
   bool rows_params_ready = false;
@@ -718,10 +724,10 @@ struct Exec {
     ++launches;
   }
   // dynamic shared memory of bwd_step_kernel for BP samples per pass: the staged tiles
-  static size_t bwd_smem_bytes(int bp) { return (size_t)BWD_STAGES * (BWD_TM + bp) * BWD_LD * sizeof(float); }
+  static size_t bwd_smem_bytes(int bp, int ld = BWD_LD) { return (size_t)BWD_STAGES * (BWD_TM + bp) * ld * sizeof(float); }
   template <int NTN, int NWARP> cudaError_t launch_bwd(const BwdParams& p, int tiles, int CS, int n_layers = 0) {
     return launch_pdl(bwd_step_kernel<NTN, NWARP>, dim3(tiles * CS, 1, n_layers ? n_layers : L), dim3(32 * NWARP),
-                      bwd_smem_bytes(8 * NTN), p, CS);
+                      bwd_smem_bytes(8 * NTN, bwd_ld(NWARP)), p, CS);
   }
 
   // BWD: layer wavefront, layer l runs L-l steps behind the last layer; then the weight
@@ -752,7 +758,7 @@ struct Exec {
       for (int r = 0; r < CS; ++r) {
         const int k_rec = (int)((long long)q_rec * (r + 1) / CS) * 4 - (int)((long long)q_rec * r / CS) * 4;
         const int k_ff = (int)((long long)q_ff * (r + 1) / CS) * 4 - (int)((long long)q_ff * r / CS) * 4;
-        res_floats = std::max(res_floats, (size_t)BWD_TM * bwd_resident_ld(k_ff, k_rec));
+        res_floats = std::max(res_floats, (size_t)BWD_TM * bwd_resident_ld(k_ff, k_rec, NWARP));
       }
     }
     const size_t smem = 4 * (res_floats + bwd_segment_region_floats<NTN, NWARP>());
@@ -781,6 +787,42 @@ struct Exec {
     p.surrogate = net->surrogate; p.cell = net->cell;
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L, main));
     if (cudaLaunchKernelEx(&cfg, k, p) != cudaSuccess) {   // e.g. refused under a profiler: one launch per step instead
+      cudaGetLastError();
+      return SNN_OK;
+    }
+    ++launches;
+    done = true;
+    return SNN_OK;
+  }
+
+  // Steps ts_hi-1 .. ts_lo of one layer in one cooperative launch (bwd_stream_kernel), if the device holds all
+  // its CTAs at once; otherwise `done` stays false and the caller launches step by step.
+  template <int NTN, int NWARP> snn_status try_backward_stream(const BwdStreamParams& sp, int tiles, bool& done) {
+    done = false;
+    void (*k)(BwdStreamParams) = bwd_stream_kernel<NTN, NWARP>;
+    const size_t smem = bwd_stream_smem_bytes<NTN, NWARP>();
+    int& cap = net->bwd_stream_capacity[NTN == 1 ? 0 : NTN == 2 ? 1 : 2];
+    if (cap < 0) {
+      int dev = 0, sms = 0, per_sm = 0, coop = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, 32 * NWARP, smem) != cudaSuccess) {
+        cudaGetLastError();
+        cap = 0;
+      } else {
+        cap = coop ? sms * per_sm : 0;
+      }
+    }
+    if (tiles > cap) return SNN_OK;
+    CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4, main));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)tiles); cfg.blockDim = dim3(32 * NWARP); cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cudaLaunchAttribute at1[1];
+    at1[0].id = cudaLaunchAttributeCooperative;
+    at1[0].val.cooperative = 1;
+    cfg.attrs = at1; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, k, sp) != cudaSuccess) {
       cudaGetLastError();
       return SNN_OK;
     }
@@ -828,22 +870,72 @@ struct Exec {
         const int lo_s = std::max(0, hi - BWD_RUN);     // steps t0+lo_s+1 .. t0+hi
         for (int l = L; l >= 1; --l) {
           if (l < L) {
-            FfGemmParams gp;
-            gp.W = a->W_ff[l]; gp.N = sz[l]; gp.K = sz[l + 1]; gp.B = B; gp.n_steps = hi - lo_s;
-            gp.delta0 = slot(op.buf_slot + lo_s, l + 1); gp.slot_stride = lo.state_bytes / 4;
-            gp.out = at<float>(lo.gff);
             end_span(span);
             span = begin_span(SNN_PHASE_FFGEMM);
-            CUDA_TRY(launch_pdl(ff_gemm_kernel, dim3((gp.n_steps * B + 8 * FFG_NTN - 1) / (8 * FFG_NTN), (sz[l] + BWD_TM - 1) / BWD_TM),
-                                dim3(32 * FFG_NWARP),
-                                bwd_smem_bytes(8 * FFG_NTN), gp));
+            const int n_run = hi - lo_s;
+            bool on_tcgen05 = false;
+            if (!(a->flags & SNN_FLAG_FF_PRODUCT_MMA_SYNC) && B <= TCG_NMAX) {
+              // tcgen05 path: 128 rows of W x up to 128 pairs per CTA, accumulator in tensor memory
+              TcGemmParams tp;
+              std::memset(&tp, 0, sizeof tp);
+              tp.steps_per_tile = std::min(n_run, TCG_NMAX / B);
+              tp.n_cols = (tp.steps_per_tile * B + 15) / 16 * 16;
+              tp.out = at<float>(lo.gff); tp.status = at<uint32_t>(lo.status);
+              tp.N = sz[l]; tp.K = sz[l + 1]; tp.B = B; tp.n_steps = n_run;
+              if (!ffw_map_ready[l]) {
+                ffw_map_ready[l] = make_tensor_map_2d(&ffw_map[l], a->W_ff[l], (uint64_t)sz[l], (uint64_t)sz[l + 1],
+                                                      (uint64_t)sz[l + 1], TCG_M, TCG_KB, true) ? 1 : -1;
+              }
+              if (ffw_map_ready[l] > 0 &&
+                  make_tensor_map_delta(&tp.map_d, slot(op.buf_slot + lo_s, l + 1), (uint64_t)sz[l + 1], (uint64_t)B,
+                                        (uint64_t)n_run, lo.state_bytes / 4, (uint32_t)tp.steps_per_tile)) {
+                tp.map_w = ffw_map[l];
+                CUDA_TRY(launch_pdl(ff_gemm_tc_kernel,
+                                    dim3((unsigned)((n_run + tp.steps_per_tile - 1) / tp.steps_per_tile),
+                                         (unsigned)((sz[l] + TCG_M - 1) / TCG_M)),
+                                    dim3(TCG_THREADS), TCG_SMEM_BYTES, tp));
+                on_tcgen05 = true;
+              }
+            }
+            if (!on_tcgen05) {
+              FfGemmParams gp;
+              gp.W = a->W_ff[l]; gp.N = sz[l]; gp.K = sz[l + 1]; gp.B = B; gp.n_steps = n_run;
+              gp.delta0 = slot(op.buf_slot + lo_s, l + 1); gp.slot_stride = lo.state_bytes / 4;
+              gp.out = at<float>(lo.gff);
+              CUDA_TRY(launch_pdl(ff_gemm_kernel, dim3((gp.n_steps * B + 8 * FFG_NTN - 1) / (8 * FFG_NTN), (sz[l] + BWD_TM - 1) / BWD_TM),
+                                  dim3(32 * FFG_NWARP),
+                                  bwd_smem_bytes(8 * FFG_NTN), gp));
+            }
             ++launches;
             end_span(span);
             span = begin_span(SNN_PHASE_BWD);
           }
           const int tiles_l = (sz[l] + BWD_TM - 1) / BWD_TM;
           int CS_l = 1;
-          while (CS_l < 8 && tiles_l * CS_l * 2 <= wave && sz[l] / (4 * CS_l * 2) >= 32) CS_l *= 2;
+          // layers with a row tile for every SM: no cluster, so that the run can be one launch that keeps the
+          // weight stream going (bwd_stream_kernel)
+          while (tiles_l < 148 && CS_l < 8 && tiles_l * CS_l * 2 <= wave && sz[l] / (4 * CS_l * 2) >= 32) CS_l *= 2;
+          if (CS_l == 1 && B <= 32 && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
+            BwdStreamParams sp;
+            std::memset(&sp, 0, sizeof sp);
+            sp.W_rec = a->W_rec[l - 1];
+            sp.g_out = l == L ? at<float>(lo.g_out) : nullptr;
+            sp.g_ff = l < L ? at<float>(lo.gff) : nullptr;
+            sp.d_first = op.t0 + hi == op.t1 ? carry(carry_cur, l) : slot(op.buf_slot + hi, l);
+            sp.carry_out = lo_s == 0 ? carry(carry_cur ^ 1, l) : nullptr;
+            sp.slots = at<float>(lo.slots); sp.slot_stride = lo.state_bytes / 4; sp.state_off = lo.layer_off[l];
+            sp.status = at<uint32_t>(lo.status); sp.progress = at<uint32_t>(lo.progress);
+            sp.N = sz[l]; sp.B = B; sp.buf_slot = op.buf_slot; sp.ts_lo = lo_s; sp.ts_hi = hi;
+            sp.alpha = net->alpha; sp.theta = net->theta; sp.beta = net->beta;
+            sp.surrogate = net->surrogate; sp.cell = net->cell;
+            bool done = false;
+            snn_status st = SNN_OK;
+            if (B <= 8) st = try_backward_stream<1, 8>(sp, tiles_l, done);
+            else if (B <= 16) st = try_backward_stream<2, 8>(sp, tiles_l, done);
+            else st = try_backward_stream<4, 16>(sp, tiles_l, done);
+            if (st != SNN_OK) return st;
+            if (done) continue;
+          }
           for (int ts = hi - 1; ts >= lo_s; --ts) {
             const int t = op.t0 + ts + 1;
             std::memset(&p.lay[0], 0, sizeof p.lay[0]);
@@ -989,9 +1081,13 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, dyn, (int)REFWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(refwd_rows_kernel, dyn, (int)refwd_rows_smem_bytes(RR_MAX_PB)));
   CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, dyn, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8)));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, dyn, (int)Exec::bwd_smem_bytes(16)));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, dyn, (int)Exec::bwd_smem_bytes(32)));
+  CUDA_TRY(cudaFuncSetAttribute(ff_gemm_tc_kernel, dyn, (int)TCG_SMEM_BYTES));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8, bwd_ld(8))));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, dyn, (int)Exec::bwd_smem_bytes(16, bwd_ld(8))));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, dyn, (int)Exec::bwd_smem_bytes(32, bwd_ld(16))));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8>, dyn, (int)bwd_stream_smem_bytes<1, 8>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8>, dyn, (int)bwd_stream_smem_bytes<2, 8>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16>, dyn, (int)bwd_stream_smem_bytes<4, 16>()));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, dyn, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, dyn, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, dyn, (int)dw_smem_bytes<4, false>(DW_WINDOW)));
@@ -1068,6 +1164,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       net->device = dev;
       net->coop_sms = -1;
       net->fwd_segment_capacity = -1;
+      net->bwd_stream_capacity[0] = net->bwd_stream_capacity[1] = net->bwd_stream_capacity[2] = -1;
     }
   }
   cudaStream_t ms = ex.main;

@@ -481,6 +481,46 @@ def test_layer_by_layer_backward_order(orc32):
     # the wavefront order agrees within tolerance (different summation, not bit-identical)
     s.train_step(bits, targets, strategy=1, chunk_size=9, extra_flags=b.SNN_FLAG_BACKWARD_WAVEFRONT)
     assert_grads_close(s.gradients(), ref)
+    # so does the feed-forward product on the mma.sync kernel instead of the tcgen05 one, and it is deterministic too
+    g = f | b.SNN_FLAG_FF_PRODUCT_MMA_SYNC
+    s.train_step(bits, targets, strategy=0, extra_flags=g)
+    assert_grads_close(s.gradients(), ref)
+    legacy = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    assert any(not np.array_equal(x, y) for x, y in zip(legacy, base))      # really another kernel
+    s.train_step(bits, targets, strategy=3, chunk_size=4, remote_chunk_size=16, extra_flags=g)
+    for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), legacy):
+        assert np.array_equal(x, y)
+    s.close()
+
+
+@pytest.mark.parametrize("B", [3, 8, 11, 19])
+def test_layer_by_layer_backward_as_one_launch_per_run(orc32, B):
+    """Wide layers under the layer-by-layer order run the steps of a run of 32 as ONE cooperative launch that
+    keeps the recurrent matrix streaming across step boundaries.  It must give the bits of the same order with
+    one launch per step, for each batch tiling (8, 16, 32 samples), a width that is no multiple of the row tile
+    or of the 128-wide chunk, runs shorter and longer than the copy ring, and agree with the oracle.  (The wide
+    layer takes that launch for up to 8 samples, where two of its thread blocks fit an SM; the narrow one always.)"""
+    b = sb()
+    w = wl.small(sizes=(48, 4772, 132, 7), T=37, B=B, p_in=0.1, g_ff=(2.5, 1.5), g_rec=(1.0, 1.0), seed=43)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    assert all(0.005 < float(x[1:].mean()) < 0.5 for x in ref["S"])
+    s, bits, targets = make_session(w, d)
+    f = b.SNN_FLAG_BACKWARD_LAYER_BY_LAYER
+    s.train_step(bits, targets, strategy=0, extra_flags=f)
+    launches_stream = s.stats().kernel_launches
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    s.train_step(bits, targets, strategy=0, extra_flags=f | b.SNN_FLAG_BACKWARD_PER_STEP)
+    assert s.stats().kernel_launches > launches_stream + 30          # the wide layer really took the other path
+    for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+        assert np.array_equal(x, y)
+    for strat, K, R in [(1, 9, 0), (3, 2, 6), (2, 35, 0)]:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, extra_flags=f)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R)
     s.close()
 
 
