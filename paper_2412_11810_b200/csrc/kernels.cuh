@@ -1440,7 +1440,10 @@ struct BwdLayer {
   const float* d_next;    // [B][N]      delta^l_{t+1}
   const float* d_above;   // [B][N_post] delta^{l+1}_t or null
   const float* g_out;     // [B][N] or null
-  const float* g_ff;      // [B][N] or null: W_ff^{l+1} delta^{l+1}_t computed ahead for a run of steps
+  const float* g_ff;      // [B][N] or null: W_ff^{l+1} delta^{l+1}_t computed ahead for a run of steps, as
+                          // g_ff_parts partial sums over slices of the contraction range, g_ff_stride floats apart
+  size_t g_ff_stride;
+  int g_ff_parts;
   float* carry_out;       // optional second copy of delta_t
   int N, N_post;
   int mode;               // 0 idle, 1 step
@@ -1505,7 +1508,10 @@ __device__ __forceinline__ BwdPre bwd_prefetch(const BwdParams& p, const BwdLaye
   const size_t k = (size_t)b * L.N + i;
   r.dn = L.d_next[k];
   r.go = L.g_out ? L.g_out[k] : 0.f;
-  r.gf = L.g_ff ? L.g_ff[k] : 0.f;
+  if (L.g_ff) {   // the partial sums in slice order
+    r.gf = L.g_ff[k];
+    for (int s = 1; s < L.g_ff_parts; ++s) r.gf += L.g_ff[(size_t)s * L.g_ff_stride + k];
+  }
   r.v = L.V_delta[k];
   return r;
 }
@@ -1795,7 +1801,10 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
 struct BwdStreamParams {
   const float* W_rec;       // [N][N]
   const float* g_out;       // [B][N] (last layer) or null
-  const float* g_ff;        // feed-forward term of the run [n_steps][B][N] (first row: step t0 + ts_lo + 1), or null
+  const float* g_ff;        // feed-forward term of the run [n_steps][B][N] (first row: step t0 + ts_lo + 1), or null;
+                            // g_ff_parts partial sums over slices of the contraction range, g_ff_stride floats apart
+  size_t g_ff_stride;
+  int g_ff_parts;
   const float* d_first;     // [B][N] delta_{t+1} of the run's latest step
   float* carry_out;         // [B][N] receives delta of the step with ts == 0, or null
   float* slots;             // state slot s starts at slots + s * slot_stride
@@ -1906,7 +1915,10 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
         const size_t k = (size_t)b * N + i;
         pre_dn[j] = __ldcg(dn + k);
         pre_go[j] = p.g_out ? p.g_out[k] : 0.f;
-        pre_gf[j] = gff ? gff[k] : 0.f;
+        if (gff) {   // the partial sums in slice order
+          pre_gf[j] = gff[k];
+          for (int q = 1; q < p.g_ff_parts; ++q) pre_gf[j] += gff[(size_t)q * p.g_ff_stride + k];
+        }
         pre_v[j] = Vd[k];
       }
     }

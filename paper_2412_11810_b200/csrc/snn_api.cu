@@ -62,7 +62,9 @@ struct Layout {
   int words[MAXL + 1];
   size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
   size_t event_bytes, total;
-  size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets)
+  size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets),
+                         // as up to TCG_MAX_KSPLIT partial products gff_stride floats apart
+  size_t gff_stride;
   bool layer_major;      // backward goes layer by layer over runs of steps, with that product batched over time
   bool weights_resident; // all weight matrices together stay in L2
   size_t rows_ev;        // event words of a run of recomputed steps (refwd_rows_kernel), then the raw words
@@ -126,7 +128,8 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     for (int l = 1; l <= L; ++l) { wbytes += 4 * ((size_t)sz[l - 1] * sz[l] + (size_t)sz[l] * sz[l]); maxN = std::max(maxN, sz[l]); }
     lo.weights_resident = wbytes <= ((size_t)96 << 20);
     lo.layer_major = L > 1 && !lo.weights_resident;
-    lo.gff = L > 1 ? take(4 * (size_t)BWD_RUN * B * maxN) : 0;
+    lo.gff_stride = (size_t)BWD_RUN * B * maxN;
+    lo.gff = L > 1 ? take(4 * lo.gff_stride * TCG_MAX_KSPLIT) : 0;
   }
   lo.rows_ev = 0; lo.rows_ev_words = 0; lo.rows_ev_stride = 0;
   if (!graded && ck->strategy != SNN_STANDARD) {
@@ -866,6 +869,7 @@ struct Exec {
       // Runs of at most BWD_RUN steps, latest first; within a run the layers go from the last to the first:
       // the feed-forward term of layer l for the whole run is one product (ff_gemm_kernel), then the steps
       // of layer l follow one launch each.
+      int gff_parts = 1;   // partial products the feed-forward term of the current layer and run consists of
       for (int hi = n; hi > 0; hi -= BWD_RUN) {
         const int lo_s = std::max(0, hi - BWD_RUN);     // steps t0+lo_s+1 .. t0+hi
         for (int l = L; l >= 1; --l) {
@@ -874,6 +878,7 @@ struct Exec {
             span = begin_span(SNN_PHASE_FFGEMM);
             const int n_run = hi - lo_s;
             bool on_tcgen05 = false;
+            gff_parts = 1;
             if (!(a->flags & SNN_FLAG_FF_PRODUCT_MMA_SYNC) && B <= TCG_NMAX) {
               // tcgen05 path: 128 rows of W x up to 128 pairs per CTA, accumulator in tensor memory
               TcGemmParams tp;
@@ -881,6 +886,12 @@ struct Exec {
               tp.steps_per_tile = std::min(n_run, TCG_NMAX / B);
               tp.n_cols = (tp.steps_per_tile * B + 15) / 16 * 16;
               tp.out = at<float>(lo.gff); tp.status = at<uint32_t>(lo.status);
+              // few row tiles: the contraction range is cut into slices so that most SMs get a CTA; a function of
+              // the layer width alone (partial products are added in slice order by the step kernel)
+              const int row_tiles = (sz[l] + TCG_M - 1) / TCG_M;
+              tp.k_split = std::max(1, std::min({TCG_MAX_KSPLIT, 148 / row_tiles, (sz[l + 1] + TCG_KB - 1) / TCG_KB}));
+              tp.out_stride = lo.gff_stride;
+              gff_parts = tp.k_split;
               tp.N = sz[l]; tp.K = sz[l + 1]; tp.B = B; tp.n_steps = n_run;
               if (!ffw_map_ready[l]) {
                 ffw_map_ready[l] = make_tensor_map_2d(&ffw_map[l], a->W_ff[l], (uint64_t)sz[l], (uint64_t)sz[l + 1],
@@ -892,7 +903,7 @@ struct Exec {
                 tp.map_w = ffw_map[l];
                 CUDA_TRY(launch_pdl(ff_gemm_tc_kernel,
                                     dim3((unsigned)((n_run + tp.steps_per_tile - 1) / tp.steps_per_tile),
-                                         (unsigned)((sz[l] + TCG_M - 1) / TCG_M)),
+                                         (unsigned)row_tiles, (unsigned)tp.k_split),
                                     dim3(TCG_THREADS), TCG_SMEM_BYTES, tp));
                 on_tcgen05 = true;
               }
@@ -921,6 +932,7 @@ struct Exec {
             sp.W_rec = a->W_rec[l - 1];
             sp.g_out = l == L ? at<float>(lo.g_out) : nullptr;
             sp.g_ff = l < L ? at<float>(lo.gff) : nullptr;
+            sp.g_ff_parts = gff_parts; sp.g_ff_stride = lo.gff_stride;
             sp.d_first = op.t0 + hi == op.t1 ? carry(carry_cur, l) : slot(op.buf_slot + hi, l);
             sp.carry_out = lo_s == 0 ? carry(carry_cur ^ 1, l) : nullptr;
             sp.slots = at<float>(lo.slots); sp.slot_stride = lo.state_bytes / 4; sp.state_off = lo.layer_off[l];
@@ -947,6 +959,7 @@ struct Exec {
             f.d_next = t == op.t1 ? carry(carry_cur, l) : slot(op.buf_slot + ts + 1, l);
             f.g_out = l == L ? at<float>(lo.g_out) : nullptr;
             f.g_ff = l < L ? at<float>(lo.gff) + (size_t)(ts - lo_s) * B * sz[l] : nullptr;
+            f.g_ff_parts = gff_parts; f.g_ff_stride = lo.gff_stride;
             f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
             cudaError_t le;
             if (B <= 8) le = launch_bwd<1, 8>(p, tiles_l, CS_l, 1);

@@ -31,6 +31,7 @@ constexpr int TCG_NMAX = 128;     // pairs per CTA at most (columns of an accumu
 constexpr int TCG_TMEM_COLS = 512;   // three accumulators of 128 columns; allocations are powers of two
 constexpr int TCG_KB = 32;        // contraction values per k-block: one 128-byte swizzle row of fp32
 constexpr int TCG_STAGES = 3;
+constexpr int TCG_MAX_KSPLIT = 4; // slices of the contraction range at most (layers with few row tiles)
 constexpr int TCG_CONV_WARPS = 8;
 constexpr int TCG_THREADS = 32 * (2 + TCG_CONV_WARPS);
 constexpr uint32_t TCG_A_BYTES = TCG_M * TCG_KB * 4;       // 16 KB
@@ -41,7 +42,9 @@ constexpr size_t TCG_SMEM_BYTES = 1024 + (size_t)TCG_STAGES * TCG_STAGE_BYTES + 
 struct TcGemmParams {
   CUtensorMap map_w;       // W [N][K] fp32, box 32 k x 128 rows, 128-byte swizzle
   CUtensorMap map_d;       // delta of the run as [n_steps][B][K], box 32 k x B samples x steps_per_tile steps
-  float* out;              // [n_steps * B][N]
+  float* out;              // [k_split][n_steps * B][N]: one partial product per slice of the contraction range
+  size_t out_stride;       // floats between the partial products
+  int k_split;             // slices of the contraction range (whole k-blocks each); blockIdx.z selects one
   uint32_t* status;
   int N, K, B, n_steps;
   int steps_per_tile;      // steps whose pairs form one tile: steps_per_tile * B <= 128
@@ -123,7 +126,10 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
   uint32_t* const s_tmem = reinterpret_cast<uint32_t*>(bars + 3 * TCG_STAGES + 1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int row0 = blockIdx.y * TCG_M, ts0 = blockIdx.x * p.steps_per_tile;
-  const int n_kb = (p.K + TCG_KB - 1) / TCG_KB;
+  // this CTA's slice of the contraction range, in k-blocks [kb0, kb0 + n_kb)
+  const int n_kb_all = (p.K + TCG_KB - 1) / TCG_KB;
+  const int kb0 = (int)((long long)n_kb_all * blockIdx.z / p.k_split);
+  const int n_kb = (int)((long long)n_kb_all * (blockIdx.z + 1) / p.k_split) - kb0;
   auto stage_a_hi = [&](int s) { return s_base + (size_t)s * TCG_STAGE_BYTES; };
   auto stage_a_lo = [&](int s) { return s_base + (size_t)s * TCG_STAGE_BYTES + TCG_A_BYTES; };
   auto stage_b_hi = [&](int s) { return s_base + (size_t)s * TCG_STAGE_BYTES + 2 * TCG_A_BYTES; };
@@ -159,8 +165,8 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
           break;
         }
         mbar_arrive_expect_tx(bar_landed + s, tx_bytes);
-        tma_load_2d(stage_a_hi(s), &p.map_w, kb * TCG_KB, row0, bar_landed + s);
-        tma_load_3d(stage_b_hi(s), &p.map_d, kb * TCG_KB, 0, ts0, bar_landed + s);
+        tma_load_2d(stage_a_hi(s), &p.map_w, (kb0 + kb) * TCG_KB, row0, bar_landed + s);
+        tma_load_3d(stage_b_hi(s), &p.map_d, (kb0 + kb) * TCG_KB, 0, ts0, bar_landed + s);
       }
     }
   } else if (warp == 1) {
@@ -230,7 +236,7 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
         const int q = warp & 3;
         const int i = row0 + 32 * q + lane;
         const int pairs_here = min(p.steps_per_tile, p.n_steps - ts0) * p.B;   // valid columns of this tile
-        float* const dst = p.out + (size_t)ts0 * p.B * p.N + i;
+        float* const dst = p.out + (size_t)blockIdx.z * p.out_stride + (size_t)ts0 * p.B * p.N + i;
         for (int c0 = 0; c0 < p.n_cols; c0 += 32) {
           uint32_t small[32], even[32], odd[32];
           const uint32_t at = tmem_acc + ((uint32_t)(32 * q) << 16) + (uint32_t)c0;
