@@ -167,6 +167,13 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
  * memory).  This flag selects the older mma.sync kernel instead; the two agree to rounding (both are three-pass
  * tf32 products with fp32 accumulation), not bit for bit. */
 #define SNN_FLAG_FF_PRODUCT_MMA_SYNC 1024u
+/* The paper keeps the sparse activations of the whole sequence in local memory (Discussion).  With this flag
+ * (REMOTE and DOUBLE only; ignored otherwise) the device holds the events of two remote segments at a time (chunk_size
+ * steps for REMOTE, remote_chunk_size for DOUBLE): each segment's events are copied to the pinned workspace on the side
+ * stream behind the forward pass and fetched one segment ahead of the backward pass, ordered with events like the
+ * state checkpoints.  max_activity then bounds the mean activity per segment.  snn_workspace_query_flags reports the
+ * sizes; snn_get_event_layout is not available for such a step.  Gradients are bit-identical to the unspilled step. */
+#define SNN_FLAG_SPILL_EVENTS 2048u
 
 typedef struct {
   int32_t T, B;
@@ -235,7 +242,9 @@ typedef struct {
   int32_t remote_state_slots; /* dense states held in pinned memory               */
   int32_t d2h_copies, h2d_copies; /* checkpoint transfers of the last step        */
   int32_t kernel_launches;    /* kernels launched by the last step                */
-  size_t event_bytes;         /* event pools + spike masks (scale with T)         */
+  size_t event_bytes;         /* event pools + spike masks held on the device (scale with T, or with the
+                                 remote segment under SNN_FLAG_SPILL_EVENTS)      */
+  int32_t event_window_copies; /* event-window transfers of the last step (SNN_FLAG_SPILL_EVENTS) */
 } snn_memory_stats;
 snn_status snn_memory_stats_get(const snn_net* net, snn_memory_stats* out);
 

@@ -27,6 +27,7 @@ SNN_FLAG_FORWARD_STREAM_WEIGHTS = 128
 SNN_FLAG_BACKWARD_PER_STEP = 256
 SNN_FLAG_REFORWARD_ROWS = 512
 SNN_FLAG_FF_PRODUCT_MMA_SYNC = 1024
+SNN_FLAG_SPILL_EVENTS = 2048
 PHASE_NAMES = ["fwd", "refwd1", "refwd2", "bwd", "dw", "readout", "d2h", "h2d", "ffgemm"]
 SNN_OP_FWD, SNN_OP_REFWD1, SNN_OP_REFWD2, SNN_OP_BWD, SNN_OP_D2H, SNN_OP_H2D, SNN_OP_ZERO = range(7)
 STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "remote", SNN_DOUBLE: "double",
@@ -62,7 +63,7 @@ class snn_step_args(C.Structure):
 class snn_memory_stats(C.Structure):
     _fields_ = [("state_bytes", C.c_size_t), ("local_state_slots", C.c_int32), ("remote_state_slots", C.c_int32),
                 ("d2h_copies", C.c_int32), ("h2d_copies", C.c_int32), ("kernel_launches", C.c_int32),
-                ("event_bytes", C.c_size_t)]
+                ("event_bytes", C.c_size_t), ("event_window_copies", C.c_int32)]
 
 
 class snn_phase_times(C.Structure):

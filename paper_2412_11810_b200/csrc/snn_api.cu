@@ -62,6 +62,10 @@ struct Layout {
   int words[MAXL + 1];
   size_t slots, state_bytes, layer_off[MAXL + 1];  // layer_off in floats within a state
   size_t event_bytes, total;
+  bool spill;              // event windows per remote segment, the rest in pinned memory
+  int ev_steps;            // steps per event window (the whole sequence without spilling)
+  int ev_segments;         // windows the sequence consists of
+  size_t ev_base, ev_window_bytes;
   size_t gff;            // [BWD_RUN * B][max N] product W_ff delta of the layer above for a run of steps (large nets),
                          // as up to TCG_MAX_KSPLIT partial products gff_stride floats apart
   size_t gff_stride;
@@ -106,20 +110,33 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.in_stage = host_input ? take(4 * (size_t)T * B * (graded ? sz[0] : lo.words[0])) : 0;
   lo.in_words = graded ? take(4 * (size_t)T * B * lo.words[0]) : 0;
   lo.tg_stage = host_input ? take(4 * (size_t)B) : 0;
+  // Events (index lists, their offsets, spike words; values for the graded cell).  Normally the events of the whole
+  // sequence stay in device memory.  With SNN_FLAG_SPILL_EVENTS (REMOTE, DOUBLE) the device holds two windows of
+  // one remote segment each (the one in use and the one being copied), and every segment's window goes to pinned
+  // memory behind the forward pass and comes back ahead of its backward pass.  Within a window rows are indexed by
+  // the step relative to the segment's first state and list offsets restart at zero.
+  lo.spill = (flags & SNN_FLAG_SPILL_EVENTS) && (ck->strategy == SNN_REMOTE || ck->strategy == SNN_DOUBLE);
+  lo.ev_steps = T;
+  if (lo.spill) lo.ev_steps = std::min(T, ck->strategy == SNN_DOUBLE ? ck->remote_chunk_size : ck->chunk_size);
+  lo.ev_segments = (T + lo.ev_steps - 1) / lo.ev_steps;
+  const int Tw = lo.ev_steps;
   const size_t ev0 = cur;
   for (int l = 0; l <= L; ++l) {
     lo.words[l] = (sz[l] + 31) / 32;
-    const double want = std::ceil((double)max_activity * sz[l] * T) + sz[l];
+    const double want = std::ceil((double)max_activity * sz[l] * Tw) + sz[l];
     if (want > 4.0e9) { why = "event pool per sample exceeds 32-bit offsets"; return false; }
     lo.cap[l] = (uint32_t)want;
-    lo.off[l] = take(4 * (size_t)(T + 2) * B);
+    lo.off[l] = take(4 * (size_t)(Tw + 2) * B);
     lo.pool[l] = take(4 * (size_t)B * lo.cap[l]);
-    lo.mask[l] = l == 0 ? 0 : take(4 * (size_t)(T + 1) * B * lo.words[l]);
+    lo.mask[l] = l == 0 ? 0 : take(4 * (size_t)(Tw + 1) * B * lo.words[l]);
     lo.vals[l] = graded ? take(4 * (size_t)B * lo.cap[l]) : 0;
-    lo.pref[l] = graded ? take(2 * (size_t)(T + 2) * B * lo.words[l]) : 0;
-    lo.act[l] = (graded && l > 0) ? take(4 * (size_t)2 * B * sz[l]) : 0;
+    lo.pref[l] = graded ? take(2 * (size_t)(Tw + 2) * B * lo.words[l]) : 0;
   }
+  lo.ev_base = ev0;
+  lo.ev_window_bytes = cur - ev0;
+  if (lo.spill) take(lo.ev_window_bytes);   // the second window
   lo.event_bytes = cur - ev0;
+  for (int l = 0; l <= L; ++l) lo.act[l] = (graded && l > 0) ? take(4 * (size_t)2 * B * sz[l]) : 0;
   {
     // Networks whose weights do not stay in L2: streaming W_ff once per run of steps instead of once per
     // step pays for giving up the layer wavefront in the backward pass.  A function of the sizes only.
@@ -210,7 +227,8 @@ extern "C" snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, i
   if (!compute_layout(net, T, B, ckpt, max_activity, flags, lo, why))
     return fail(const_cast<snn_net*>(net), SNN_ERR_INVALID_ARG, "%s", why.c_str());
   if (device_bytes) *device_bytes = lo.total;
-  if (pinned_bytes) *pinned_bytes = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
+  if (pinned_bytes) *pinned_bytes = (lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes) +
+                                    (lo.spill ? (size_t)lo.ev_segments * lo.ev_window_bytes : 0);
   return SNN_OK;
 }
 
@@ -311,12 +329,80 @@ struct Exec {
   const float* in_dense(int t) const {   // graded input values at step t
     return reinterpret_cast<const float*>(in_base()) + (size_t)(t - 1) * B * net->sizes[0];
   }
-  float* vals(int l) const { return at<float>(lo.vals[l]); }
-  uint16_t* pref(int l, int t) const { return at<uint16_t>(lo.pref[l]) + (size_t)t * B * lo.words[l]; }
+  // Event arrays of the window in use: rows are addressed by the absolute step t, which must lie within the
+  // window's segment, [ev_r0, ev_r0 + ev_steps + 1]; kernels that index by step get a base shifted accordingly.
+  int ev_seg = 0, ev_r0 = 0;       // segment whose window the accessors address, and its first state
+  size_t ev_shift = 0;             // byte offset of that window from the first one
+  float* vals(int l) const { return at<float>(lo.vals[l] + ev_shift); }
+  uint16_t* pref(int l, int t) const { return at<uint16_t>(lo.pref[l] + ev_shift) + ((ptrdiff_t)t - ev_r0) * B * lo.words[l]; }
   float* act(int l, int parity) const { return at<float>(lo.act[l]) + (size_t)parity * B * net->sizes[l]; }
-  uint32_t* mask(int l, int t) const { return at<uint32_t>(lo.mask[l]) + (size_t)t * B * lo.words[l]; }
-  uint32_t* off(int l, int t) const { return at<uint32_t>(lo.off[l]) + (size_t)t * B; }
-  uint32_t* pool(int l) const { return at<uint32_t>(lo.pool[l]); }
+  uint32_t* mask(int l, int t) const { return at<uint32_t>(lo.mask[l] + ev_shift) + ((ptrdiff_t)t - ev_r0) * B * lo.words[l]; }
+  uint32_t* off(int l, int t) const { return at<uint32_t>(lo.off[l] + ev_shift) + ((ptrdiff_t)t - ev_r0) * B; }
+  uint32_t* pool(int l) const { return at<uint32_t>(lo.pool[l] + ev_shift); }
+
+  // ---- event windows (SNN_FLAG_SPILL_EVENTS)
+  int ev_resident[2] = {0, -1};    // segment each window holds
+  int ev_copy_event[2] = {-1, -1}; // copy event (index into net->copy_events, from the end) the window still waits on
+  cudaEvent_t ev_events[2] = {nullptr, nullptr};
+  bool ev_pending[2] = {false, false};
+  char* ev_host(int seg) const {
+    return static_cast<char*>(a->pinned_ws) + (lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes) +
+           (size_t)seg * lo.ev_window_bytes;
+  }
+  void ev_select(int seg) {
+    ev_seg = seg; ev_r0 = seg * lo.ev_steps; ev_shift = (size_t)(seg & 1) * lo.ev_window_bytes;
+    rows_params_ready = false;
+  }
+  // The main stream waits for the copy that last touched window w, if one is pending.
+  snn_status ev_wait(int w) {
+    if (ev_pending[w]) { CUDA_TRY(cudaStreamWaitEvent(main, ev_events[w], 0)); ev_pending[w] = false; }
+    return SNN_OK;
+  }
+  // A copy of window w on the side stream, after everything issued so far on the main stream.
+  snn_status ev_copy(int w, int seg, bool to_host) {
+    if (!ev_events[w]) CUDA_TRY(cudaEventCreateWithFlags(&ev_events[w], cudaEventDisableTiming));
+    CUDA_TRY(cudaEventRecord(net->ev_main, main));
+    CUDA_TRY(cudaStreamWaitEvent(side, net->ev_main, 0));
+    char* dev = ws + lo.ev_base + (size_t)w * lo.ev_window_bytes;
+    const int span = begin_span(to_host ? SNN_PHASE_D2H : SNN_PHASE_H2D, side);
+    if (to_host) CUDA_TRY(cudaMemcpyAsync(ev_host(seg), dev, lo.ev_window_bytes, cudaMemcpyDeviceToHost, side));
+    else CUDA_TRY(cudaMemcpyAsync(dev, ev_host(seg), lo.ev_window_bytes, cudaMemcpyHostToDevice, side));
+    end_span(span, side);
+    CUDA_TRY(cudaEventRecord(ev_events[w], side));
+    ev_pending[w] = true;
+    ++ev_copies;
+    return SNN_OK;
+  }
+  int ev_copies = 0;
+  // Forward pass enters segment seg (> 0): its window is free once the segment before the previous one has been
+  // written out; the spike words of the boundary state come over from the previous window, list offsets restart.
+  snn_status ev_enter_forward(int seg) {
+    const int w = seg & 1, r0 = seg * lo.ev_steps;
+    if (ev_wait(w) != SNN_OK) return SNN_ERR_CUDA;
+    for (int l = 1; l <= L; ++l) {
+      const uint32_t* src = mask(l, r0);   // still the previous segment's window: its last row
+      uint32_t* dst = at<uint32_t>(lo.mask[l] + (size_t)w * lo.ev_window_bytes);
+      CUDA_TRY(cudaMemcpyAsync(dst, src, 4 * (size_t)B * lo.words[l], cudaMemcpyDeviceToDevice, main));
+    }
+    for (int l = 0; l <= L; ++l)
+      CUDA_TRY(cudaMemsetAsync(ws + lo.off[l] + (size_t)w * lo.ev_window_bytes, 0, 4 * (size_t)2 * B, main));
+    ev_select(seg);
+    ev_resident[w] = seg;
+    return SNN_OK;
+  }
+  // Backward pass enters segment seg: its window must have arrived; the window of the segment after it is done
+  // with and receives the segment before it.
+  snn_status ev_enter_backward(int seg) {
+    const int w = seg & 1;
+    if (ev_resident[w] != seg) return fail(net, SNN_ERR_CUDA, "event window of segment %d is not resident", seg);
+    if (ev_wait(w) != SNN_OK) return SNN_ERR_CUDA;
+    ev_select(seg);
+    if (seg >= 1 && ev_resident[w ^ 1] != seg - 1) {
+      if (ev_wait(w ^ 1) != SNN_OK || ev_copy(w ^ 1, seg - 1, false) != SNN_OK) return SNN_ERR_CUDA;
+      ev_resident[w ^ 1] = seg - 1;
+    }
+    return SNN_OK;
+  }
 
   // The main stream waits for the checkpoint copy that last touched local slot s, if one is pending.
   snn_status wait_slot(int s) {
@@ -680,16 +766,16 @@ struct Exec {
     return SNN_OK;
   }
 
-  // After the last forward step: store the event lists of the final spikes.
-  snn_status run_flush() {
+  // After the last forward step (of the sequence, or of an event window): store the event lists of its spikes.
+  snn_status run_flush(int t_end) {
     FwdParams p;
     std::memset(&p, 0, sizeof p);
     p.B = B; p.alpha = net->alpha; p.theta = net->theta; p.status = at<uint32_t>(lo.status);
     for (int l = 1; l <= L; ++l) {
       FwdLayer& f = p.lay[l - 1];
       f.mode = 2; f.N = net->sizes[l]; f.W = lo.words[l];
-      f.rec_mask = mask(l, T); f.rec_pool = pool(l); f.rec_off = off(l, T); f.rec_cap = lo.cap[l];
-      if (graded()) { f.rec_val_src = act(l, T & 1); f.rec_vals = vals(l); f.rec_pref = pref(l, T); }
+      f.rec_mask = mask(l, t_end); f.rec_pool = pool(l); f.rec_off = off(l, t_end); f.rec_cap = lo.cap[l];
+      if (graded()) { f.rec_val_src = act(l, t_end & 1); f.rec_vals = vals(l); f.rec_pref = pref(l, t_end); }
     }
     return launch_fwd(p, true);
   }
@@ -1148,7 +1234,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   if (!compute_layout(net, T, B, &a->ckpt, a->max_activity, a->flags, ex.lo, why))
     return fail(net, SNN_ERR_INVALID_ARG, "%s", why.c_str());
   const Layout& lo = ex.lo;
-  const size_t pinned_need = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
+  const size_t pinned_states = lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes;
+  const size_t pinned_need = pinned_states + (lo.spill ? (size_t)lo.ev_segments * lo.ev_window_bytes : 0);
   if (a->device_ws_bytes < lo.total)
     return fail(net, SNN_ERR_WORKSPACE_TOO_SMALL, "device workspace %zu < %zu bytes", a->device_ws_bytes, lo.total);
   if (pinned_need > 0 && (!a->pinned_ws || a->pinned_ws_bytes < pinned_need))
@@ -1227,20 +1314,23 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
         if (st == SNN_OK)
           CUDA_TRY(cudaMemsetAsync(ex.ws + lo.slots + (size_t)op.keep_slot * lo.state_bytes, 0, lo.state_bytes, ms));
         break;
-      case SNN_OP_FWD:
-        st = ex.run_forward(op, true);
-        if (st == SNN_OK && i == last_fwd) {
-          st = ex.run_flush();
-          if (st == SNN_OK) st = ex.run_readout();
-        }
+      case SNN_OP_FWD: {
+        const int seg = op.t0 / lo.ev_steps;
+        if (lo.spill && seg != ex.ev_seg) st = ex.ev_enter_forward(seg);
+        if (st == SNN_OK) st = ex.run_forward(op, true);
+        if (st == SNN_OK && (i == last_fwd || lo.spill)) st = ex.run_flush(op.t1);
+        if (st == SNN_OK && lo.spill && i != last_fwd) st = ex.ev_copy(seg & 1, seg, true);   // behind the forward pass
+        if (st == SNN_OK && i == last_fwd) st = ex.run_readout();
         break;
+      }
       case SNN_OP_REFWD1:
       case SNN_OP_REFWD2:
-        st = ex.run_forward(op, false);
+      case SNN_OP_BWD: {
+        const int seg = op.t0 / lo.ev_steps;
+        if (lo.spill && seg != ex.ev_seg) st = ex.ev_enter_backward(seg);
+        if (st == SNN_OK) st = op.kind == SNN_OP_BWD ? ex.run_backward(op) : ex.run_forward(op, false);
         break;
-      case SNN_OP_BWD:
-        st = ex.run_backward(op);
-        break;
+      }
       case SNN_OP_D2H:
       case SNN_OP_H2D:
         st = ex.run_copy(op);
@@ -1256,6 +1346,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   // ---- finish: everything on both streams, then status and loss
   cudaError_t e1 = cudaStreamSynchronize(ex.side);
   cudaError_t e2 = cudaStreamSynchronize(ex.main);
+  for (cudaEvent_t& e : ex.ev_events)
+    if (e) { cudaEventDestroy(e); e = nullptr; }
   if (st != SNN_OK) return st;
   if (e1 != cudaSuccess || e2 != cudaSuccess)
     return fail(net, SNN_ERR_CUDA, "stream synchronize failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
@@ -1266,6 +1358,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   if (a->flags & SNN_FLAG_TIME_PHASES) ex.collect_spans();
   net->dev_peak = lo.total;
   net->pin_peak = pinned_need;
+  (void)pinned_states;
   net->stats.state_bytes = lo.state_bytes;
   net->stats.local_state_slots = lo.n_local;
   net->stats.remote_state_slots = lo.n_remote;
@@ -1273,8 +1366,9 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   net->stats.h2d_copies = ex.h2d;
   net->stats.kernel_launches = ex.launches;
   net->stats.event_bytes = lo.event_bytes;
-  net->ev_layout.assign(L + 1, snn_event_layout{});
-  for (int l = 0; l <= L; ++l) {
+  net->stats.event_window_copies = ex.ev_copies;
+  net->ev_layout.assign(lo.spill ? 0 : L + 1, snn_event_layout{});   // spilled events are not all on the device
+  for (int l = 0; l <= L && !lo.spill; ++l) {
     snn_event_layout& e = net->ev_layout[l];
     e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = lo.vals[l]; e.pool_capacity = lo.cap[l];
     e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];

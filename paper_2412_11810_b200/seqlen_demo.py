@@ -8,6 +8,10 @@ DOUBLE at a multiple of that length under the same cap, and prints one JSON line
 per sample-timestep, the peak bytes and the overhead.
 
     python paper_2412_11810_b200/seqlen_demo.py --workload c3 --cap-gib 2 --factor 10
+    python paper_2412_11810_b200/seqlen_demo.py --workload c3 --cap-gib 2 --factor 30 --spill
+
+With --spill the DOUBLE run keeps only two remote segments' events on the device (SNN_FLAG_SPILL_EVENTS); the events of
+the other segments wait in pinned host memory, so the device workspace no longer grows with the sequence.
 """
 from __future__ import annotations
 
@@ -41,6 +45,7 @@ def main():
     ap.add_argument("--max-activity", type=float, default=0.06)
     ap.add_argument("--remote-chunk", type=int, default=256)
     ap.add_argument("--chunk", type=int, default=16)
+    ap.add_argument("--spill", action="store_true", help="DOUBLE spills the events of finished remote segments to pinned memory")
     args = ap.parse_args()
 
     import torch
@@ -50,21 +55,24 @@ def main():
     cap = int(args.cap_gib * (1 << 30))
     net = sb.snn_create(list(base.sizes), base.tau_mem, base.theta, cell=base.cell)
 
-    def fits(ck):
+    dbl_flags = sb.SNN_FLAG_SPILL_EVENTS if args.spill else 0
+
+    def fits(ck, flags=0):
         def f(T):
             try:
-                return sb.snn_workspace_query(net, T, base.B, ck, args.max_activity)[0] <= cap
+                return sb.snn_workspace_query(net, T, base.B, ck, args.max_activity, flags)[0] <= cap
             except sb.SnnError:
                 return False
         return f
 
     T_std = longest(fits(sb.snn_ckpt(sb.SNN_STANDARD, 0, 0)))
-    T_dbl_max = longest(fits(sb.snn_ckpt(sb.SNN_DOUBLE, args.chunk, args.remote_chunk)))
+    T_dbl_max = longest(fits(sb.snn_ckpt(sb.SNN_DOUBLE, args.chunk, args.remote_chunk), dbl_flags))
     sb.snn_destroy(net)
     T_dbl = args.factor * T_std
     out = {"workload": base.name, "sizes": list(base.sizes), "B": base.B, "cap_bytes": cap,
            "max_activity": args.max_activity, "T_standard_max": T_std, "T_double": T_dbl,
-           "T_double_max_under_cap": T_dbl_max, "chunk_size": args.chunk, "remote_chunk_size": args.remote_chunk}
+           "T_double_max_under_cap": T_dbl_max, "chunk_size": args.chunk, "remote_chunk_size": args.remote_chunk,
+           "events_spilled": bool(args.spill)}
     if T_dbl > T_dbl_max:
         out["error"] = "DOUBLE does not fit the requested multiple under the cap"
         print(json.dumps(out))
@@ -82,7 +90,8 @@ def main():
         x = torch.from_numpy(np.ascontiguousarray(x_all[:T])).to(s.device)
         s.device_ws = None                            # a fresh workspace of exactly the queried size
         torch.cuda.empty_cache()
-        kw = dict(strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=args.max_activity)
+        kw = dict(strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=args.max_activity,
+                  extra_flags=dbl_flags if name == "double" else 0)
         s.train_step(x, targets, **kw)
         ms = []
         for _ in range(2):
@@ -99,7 +108,8 @@ def main():
         out[name] = {"T": T, "ms_per_step": min(ms), "ns_per_sample_timestep": 1e6 * min(ms) / (T * base.B),
                      "device_peak_bytes": dev, "pinned_peak_bytes": pin, "local_state_slots": st.local_state_slots,
                      "state_bytes": st.state_bytes, "event_bytes": st.event_bytes, "loss": loss,
-                     "d2h_copies": st.d2h_copies, "h2d_copies": st.h2d_copies}
+                     "d2h_copies": st.d2h_copies, "h2d_copies": st.h2d_copies,
+                     "event_window_copies": st.event_window_copies}
         del x
     out["sequence_length_ratio"] = T_dbl / T_std
     out["time_overhead_per_sample_timestep"] = (out["double"]["ns_per_sample_timestep"] /

@@ -350,6 +350,39 @@ def test_bad_targets_and_input_padding_bits_are_guarded(orc32):
     s.close()
 
 
+def test_events_spilled_to_host_memory(orc32):
+    """With SNN_FLAG_SPILL_EVENTS the device keeps the events of two remote segments only; the rest waits in
+    pinned memory.  Same bits as the step that keeps every event on the device, for REMOTE and DOUBLE, a last
+    segment that is short, every forward and recomputation path, the spiking and the graded cell; the device
+    workspace shrinks and the number of window transfers is 2 n - 3 for n segments."""
+    b = sb()
+    cases = [(wl.small(sizes=(40, 260, 132, 6), T=53, B=5, p_in=0.1, g_ff=(2.5, 1.6), seed=71), 0),
+             (_graded(sizes=(48, 264, 132, 9), T=45, B=4, seed=72), 0)]
+    for w, _ in cases:
+        d = wl.make(w)
+        s, bits, targets = make_session(w, d)
+        s.train_step(bits, targets, strategy=0, max_activity=1.0)
+        assert_grads_close(s.gradients(), run_oracle(orc32, w, d))
+        base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+        for strat, K, R in [(2, 7, 0), (3, 3, 12), (3, 4, 8), (2, 60, 0)]:
+            E = R if strat == 3 else K
+            n_seg = -(-w.T // min(E, w.T))
+            for flags in (0, b.SNN_FLAG_FORWARD_PER_STEP | b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_FORWARD_STREAM_WEIGHTS,
+                          b.SNN_FLAG_REFORWARD_ROWS):
+                for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+                    g.fill_(float("nan"))
+                s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0,
+                             extra_flags=flags | b.SNN_FLAG_SPILL_EVENTS)
+                for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+                    assert np.array_equal(x, y), (w.cell, strat, K, R, flags)
+                assert s.stats().event_window_copies == max(0, 2 * n_seg - 3)
+        ck = s.ckpt(3, 3, 12)
+        d_all, p_all = b.snn_workspace_query(s.net, w.T, w.B, ck, 1.0)
+        d_win, p_win = b.snn_workspace_query(s.net, w.T, w.B, ck, 1.0, b.SNN_FLAG_SPILL_EVENTS)
+        assert d_win < d_all and p_win > p_all
+        s.close()
+
+
 # ---------------------------------------------------------------- graded (thresholded-ReLU) cell
 def _graded(**kw):
     a = dict(cell=wl.CELL_GRADED, theta=0.3, g_ff=(1.2, 0.8), g_rec=(0.3, 0.3), p_in=0.3)
