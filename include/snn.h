@@ -174,6 +174,13 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
  * state checkpoints.  max_activity then bounds the mean activity per segment.  snn_workspace_query_flags reports the
  * sizes; snn_get_event_layout is not available for such a step.  Gradients are bit-identical to the unspilled step. */
 #define SNN_FLAG_SPILL_EVENTS 2048u
+/* Event-driven backward pass (an extension in the spirit of the paper's Discussion: exploit the sparse activations).
+ * With SNN_SURR_TRIANGLE the pseudo-derivative is zero unless |V - threshold| < 1 / beta, so only the rows of W_rec and
+ * W_ff of near-threshold (sample, neuron) pairs are read and multiplied; everywhere else delta_t = alpha delta_{t+1}.
+ * Pays when batch x fraction of near-threshold neurons is well below one; otherwise the dense tensor-core kernels,
+ * which read every row once for the whole batch, are faster.  SNN_ERR_UNSUPPORTED for other surrogates or the graded
+ * cell.  Gradients are bit-identical across strategies under this flag, and agree with the dense orders to rounding. */
+#define SNN_FLAG_BACKWARD_EVENT_DRIVEN 4096u
 
 typedef struct {
   int32_t T, B;

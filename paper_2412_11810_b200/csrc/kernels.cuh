@@ -1787,6 +1787,100 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_step_kerne
 }
 
 // ------------------------------------------------------------------------------------------
+// Event-driven backward step for a pseudo-derivative with compact support (SNN_SURR_TRIANGLE, LIF cell).
+//
+// sigma'(V - theta) = beta max(0, 1 - beta |V - theta|) is exactly zero unless the membrane is within 1 / beta of
+// the threshold, and then delta_t = alpha delta_{t+1} needs no product at all.  Only for the near-threshold
+// (sample, neuron) pairs are row i of W_rec (and of W_ff of the layer above) multiplied with the deltas: the
+// backward pass reads the rows the activity selects, like the forward pass, instead of streaming every matrix
+// every step.  A warp owns 32 adjacent neurons of one sample and finds the near-threshold ones by ballot; the
+// eight warps of a CTA then share out the CTA's near-threshold neurons in turn and compute their dot products,
+// the 32 lanes striding over the contraction index (16-byte
+// loads; four accumulators per lane combined in a fixed order, then a fixed shuffle tree: the sum does not depend
+// on how the sequence is cut).  Launched as a layer wavefront like bwd_step_kernel (blockIdx.z = layer).
+constexpr int BEV_WARPS = 8;
+
+__device__ __forceinline__ float warp_dot(const float* __restrict__ w, const float* __restrict__ d, int n, int lane) {
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  int k = lane * 4;   // n is a multiple of 4
+  // eight 16-byte pieces of each operand in flight per lane; the order of the additions is that of the plain loop
+  for (; k + 7 * 128 < n; k += 8 * 128) {
+    float4 x[8], y[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      x[u] = ldg4_stream(w + k + u * 128);
+      y[u] = __ldcg(reinterpret_cast<const float4*>(d + k + u * 128));
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      a0 = fmaf(x[u].x, y[u].x, a0); a1 = fmaf(x[u].y, y[u].y, a1);
+      a2 = fmaf(x[u].z, y[u].z, a2); a3 = fmaf(x[u].w, y[u].w, a3);
+    }
+  }
+  for (; k < n; k += 128) {
+    const float4 x = ldg4_stream(w + k);
+    const float4 y = __ldcg(reinterpret_cast<const float4*>(d + k));
+    a0 = fmaf(x.x, y.x, a0); a1 = fmaf(x.y, y.y, a1); a2 = fmaf(x.z, y.z, a2); a3 = fmaf(x.w, y.w, a3);
+  }
+  float a = (a0 + a1) + (a2 + a3);
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) a += __shfl_xor_sync(0xffffffffu, a, s);
+  return a;
+}
+
+__global__ void __launch_bounds__(32 * BEV_WARPS) bwd_event_kernel(const __grid_constant__ BwdParams p) {
+  pdl_launch_dependents();
+  const BwdLayer& L = p.lay[blockIdx.z];
+  if (L.mode == 0) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int strips = (L.N + 31) / 32;   // per sample
+  const long long n_strips = (long long)strips * p.B, strip0 = (long long)blockIdx.x * BEV_WARPS;
+  if (strip0 >= n_strips) return;       // the whole CTA
+  __shared__ uint32_t s_near[BEV_WARPS];
+  __shared__ float s_sum[BEV_WARPS * 32];
+  const long long strip = strip0 + warp;
+  const bool live = strip < n_strips;
+  const int b = live ? (int)(strip / strips) : 0, i = live ? (int)(strip % strips) * 32 + lane : 0;
+  const bool ok = live && i < L.N;
+  pdl_wait();
+  const size_t k = (size_t)b * L.N + (ok ? i : 0);
+  const float v = ok ? L.V_delta[k] : 0.f;
+  const float dn = ok ? __ldcg(L.d_next + k) : 0.f;
+  const float u = fmaf(-p.beta, fabsf(v - p.theta), 1.f);
+  const float sp = ok && u > 0.f ? p.beta * u : 0.f;   // the same expression as surrogate_grad
+  const uint32_t near = __ballot_sync(0xffffffffu, sp != 0.f);
+  if (lane == 0) s_near[warp] = near;
+  __syncthreads();
+  // the near-threshold neurons of the CTA's strips, dealt out to its warps in turn (a strip may hold several)
+  int e = 0;
+  for (int ws = 0; ws < BEV_WARPS; ++ws) {
+    uint32_t bits = s_near[ws];
+    while (bits) {
+      const int j = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (e++ % BEV_WARPS != warp) continue;
+      const long long st = strip0 + ws;
+      const int bb = (int)(st / strips), row = (int)(st % strips) * 32 + j;
+      float sum = 0.f;
+      if (L.W_ffa) sum = warp_dot(L.W_ffa + (size_t)row * L.N_post, L.d_above + (size_t)bb * L.N_post, L.N_post, lane);
+      sum += warp_dot(L.W_rec + (size_t)row * L.N, L.d_next + (size_t)bb * L.N, L.N, lane);
+      if (lane == 0) s_sum[ws * 32 + j] = sum;
+    }
+  }
+  __syncthreads();
+  if (ok) {
+    float dl = p.alpha * dn;
+    if (sp != 0.f) {
+      float g = s_sum[warp * 32 + lane] + (L.g_out ? L.g_out[k] : 0.f);
+      g = fmaf(-p.theta, dn, g);
+      dl = fmaf(g, sp, dl);
+    }
+    L.V_delta[k] = dl;
+    if (L.carry_out) L.carry_out[k] = dl;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Backward steps of ONE layer over a run of steps in one cooperative launch, the recurrent matrix streaming
 // from HBM without a pause (networks whose weights exceed L2: the layer-by-layer order).
 //

@@ -939,10 +939,12 @@ struct Exec {
     int CS = 1;
     while (CS < 8 && tiles * L * CS * 2 <= wave && minN / (4 * CS * 2) >= 32) CS *= 2;
     int span = begin_span(SNN_PHASE_BWD);
-    const bool layer_major = L > 1 && ((a->flags & SNN_FLAG_BACKWARD_LAYER_BY_LAYER) ||
+    // event-driven steps (compact-support surrogate): a layer wavefront, one launch per step
+    const bool event_driven = (a->flags & SNN_FLAG_BACKWARD_EVENT_DRIVEN) != 0;
+    const bool layer_major = !event_driven && L > 1 && ((a->flags & SNN_FLAG_BACKWARD_LAYER_BY_LAYER) ||
                                        (lo.layer_major && !(a->flags & SNN_FLAG_BACKWARD_WAVEFRONT)));
     bool segment_done = false;
-    if (!layer_major && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
+    if (!layer_major && !event_driven && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
       // small networks: the whole segment in one cooperative launch, the weights resident in shared memory
       snn_status st = SNN_OK;
       if (B <= 8) st = try_backward_segment<1, 8>(op, CS, segment_done);
@@ -1073,7 +1075,12 @@ struct Exec {
         f.carry_out = t == op.t0 + 1 ? carry(carry_cur ^ 1, l) : nullptr;
       }
       cudaError_t le;
-      if (B <= 8) le = launch_bwd<1, 8>(p, tiles, CS);
+      if (event_driven) {
+        const long long warps = (long long)((maxN + 31) / 32) * B;
+        le = launch_pdl(bwd_event_kernel, dim3((unsigned)((warps + BEV_WARPS - 1) / BEV_WARPS), 1, (unsigned)L),
+                        dim3(32 * BEV_WARPS), 0, p);
+      }
+      else if (B <= 8) le = launch_bwd<1, 8>(p, tiles, CS);
       else if (B <= 16) le = launch_bwd<2, 8>(p, tiles, CS);
       else le = launch_bwd<4, 16>(p, tiles, CS);
       if (le != cudaSuccess) return fail(net, SNN_ERR_CUDA, "backward launch failed: %s", cudaGetErrorString(le));
@@ -1225,6 +1232,8 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   if (net->cell == SNN_CELL_GRADED && a->input_format != SNN_INPUT_DENSE)
     return fail(net, SNN_ERR_UNSUPPORTED, "the graded cell takes dense fp32 input (SNN_INPUT_DENSE)");
   if (!(a->max_activity > 0.f) || a->max_activity > 1.f) return fail(net, SNN_ERR_INVALID_ARG, "max_activity not in (0, 1]");
+  if ((a->flags & SNN_FLAG_BACKWARD_EVENT_DRIVEN) && (net->surrogate != SNN_SURR_TRIANGLE || net->cell != SNN_CELL_LIF))
+    return fail(net, SNN_ERR_UNSUPPORTED, "the event-driven backward pass needs SNN_SURR_TRIANGLE and the LIF cell");
   if (reinterpret_cast<uintptr_t>(a->device_ws) % ALIGN != 0)
     return fail(net, SNN_ERR_INVALID_ARG, "device workspace must be 256-byte aligned");
 

@@ -107,13 +107,59 @@ def sweeps(base, quick):
     yield "hidden width (T = 1000)", "sizes", pts
 
 
+def event_backward_table(base, T=192, K=16):
+    """Dense against event-driven backward pass (SNN_SURR_TRIANGLE) on the network of `base`: per batch size and
+    surrogate width the fraction of near-threshold neurons and the time of the backward steps of one train step of
+    T steps (CHUNK, chunk size K), from the per-pass CUDA-event timers.  Prints a markdown table."""
+    import torch
+    from paper_2412_11810_b200 import Session, binding as sb
+
+    print(f"\n## event-driven against dense backward steps ({'-'.join(map(str, base.sizes))}, T = {T}, chunk {K}, triangle surrogate)\n")
+    print("| B | beta | near-threshold fraction per layer | dense: backward steps + feed-forward product ms | "
+          "event-driven: backward steps ms | ratio |")
+    print("|---|---|---|---|---|---|")
+    for B in (1, 8, 32):
+        w = replace(base, T=T, B=B, readout_scale=1.0 / T)
+        d = wl.make(w, dense_input=False)
+        x = torch.from_numpy(np.ascontiguousarray(d["input_bits"].view(np.int32))).cuda()
+        tg = torch.from_numpy(d["targets"]).cuda()
+        for beta in (3.0, 10.0):
+            s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate=sb.SNN_SURR_TRIANGLE,
+                        surrogate_beta=beta, readout_scale=w.scale())
+            s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+            s.train_step(x[:64], tg, strategy=0, forward_only=True, keep_V=True)
+            near = [float(((v[1:] - w.theta).abs() * beta < 1).float().mean()) for v in s.debug_V]
+            s.debug_V = None
+            res = {}
+            for name, flags in (("dense", 0), ("event", sb.SNN_FLAG_BACKWARD_EVENT_DRIVEN)):
+                kw = dict(strategy=1, chunk_size=K, extra_flags=flags)
+                s.train_step(x, tg, **kw)
+                best = None
+                for _ in range(2):
+                    s.train_step(x, tg, time_phases=True, **kw)
+                    ph = s.phase_times()
+                    ms = ph["bwd"][0] + ph["ffgemm"][0]
+                    best = ms if best is None else min(best, ms)
+                res[name] = best
+            print(f"| {B} | {beta:g} | {' / '.join(f'{100 * v:.1f} %' for v in near)} | {res['dense']:.1f} | "
+                  f"{res['event']:.1f} | {res['event'] / res['dense']:.2f} |", flush=True)
+            s.close()
+            del s
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="c2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--quick", action="store_true", help="a few points per sweep")
     ap.add_argument("--markdown", action="store_true", help="tables instead of JSON lines")
+    ap.add_argument("--event-backward", action="store_true",
+                    help="only the table of the event-driven against the dense backward pass (triangle surrogate)")
     args = ap.parse_args()
     base = wl.WORKLOADS[args.workload]
+    if args.event_backward:
+        event_backward_table(base)
+        return 0
     for name, key, pts in sweeps(base, args.quick):
         rows = [measure(**p) for p in pts]
         if not args.markdown:

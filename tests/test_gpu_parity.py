@@ -237,6 +237,45 @@ def test_triangle_surrogate(orc32):
     s.close()
 
 
+@pytest.mark.parametrize("beta", [3.0, 10.0])
+def test_event_driven_backward_pass(orc32, beta):
+    """With the compact-support pseudo-derivative the backward step needs the rows of W only for the (sample, neuron)
+    pairs within 1 / beta of the threshold: the event-driven kernel reads just those.  Against the oracle, against
+    the dense kernels (to rounding), bit-identical across strategies, widths that are no multiple of 32 or 128; and
+    refused for a surrogate without compact support."""
+    from oracle.oracle import SURR_TRIANGLE, NetSpec, leak_from_tau
+    from paper_2412_11810_b200 import Session
+    b = sb()
+    w = wl.small(sizes=(70, 700, 260, 132, 7), T=41, B=5, p_in=0.05, g_ff=(2.5, 1.4, 1.5), g_rec=(1.0, 1.0, 1.0), seed=73)
+    d = wl.make(w)
+    spec = NetSpec(w.sizes, leak_from_tau(w.tau_mem), w.theta, beta, w.scale(), surrogate=SURR_TRIANGLE)
+    ref = orc32.bptt_full(spec, d["input_dense"], d["targets"], d["W_ff"], d["W_rec"], d["W_out"])
+    near = [float((np.abs(v[1:] - w.theta) * beta < 1).mean()) for v in ref["V"]]
+    assert all(0.0 < x < 0.6 for x in near), near            # some, not all, neurons are near the threshold
+    assert all(np.abs(g).max() > 0 for g in ref["dW_rec"])
+    s = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate=b.SNN_SURR_TRIANGLE, surrogate_beta=beta,
+                readout_scale=w.scale())
+    s.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    f = b.SNN_FLAG_BACKWARD_EVENT_DRIVEN
+    s.train_step(d["input_bits"], d["targets"], strategy=0, max_activity=1.0, extra_flags=f)
+    assert_grads_close(s.gradients(), ref)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    for strat, K, R in [(1, 6, 0), (3, 4, 16), (2, 9, 0)]:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        s.train_step(d["input_bits"], d["targets"], strategy=strat, chunk_size=K, remote_chunk_size=R,
+                     max_activity=1.0, extra_flags=f)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R)
+    s.close()
+    s2 = Session(w.sizes, tau_mem=w.tau_mem, threshold=w.theta, surrogate_beta=beta, readout_scale=w.scale())
+    s2.set_weights(d["W_ff"], d["W_rec"], d["W_out"])
+    with pytest.raises(b.SnnError) as e:
+        s2.train_step(d["input_bits"], d["targets"], strategy=0, max_activity=1.0, extra_flags=f)
+    assert e.value.status == b.SNN_ERR_UNSUPPORTED
+    s2.close()
+
+
 def test_c1_gradients_all_strategies(orc32):
     w = wl.WORKLOADS["c1"]
     d = wl.make(w)
