@@ -44,7 +44,8 @@ typedef enum {
   SNN_ERR_EVENT_OVERFLOW = 3, /* more events than max_activity allows; gradients unspecified */
   SNN_ERR_DEVICE_TIMEOUT = 4,
   SNN_ERR_CUDA = 5,
-  SNN_ERR_UNSUPPORTED = 6
+  SNN_ERR_UNSUPPORTED = 6,
+  SNN_ERR_DEBUG_CHECK = 7 /* bounds-checked build only: an index check failed; nothing was accessed out of bounds */
 } snn_status;
 
 typedef enum { SNN_STANDARD = 0, SNN_CHUNK = 1, SNN_REMOTE = 2, SNN_DOUBLE = 3, SNN_HIERARCHICAL = 4,
@@ -89,6 +90,12 @@ void snn_destroy(snn_net* net);
 
 /* The leak alpha = exp(-1/tau_mem), evaluated in double and rounded once to fp32. */
 float snn_alpha(const snn_net* net);
+
+/* 1 if the library was compiled with -DSNN_DEBUG_CHECKS=1 (libsnnckpt_debug.so), else 0.  That build tests the
+ * data-dependent indices of the gather kernels (position in an event pool, presynaptic row of an event) and the state
+ * slots the executor addresses before use; a bad index is replaced by a valid one and the step returns
+ * SNN_ERR_DEBUG_CHECK.  Results of a correct step are bit-identical to the ordinary build. */
+int32_t snn_debug_checks_enabled(void);
 
 /* Checkpoint hyper-parameters (paper: chunk_size, Eq. 1; remote_chunk_size, Eq. 11; nb_local, Eq. 8).
  * STANDARD ignores all; CHUNK and REMOTE need chunk_size >= 1; DOUBLE and DOUBLE_LOCAL need

@@ -11,10 +11,11 @@ import os
 from typing import List, Optional, Sequence
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libsnnckpt.so")
+# SNN_DEBUG_CHECKS=1 in the environment selects the bounds-checked build of the same sources
+LIB_PATH = os.path.join(HERE, "libsnnckpt_debug.so" if os.environ.get("SNN_DEBUG_CHECKS") == "1" else "libsnnckpt.so")
 
 SNN_OK, SNN_ERR_INVALID_ARG, SNN_ERR_WORKSPACE_TOO_SMALL, SNN_ERR_EVENT_OVERFLOW = 0, 1, 2, 3
-SNN_ERR_DEVICE_TIMEOUT, SNN_ERR_CUDA, SNN_ERR_UNSUPPORTED = 4, 5, 6
+SNN_ERR_DEVICE_TIMEOUT, SNN_ERR_CUDA, SNN_ERR_UNSUPPORTED, SNN_ERR_DEBUG_CHECK = 4, 5, 6, 7
 SNN_STANDARD, SNN_CHUNK, SNN_REMOTE, SNN_DOUBLE, SNN_HIERARCHICAL, SNN_DOUBLE_LOCAL = 0, 1, 2, 3, 4, 5
 SNN_CELL_LIF, SNN_CELL_GRADED = 0, 1
 SNN_SURR_FAST_SIGMOID, SNN_SURR_SIGMOID, SNN_SURR_TRIANGLE = 0, 1, 2
@@ -36,7 +37,8 @@ STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "rem
 
 EXPORTS = ["snn_create", "snn_destroy", "snn_alpha", "snn_workspace_query", "snn_workspace_query_flags", "snn_train_step", "snn_peak_memory",
            "snn_memory_stats_get", "snn_last_error", "snn_plan", "snn_compact_spikes", "snn_get_event_layout",
-           "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt", "snn_selftest_wait_timeout"]
+           "snn_phase_times_get", "snn_train_step_static", "snn_suggest_ckpt", "snn_selftest_wait_timeout",
+           "snn_debug_checks_enabled"]
 SNN_STATIC_WORKSPACE_BYTES = 32 << 20
 
 
@@ -91,6 +93,8 @@ def _load() -> C.CDLL:
     lib.snn_destroy.restype = None
     lib.snn_alpha.argtypes = [C.c_void_p]
     lib.snn_alpha.restype = C.c_float
+    lib.snn_debug_checks_enabled.argtypes = []
+    lib.snn_debug_checks_enabled.restype = C.c_int32
     lib.snn_workspace_query.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(snn_ckpt), C.c_float,
                                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.snn_workspace_query_flags.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(snn_ckpt), C.c_float,

@@ -25,6 +25,21 @@ constexpr int MAX_WORDS = 2048;             // 65536 neurons / 32
 constexpr uint32_t STATUS_EVENT_OVERFLOW = 1u;
 constexpr uint32_t STATUS_SYNC_TIMEOUT = 2u;     // a bounded wait (on a counter or an mbarrier) ran out
 constexpr uint32_t STATUS_BAD_TARGET = 4u;   // a target outside [0, N_out)
+constexpr uint32_t STATUS_DEBUG_CHECK = 8u;  // an index check of the bounds-checked build (SNN_DEBUG_CHECKS) failed
+
+// Bounds-checked build (compiled with -DSNN_DEBUG_CHECKS=1): the data-dependent indices of the gather kernels -- a
+// position in an event pool, the presynaptic row an event names -- are tested before use; a bad one raises
+// STATUS_DEBUG_CHECK and is replaced by index 0, so that the access stays inside its array and the step ends with
+// SNN_ERR_DEBUG_CHECK instead of a memory fault.  In the ordinary build the function is the identity.
+__device__ __forceinline__ uint32_t checked_index(uint32_t idx, uint32_t limit, uint32_t* status) {
+#ifdef SNN_DEBUG_CHECKS
+  if (idx >= limit) {
+    atomicOr(status, STATUS_DEBUG_CHECK);
+    return 0u;
+  }
+#endif
+  return idx;
+}
 
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 
@@ -361,8 +376,9 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
     } else {
       for (int i = threadIdx.x; i < n; i += FWD_THREADS) {
         const uint32_t q = c0 + i;
-        s_row[i] = q < n_ff ? Wff_tile + (size_t)ff_pool[s_ff + q] * L.N
-                            : Wrec_tile + (size_t)rec_pool[s_rec + (q - n_ff)] * L.N;
+        s_row[i] = q < n_ff
+            ? Wff_tile + (size_t)checked_index(ff_pool[checked_index(s_ff + q, L.ff_cap, p.status)], L.N_pre, p.status) * L.N
+            : Wrec_tile + (size_t)checked_index(rec_pool[checked_index(s_rec + (q - n_ff), L.rec_cap, p.status)], L.N, p.status) * L.N;
         if (GRADED)
           s_val[i] = q < n_ff ? L.ff_vals[(size_t)b * L.ff_cap + s_ff + q]
                               : L.rec_vals[(size_t)b * L.rec_cap + s_rec + (q - n_ff)];
@@ -497,11 +513,12 @@ struct SegLayer {
   const float* rec_vals;      // graded cell: values that go with rec_pool
   size_t state_off;           // offset of this layer inside a state slot, in floats
   uint32_t ff_cap, rec_cap;
-  int N;
+  int N, N_pre;
 };
 
 struct SegParams {
   SegLayer lay[MAXL];
+  uint32_t* status;
   float* slots;               // state slot s starts at slots + s * slot_stride
   size_t slot_stride;         // floats
   int B;
@@ -540,8 +557,9 @@ __global__ void __launch_bounds__(FWD_THREADS, 4) refwd_gather_kernel(const __gr
     const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
     for (int i = tid; i < n; i += FWD_THREADS) {
       const uint32_t q = c0 + i;
-      s_row[i] = q < n_ff ? Wff_tile + (size_t)ff_pool[s_ff + q] * L.N
-                          : Wrec_tile + (size_t)rec_pool[s_rec + (q - n_ff)] * L.N;
+      s_row[i] = q < n_ff
+          ? Wff_tile + (size_t)checked_index(ff_pool[checked_index(s_ff + q, L.ff_cap, p.status)], L.N_pre, p.status) * L.N
+          : Wrec_tile + (size_t)checked_index(rec_pool[checked_index(s_rec + (q - n_ff), L.rec_cap, p.status)], L.N, p.status) * L.N;
       if (GRADED)
         s_val[i] = q < n_ff ? L.ff_vals[(size_t)b * L.ff_cap + s_ff + q]
                             : L.rec_vals[(size_t)b * L.rec_cap + s_rec + (q - n_ff)];

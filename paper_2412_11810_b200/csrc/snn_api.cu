@@ -10,6 +10,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/snn.h"
 #include "kernels.cuh"
 #include "tc_gemm.cuh"
@@ -37,6 +39,14 @@ struct snn_net {
 };
 
 namespace {
+
+// A named range on the profiler's timeline (NVTX; costs nothing while no tool is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 snn_status fail(snn_net* net, snn_status st, const char* fmt, ...) {
   if (net) {
@@ -211,6 +221,14 @@ extern "C" void snn_destroy(snn_net* net) {
 
 extern "C" float snn_alpha(const snn_net* net) { return net ? net->alpha : 0.f; }
 
+extern "C" int32_t snn_debug_checks_enabled(void) {
+#ifdef SNN_DEBUG_CHECKS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 extern "C" const char* snn_last_error(const snn_net* net) { return net ? net->err.c_str() : "null net"; }
 
 extern "C" snn_status snn_workspace_query(const snn_net* net, int32_t T, int32_t B, const snn_ckpt* ckpt,
@@ -318,7 +336,13 @@ struct Exec {
   }
 
   template <class Tp> Tp* at(size_t off) const { return reinterpret_cast<Tp*>(ws + off); }
-  float* slot(int s, int l) const { return at<float>(lo.slots + (size_t)s * lo.state_bytes) + lo.layer_off[l]; }
+  mutable bool debug_violation = false;   // bounds-checked build: the plan named a state slot the layout does not have
+  float* slot(int s, int l) const {
+#ifdef SNN_DEBUG_CHECKS
+    if (s < 0 || s >= lo.n_local) { debug_violation = true; s = 0; }
+#endif
+    return at<float>(lo.slots + (size_t)s * lo.state_bytes) + lo.layer_off[l];
+  }
   float* carry(int which, int l) const { return at<float>(lo.carry[which]) + lo.layer_off[l]; }
   bool graded() const { return net->cell == SNN_CELL_GRADED; }
   const void* in_base() const { return (a->flags & SNN_FLAG_INPUT_ON_HOST) ? (const void*)(ws + lo.in_stage) : a->input; }
@@ -560,8 +584,9 @@ struct Exec {
       s.rec_pool = pool(l); s.rec_off = off(l, 0); s.rec_cap = lo.cap[l];
       if (graded()) { s.ff_vals = vals(l - 1); s.rec_vals = vals(l); }
       s.state_off = lo.layer_off[l];
-      s.N = net->sizes[l];
+      s.N = net->sizes[l]; s.N_pre = net->sizes[l - 1];
     }
+    g.status = at<uint32_t>(lo.status);
     ScanParams c;
     std::memset(&c, 0, sizeof c);
     c.slots = g.slots; c.slot_stride = g.slot_stride; c.n_quads = lo.state_bytes / 16;
@@ -1281,6 +1306,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
 
   // Everything the step enqueues; an error ends the enqueueing, and the caller below still waits for both
   // streams before it returns, so no work is in flight on the caller's buffers after any return.
+  NvtxRange step_range("snn_train_step");
   auto enqueue = [&]() -> snn_status {
   // ---- start-of-step state: status, counts, delta carry, list offsets, spikes at t = 0, gradients
   CUDA_TRY(cudaMemsetAsync(ex.ws + lo.status, 0, 256, ms));
@@ -1315,8 +1341,11 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   for (int i = 0; i < (int)ops.size(); ++i)
     if (ops[i].kind == SNN_OP_FWD) last_fwd = i;
   snn_status st = SNN_OK;
+  static const char* const op_names[] = {"snn:forward", "snn:re-forward 1", "snn:re-forward 2", "snn:backward",
+                                         "snn:checkpoint to host", "snn:checkpoint from host", "snn:clear state"};
   for (int i = 0; i < (int)ops.size() && st == SNN_OK; ++i) {
     const snn_op& op = ops[i];
+    NvtxRange range(op.kind >= 0 && op.kind <= SNN_OP_ZERO ? op_names[op.kind] : "snn:op");
     switch (op.kind) {
       case SNN_OP_ZERO:
         st = ex.wait_slot(op.keep_slot);
@@ -1382,6 +1411,9 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     e.offsets_off = lo.off[l]; e.pool_off = lo.pool[l]; e.values_off = lo.vals[l]; e.pool_capacity = lo.cap[l];
     e.mask_off = lo.mask[l]; e.mask_words = lo.words[l];
   }
+  if ((host_status[0] & STATUS_DEBUG_CHECK) || ex.debug_violation)
+    return fail(net, SNN_ERR_DEBUG_CHECK, "an index check of the bounds-checked build failed (%s)",
+                ex.debug_violation ? "state slot outside the layout" : "event position or row index out of range");
   if (host_status[0] & STATUS_BAD_TARGET)
     return fail(net, SNN_ERR_INVALID_ARG, "a target is outside [0, %d)", sz[L + 1]);
   if (host_status[0] & STATUS_SYNC_TIMEOUT)

@@ -678,6 +678,44 @@ def test_backward_as_one_launch_per_segment(orc32):
         s.close()
 
 
+def test_bounds_checked_build_gives_the_same_bits(tmp_path):
+    """libsnnckpt_debug.so (the same sources with -DSNN_DEBUG_CHECKS=1) tests event positions, row indices and state
+    slots before use.  On a correct step no check fires and every gradient has the bits of the ordinary build, on the
+    paths that replay stored event lists and on the default ones.  Runs in a child process: the library is chosen at
+    import time by SNN_DEBUG_CHECKS=1."""
+    import os, subprocess, sys, textwrap
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "debug_step.py"
+    script.write_text(textwrap.dedent(f"""
+        import sys, hashlib
+        sys.path.insert(0, {root!r}); sys.path.insert(0, {os.path.join(root, "tests")!r})
+        import snn_workloads as wl
+        from gpu_helpers import make_session
+        from paper_2412_11810_b200 import binding as b
+        print("checks", b.lib.snn_debug_checks_enabled())
+        w = wl.small(sizes=(40, 260, 132, 6), T=21, B=5, p_in=0.1, g_ff=(2.5, 1.6), seed=19)
+        d = wl.make(w)
+        s, bits, targets = make_session(w, d)
+        for strat, K, R, flags in ((0, 0, 0, 0), (3, 2, 8, 0), (3, 2, 8, b.SNN_FLAG_REFORWARD_PER_STEP), (2, 5, 0, 0),
+                                   (1, 4, 0, b.SNN_FLAG_FORWARD_PER_STEP | b.SNN_FLAG_REFORWARD_PER_STEP)):
+            s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0, extra_flags=flags)
+            h = hashlib.sha256()
+            for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+                h.update(g.cpu().numpy().tobytes())
+            print("grad", strat, K, R, flags, h.hexdigest())
+        s.close()
+    """))
+    outs = []
+    for debug in ("0", "1"):
+        env = dict(os.environ, SNN_DEBUG_CHECKS=debug)
+        r = subprocess.run([sys.executable, str(script)], capture_output=True, text=True, env=env, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        lines = r.stdout.splitlines()
+        assert lines[0] == f"checks {debug}"
+        outs.append([l for l in lines if l.startswith("grad")])
+    assert len(outs[0]) == 5 and outs[0] == outs[1]
+
+
 def test_a_wait_that_cannot_end_gives_up():
     """The waits between thread blocks are bounded: one that nothing satisfies raises the time-out status
     after its poll limit and the kernel ends; the context stays usable for a normal step afterwards."""
