@@ -1553,12 +1553,13 @@ __device__ __forceinline__ void bwd_epilogue(const BwdParams& p, const BwdLayer&
 constexpr int BWD_LD = 132;   // padded row length (floats) of the staged tiles: fragment loads hit 32 banks
 
 // fp32 -> two tf32 pieces (10 mantissa bits each): hi = x with its 13 low mantissa bits cleared, lo = x - hi (exact
-// in fp32: the cleared bits) cut to tf32 the same way.  Three integer / floating-point operations at full rate per
-// value; conversion instructions run at an eighth of it and would cost as much as the tensor-core work they feed.
-// hi + lo differs from x by less than 2^-20 |x|.
+// in fp32: the cleared bits).  mma.sync reads only the 19 high bits of a tf32 operand (checked on the device: clearing
+// the low bits of lo as well changes no result bit), so lo is passed as it is and the tensor core cuts it to tf32.
+// Two operations at full rate per value; conversion instructions run at an eighth of it and would cost as much as the
+// tensor-core work they feed.  hi + tf32(lo) differs from x by less than 2^-20 |x|.
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
   hi = __float_as_uint(x) & 0xffffe000u;
-  lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
+  lo = __float_as_uint(x - __uint_as_float(hi));
 }
 // D(16x8) += A(16x8, row) * B(8x8, col); lane = 4 g + t holds A[g][t], A[g+8][t], A[g][t+4], A[g+8][t+4],
 // B[t][g], B[t+4][g] and D[g][2t], D[g][2t+1], D[g+8][2t], D[g+8][2t+1].

@@ -206,12 +206,13 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
       float4* const al = reinterpret_cast<float4*>(stage_a_lo(s));
       float4* const bh = reinterpret_cast<float4*>(stage_b_hi(s));
       float4* const bl = reinterpret_cast<float4*>(stage_b_lo(s));
-      auto split4 = [](float4 x, float4& hi, float4& lo) {
-        uint32_t h, l;
-        split_tf32(x.x, h, l); hi.x = __uint_as_float(h); lo.x = __uint_as_float(l);
-        split_tf32(x.y, h, l); hi.y = __uint_as_float(h); lo.y = __uint_as_float(l);
-        split_tf32(x.z, h, l); hi.z = __uint_as_float(h); lo.z = __uint_as_float(l);
-        split_tf32(x.w, h, l); hi.w = __uint_as_float(h); lo.w = __uint_as_float(l);
+      // both pieces are cut to tf32 here, so that what the tensor cores read needs no rounding of theirs
+      auto cut = [](float v) { return __uint_as_float(__float_as_uint(v) & 0xffffe000u); };
+      auto split4 = [&](float4 x, float4& hi, float4& lo) {
+        hi.x = cut(x.x); lo.x = cut(x.x - hi.x);
+        hi.y = cut(x.y); lo.y = cut(x.y - hi.y);
+        hi.z = cut(x.z); lo.z = cut(x.z - hi.z);
+        hi.w = cut(x.w); lo.w = cut(x.w - hi.w);
       };
 #pragma unroll
       for (int q = 0; q < (int)(TCG_A_BYTES / 16) / (32 * TCG_CONV_WARPS); ++q) {
