@@ -153,7 +153,8 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
 /* Networks whose weights exceed L2 compute those input currents with the weight rows as the stationary
  * operand instead: a thread block reads each row of its column slab once per run and adds it to every
  * (step, sample) of the run in which that neuron fired (spiking cell).  This flag forces that order for
- * smaller networks too.  Results are bit-identical either way. */
+ * smaller networks, and for the graded cell (each event then multiplies the row by its value), too.  Results are
+ * bit-identical either way. */
 #define SNN_FLAG_REFORWARD_ROWS 512u
 /* The forward pass of a spiking (LIF) network whose weights fit in L2 runs as one cooperative launch per
  * forward operation of the plan when the device can hold all its thread blocks at once: blocks wait for

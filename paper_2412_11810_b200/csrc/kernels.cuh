@@ -887,6 +887,202 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
   }
 }
 
+// The same for the graded cell: an event carries a value, and an accumulator takes fma(value, w, acc) per event in
+// the same ascending order.  The pre-pass stores, per (block of 32 rows, pair), the count, up to eight row numbers
+// (two words, one byte each) and the eight values that go with them (read from the value pool at the position the
+// stored list offsets and per-word prefixes give); a block with more events keeps its raw spike word and the pool
+// position of its first value, and the consumer reads those values from the pool.
+struct RowsGradedLayer {
+  const uint32_t* ff_off;     // list offsets of the layer below, row 0: [(T+2)][B]
+  const uint16_t* ff_pref;    // events before each spike word of the layer below, row 0: [(T+2)][B][W_pre]
+  const float* ff_vals;       // its value pool [B][ff_cap]
+  const uint32_t* rec_off;    // the same for the own layer
+  const uint16_t* rec_pref;
+  const float* rec_vals;
+  size_t ff_cap, rec_cap;
+};
+
+struct RowsGradedParams {
+  RowsParams r;               // events: plane 0 counts, 1 and 2 row numbers, 3 .. 10 values [block][pair][8]
+  RowsGradedLayer g[MAXL];
+  size_t plane;               // words per plane
+};
+
+constexpr uint32_t RRG_MAX = 8;        // events of a block held in the staged words
+constexpr uint32_t RRG_MANY = 15u;     // count of a block with more
+__host__ __device__ inline size_t refwd_rows_graded_smem_bytes(int pb) {
+  return (size_t)RR_STAGES * (RR_TILE_BYTES + 11 * (size_t)pb * sizeof(uint32_t)) + 2 * RR_STAGES * sizeof(uint64_t);
+}
+
+__global__ void __launch_bounds__(128) rows_events_graded_kernel(const __grid_constant__ RowsGradedParams gp) {
+  pdl_launch_dependents();
+  const RowsParams& p = gp.r;
+  const RowsLayer& L = p.lay[blockIdx.z];
+  const RowsGradedLayer& G = gp.g[blockIdx.z];
+  const int rb = blockIdx.y, pair = blockIdx.x * 128 + threadIdx.x;
+  if (rb >= L.W_pre + L.W || pair >= p.ev_stride) return;
+  pdl_wait();
+  uint32_t bits = 0;
+  uint32_t first = 0;          // position of the block's first value in its sample's pool
+  const float* pool = G.ff_vals;   // ... which starts here
+  if (pair < p.n * p.B) {
+    const int t = p.t0 + p.d0 + 1 + pair / p.B, b = pair % p.B;
+    if (rb < L.W_pre) {
+      const size_t row = (size_t)(t - L.ff_row0) * p.B + b;        // spike words of the layer below at step t
+      bits = L.ff_words[row * L.W_pre + rb];
+      if (rb == L.W_pre - 1) bits &= last_word_mask(L.N_pre);
+      const size_t lrow = (size_t)t * p.B + b;                      // its list (step t) in the offset and prefix rows
+      first = G.ff_off[lrow] + G.ff_pref[lrow * L.W_pre + rb];
+      pool = G.ff_vals + (size_t)b * G.ff_cap;
+    } else {
+      const size_t lrow = (size_t)(t - 1) * p.B + b;                // own layer at step t - 1
+      bits = L.words[lrow * L.W + (rb - L.W_pre)];
+      first = G.rec_off[lrow] + G.rec_pref[lrow * L.W + (rb - L.W_pre)];
+      pool = G.rec_vals + (size_t)b * G.rec_cap;
+    }
+  }
+  const uint32_t cnt = __popc(bits);
+  const size_t at = L.ev_off + (size_t)rb * p.ev_stride + pair;
+  uint32_t ra = bits, rbw = first;   // more than RRG_MAX events: the raw word and the position in the sample's pool
+  float v[RRG_MAX];
+#pragma unroll
+  for (int k = 0; k < (int)RRG_MAX; ++k) v[k] = 0.f;
+  if (cnt <= RRG_MAX) {
+    ra = 0; rbw = 0;
+    uint32_t rest = bits;
+#pragma unroll
+    for (int k = 0; k < (int)RRG_MAX; ++k) {
+      if (rest) {
+        const uint32_t r = (uint32_t)(__ffs(rest) - 1);
+        rest &= rest - 1;
+        if (k < 4) ra |= r << (8 * k); else rbw |= r << (8 * (k - 4));
+        v[k] = pool[first + k];
+      }
+    }
+  }
+  p.events[at] = cnt <= RRG_MAX ? cnt : RRG_MANY;
+  p.events[gp.plane + at] = ra;
+  p.events[2 * gp.plane + at] = rbw;
+  float4* vdst = reinterpret_cast<float4*>(p.events + 3 * gp.plane + 8 * at);
+  vdst[0] = make_float4(v[0], v[1], v[2], v[3]);
+  vdst[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+// a = fma(v, w, a) on two fp32 lanes, each rounded once (as __fmaf_rn)
+__device__ __forceinline__ void fma_f32x2(unsigned long long& a, const unsigned long long w, const unsigned long long vv) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a) : "l"(w), "l"(vv));
+}
+
+__global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_graded_kernel(const __grid_constant__ RowsGradedParams gp) {
+  pdl_launch_dependents();
+  const RowsParams& p = gp.r;
+  const int l = blockIdx.z;
+  const RowsLayer& L = p.lay[l];
+  const RowsGradedLayer& G = gp.g[l];
+  const int col0 = blockIdx.y * RR_COLS;
+  const int pairs = p.n * p.B, pair0 = blockIdx.x * p.pb;
+  if (col0 >= L.N || pair0 >= pairs) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_consumers = p.pb / RR_PPW;
+  extern __shared__ __align__(128) unsigned char s_raw_bytes[];
+  float4* const s_tiles = reinterpret_cast<float4*>(s_raw_bytes);                                         // [RR_STAGES][32][32]
+  uint32_t* const s_ev = reinterpret_cast<uint32_t*>(s_raw_bytes + (size_t)RR_STAGES * RR_TILE_BYTES);   // [RR_STAGES][11][pb]
+  uint64_t* const s_full = reinterpret_cast<uint64_t*>(s_ev + (size_t)RR_STAGES * 11 * p.pb);
+  uint64_t* const s_empty = s_full + RR_STAGES;
+  const int n_blocks = L.W_pre + L.W;
+  if (tid == 0) {
+    for (int s = 0; s < RR_STAGES; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, n_consumers); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  const uint32_t ev_bytes = (uint32_t)p.pb * sizeof(uint32_t);
+  if (warp == n_consumers) {
+    if (lane == 0) {
+      const uint32_t* ev_src = p.events + L.ev_off + pair0;
+      for (int rb = 0; rb < n_blocks; ++rb) {
+        const int stage = rb % RR_STAGES;
+        if (rb >= RR_STAGES && !mbar_wait(s_empty + stage, (uint32_t)(rb / RR_STAGES - 1) & 1u)) {
+          atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+          break;
+        }
+        mbar_arrive_expect_tx(s_full + stage, RR_TILE_BYTES + 11 * ev_bytes);
+        const bool ff = rb < L.W_pre;
+        tma_load_2d(s_tiles + (size_t)stage * (RR_TILE_BYTES / 16), ff ? &p.map_ff[l] : &p.map_rec[l], col0,
+                    (ff ? rb : rb - L.W_pre) * RR_ROWS, s_full + stage);
+        uint32_t* const dst = s_ev + (size_t)stage * 11 * p.pb;
+        const uint32_t* const src = ev_src + (size_t)rb * p.ev_stride;
+        bulk_load(dst, src, ev_bytes, s_full + stage);
+        bulk_load(dst + p.pb, src + gp.plane, ev_bytes, s_full + stage);
+        bulk_load(dst + 2 * p.pb, src + 2 * gp.plane, ev_bytes, s_full + stage);
+        bulk_load(dst + 3 * p.pb, p.events + 3 * gp.plane + 8 * (L.ev_off + (size_t)rb * p.ev_stride + pair0), 8 * ev_bytes,
+                  s_full + stage);
+      }
+    }
+    return;
+  }
+  unsigned long long acc01[RR_PPW], acc23[RR_PPW];
+#pragma unroll
+  for (int i = 0; i < RR_PPW; ++i) acc01[i] = acc23[i] = 0ull;
+  const uint32_t lane_off = smem_u32(s_tiles) + (uint32_t)lane * 16u;
+  for (int rb = 0; rb < n_blocks; ++rb) {
+    const int stage = rb % RR_STAGES;
+    if (!mbar_wait(s_full + stage, (uint32_t)(rb / RR_STAGES) & 1u)) {
+      if (lane == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+      return;
+    }
+    const uint32_t tile = lane_off + (uint32_t)stage * RR_TILE_BYTES;
+    const uint32_t* const evs = s_ev + (size_t)stage * 11 * p.pb + warp * RR_PPW;
+    const float* const vals = reinterpret_cast<const float*>(s_ev + (size_t)stage * 11 * p.pb + 3 * p.pb) + warp * RR_PPW * 8;
+    auto fma_row = [&](int i, uint32_t r, float v) {
+      unsigned long long w01, w23, vv;
+      lds_2x64(tile + r * (RR_COLS * 4u), w01, w23);
+      asm("mov.b64 %0, {%1, %1};" : "=l"(vv) : "f"(v));
+      fma_f32x2(acc01[i], w01, vv); fma_f32x2(acc23[i], w23, vv);
+    };
+#pragma unroll
+    for (int i = 0; i < RR_PPW; ++i) {
+      const uint32_t cnt = evs[i];
+      if (cnt == 0) continue;
+      if (cnt != RRG_MANY) {
+        uint32_t rows = evs[p.pb + i];
+        for (uint32_t k = 0; k < cnt; ++k) {   // ascending rows; the count is the same for the whole warp
+          if (k == 4) rows = evs[2 * p.pb + i];
+          fma_row(i, rows & 0xffu, vals[i * 8 + k]);
+          rows >>= 8;
+        }
+      } else {
+        uint32_t bits = evs[p.pb + i];
+        const int b = (pair0 + warp * RR_PPW + i) % p.B;
+        const float* src = rb < L.W_pre ? G.ff_vals + (size_t)b * G.ff_cap : G.rec_vals + (size_t)b * G.rec_cap;
+        size_t at = evs[2 * p.pb + i];   // position of the block's first value in the sample's pool
+        while (bits) {
+          fma_row(i, (uint32_t)__ffs(bits) - 1u, __ldg(src + at));
+          bits &= bits - 1;
+          ++at;
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(s_empty + stage);
+  }
+  const int col = col0 + lane * 4;
+  if (col < L.N) {
+#pragma unroll
+    for (int i = 0; i < RR_PPW; ++i) {
+      const int pair = pair0 + warp * RR_PPW + i;
+      if (pair < pairs) {
+        const int d = p.d0 + 1 + pair / p.B, b = pair % p.B;
+        float4 v;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(v.x), "=f"(v.y) : "l"(acc01[i]));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(v.z), "=f"(v.w) : "l"(acc23[i]));
+        *reinterpret_cast<float4*>(p.slots + (size_t)(p.buf_slot + (d - 1) % p.buf_len) * p.slot_stride + L.state_off +
+                                   (size_t)b * L.N + col) = v;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // Forward pass over a whole segment of steps in one cooperative launch (LIF cell).
 //

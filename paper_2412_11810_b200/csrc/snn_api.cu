@@ -159,7 +159,7 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     lo.gff = L > 1 ? take(4 * lo.gff_stride * TCG_MAX_KSPLIT) : 0;
   }
   lo.rows_ev = 0; lo.rows_ev_words = 0; lo.rows_ev_stride = 0;
-  if (!graded && ck->strategy != SNN_STANDARD) {
+  if (ck->strategy != SNN_STANDARD) {
     // one word per (32 presynaptic rows, pair) for the pairs of a run (at most chunk_size steps), twice
     const int Kc = std::min(std::max(ck->chunk_size, 1), T);
     const size_t stride = ((size_t)Kc * B + RR_MAX_PB - 1) / RR_MAX_PB * RR_MAX_PB;
@@ -167,7 +167,7 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
     for (int l = 1; l <= L; ++l) blocks += (size_t)lo.words[l - 1] + lo.words[l];
     lo.rows_ev_stride = stride;
     lo.rows_ev_words = stride * blocks;
-    lo.rows_ev = take(2 * 4 * lo.rows_ev_words);
+    lo.rows_ev = take((graded ? 11 : 2) * 4 * lo.rows_ev_words);   // graded cell: counts, two words of rows, eight values
   }
   lo.slots = take((size_t)lo.n_local * lo.state_bytes);
   lo.tier2_on_device = ck->strategy == SNN_DOUBLE_LOCAL;
@@ -513,8 +513,10 @@ struct Exec {
     return (long long)L * std::min(op.buf_len, op.t1 - op.t0) <= 65535;
   }
   // the currents of a run come from refwd_rows_kernel (weight rows stationary) rather than refwd_gather_kernel
+  // (spiking cell beyond L2 by default; the graded cell only on request: with values to fetch per event and 10 %
+  // activity its rows-stationary pass measured slower than the per-step gather on the benchmark's graded network)
   bool reforward_rows() const {
-    return !graded() && (!lo.weights_resident || (a->flags & SNN_FLAG_REFORWARD_ROWS));
+    return (!lo.weights_resident && !graded()) || (a->flags & SNN_FLAG_REFORWARD_ROWS);
   }
 
   // tensor maps of the feed-forward matrices for ff_gemm_tc_kernel: 0 not tried yet, 1 ready, -1 not encodable
@@ -564,6 +566,23 @@ struct Exec {
     }
     r.t0 = op.t0; r.d0 = d0; r.n = n; r.buf_slot = op.buf_slot; r.buf_len = op.buf_len;
     r.pb = pb; r.ev_stride = n_pb * pb;
+    if (graded()) {
+      RowsGradedParams gp;
+      std::memset(&gp, 0, sizeof gp);
+      gp.r = r;
+      gp.plane = lo.rows_ev_words;
+      for (int l = 1; l <= L; ++l) {
+        RowsGradedLayer& g = gp.g[l - 1];
+        g.ff_off = off(l - 1, 0); g.ff_pref = pref(l - 1, 0); g.ff_vals = vals(l - 1); g.ff_cap = lo.cap[l - 1];
+        g.rec_off = off(l, 0); g.rec_pref = pref(l, 0); g.rec_vals = vals(l); g.rec_cap = lo.cap[l];
+      }
+      CUDA_TRY(launch_pdl(rows_events_graded_kernel, dim3((unsigned)((r.ev_stride + 127) / 128), (unsigned)blocks_max, (unsigned)L),
+                          dim3(128), 0, gp));
+      CUDA_TRY(launch_pdl(refwd_rows_graded_kernel, dim3((unsigned)n_pb, (unsigned)slabs_max, (unsigned)L),
+                          dim3(32 * (pb / RR_PPW + 1)), refwd_rows_graded_smem_bytes(pb), gp));
+      launches += 2;
+      return SNN_OK;
+    }
     CUDA_TRY(launch_pdl(rows_events_kernel, dim3((unsigned)((r.ev_stride + 127) / 128), (unsigned)blocks_max, (unsigned)L),
                         dim3(128), 0, r));
     CUDA_TRY(launch_pdl(refwd_rows_kernel, dim3((unsigned)n_pb, (unsigned)slabs_max, (unsigned)L),
@@ -1211,6 +1230,7 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, dyn, (int)REFWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, dyn, (int)REFWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(refwd_rows_kernel, dyn, (int)refwd_rows_smem_bytes(RR_MAX_PB)));
+  CUDA_TRY(cudaFuncSetAttribute(refwd_rows_graded_kernel, dyn, (int)refwd_rows_graded_smem_bytes(RR_MAX_PB)));
   CUDA_TRY(cudaFuncSetAttribute(ff_gemm_kernel, dyn, (int)Exec::bwd_smem_bytes(8 * FFG_NTN)));
   CUDA_TRY(cudaFuncSetAttribute(ff_gemm_tc_kernel, dyn, (int)TCG_SMEM_BYTES));
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8, bwd_ld(8))));

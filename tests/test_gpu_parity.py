@@ -641,12 +641,27 @@ def test_graded_reforward_as_one_launch_per_segment(orc32):
     assert_grads_close(s.gradients(), run_oracle(orc32, w, d))
     base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
     for strat, K, R in [(1, 6, 0), (3, 4, 12), (2, 40, 0)]:
-        for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP):
+        for flags in (0, b.SNN_FLAG_REFORWARD_PER_STEP, b.SNN_FLAG_REFORWARD_ROWS):
+            for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+                g.fill_(float("nan"))
             s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0,
                          extra_flags=flags)
             for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
                 assert np.array_equal(x, y), (strat, K, R, flags)
     s.close()
+    # the rows-stationary order (large networks) with few and with many events per block of 32 rows
+    for kw in (dict(p_in=0.05, g_ff=(2.5, 1.2), seed=56), dict(p_in=0.5, g_ff=(1.5, 1.2), seed=57)):
+        w = _graded(sizes=(40, 264, 132, 9), T=30, B=21, **kw)
+        d = wl.make(w)
+        s, bits, targets = make_session(w, d)
+        s.train_step(bits, targets, strategy=0, max_activity=1.0)
+        base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+        for strat, K, R in [(1, 7, 0), (3, 4, 12)]:
+            s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0,
+                         extra_flags=b.SNN_FLAG_REFORWARD_ROWS)
+            for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+                assert np.array_equal(x, y), (kw, strat, K, R)
+        s.close()
 
 
 def test_backward_as_one_launch_per_segment(orc32):
