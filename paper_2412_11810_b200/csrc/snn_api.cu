@@ -29,6 +29,7 @@ struct snn_net {
   // layout of the last step, for inspection
   std::vector<snn_event_layout> ev_layout;
   cudaEvent_t ev_main = nullptr;
+  cudaEvent_t ev_window[2] = {nullptr, nullptr};   // completion of the last copy of each event window (spilled events)
   std::vector<cudaEvent_t> copy_events;    // one per checkpoint copy in flight, grown on demand
   std::vector<cudaEvent_t> timing_events;  // grown on demand, reused by every timed step
   snn_phase_times phases{};
@@ -214,6 +215,8 @@ extern "C" snn_status snn_create(const snn_config* cfg, snn_net** out) {
 extern "C" void snn_destroy(snn_net* net) {
   if (!net) return;
   if (net->ev_main) cudaEventDestroy(net->ev_main);
+  for (cudaEvent_t e : net->ev_window)
+    if (e) cudaEventDestroy(e);
   for (auto& e : net->copy_events) cudaEventDestroy(e);
   for (auto& e : net->timing_events) cudaEventDestroy(e);
   delete net;
@@ -366,8 +369,6 @@ struct Exec {
 
   // ---- event windows (SNN_FLAG_SPILL_EVENTS)
   int ev_resident[2] = {0, -1};    // segment each window holds
-  int ev_copy_event[2] = {-1, -1}; // copy event (index into net->copy_events, from the end) the window still waits on
-  cudaEvent_t ev_events[2] = {nullptr, nullptr};
   bool ev_pending[2] = {false, false};
   char* ev_host(int seg) const {
     return static_cast<char*>(a->pinned_ws) + (lo.tier2_on_device ? 0 : (size_t)lo.n_remote * lo.state_bytes) +
@@ -379,12 +380,12 @@ struct Exec {
   }
   // The main stream waits for the copy that last touched window w, if one is pending.
   snn_status ev_wait(int w) {
-    if (ev_pending[w]) { CUDA_TRY(cudaStreamWaitEvent(main, ev_events[w], 0)); ev_pending[w] = false; }
+    if (ev_pending[w]) { CUDA_TRY(cudaStreamWaitEvent(main, net->ev_window[w], 0)); ev_pending[w] = false; }
     return SNN_OK;
   }
   // A copy of window w on the side stream, after everything issued so far on the main stream.
   snn_status ev_copy(int w, int seg, bool to_host) {
-    if (!ev_events[w]) CUDA_TRY(cudaEventCreateWithFlags(&ev_events[w], cudaEventDisableTiming));
+    if (!net->ev_window[w]) CUDA_TRY(cudaEventCreateWithFlags(&net->ev_window[w], cudaEventDisableTiming));   // once per net
     CUDA_TRY(cudaEventRecord(net->ev_main, main));
     CUDA_TRY(cudaStreamWaitEvent(side, net->ev_main, 0));
     char* dev = ws + lo.ev_base + (size_t)w * lo.ev_window_bytes;
@@ -392,7 +393,7 @@ struct Exec {
     if (to_host) CUDA_TRY(cudaMemcpyAsync(ev_host(seg), dev, lo.ev_window_bytes, cudaMemcpyDeviceToHost, side));
     else CUDA_TRY(cudaMemcpyAsync(dev, ev_host(seg), lo.ev_window_bytes, cudaMemcpyHostToDevice, side));
     end_span(span, side);
-    CUDA_TRY(cudaEventRecord(ev_events[w], side));
+    CUDA_TRY(cudaEventRecord(net->ev_window[w], side));
     ev_pending[w] = true;
     ++ev_copies;
     return SNN_OK;
@@ -1404,8 +1405,6 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
   // ---- finish: everything on both streams, then status and loss
   cudaError_t e1 = cudaStreamSynchronize(ex.side);
   cudaError_t e2 = cudaStreamSynchronize(ex.main);
-  for (cudaEvent_t& e : ex.ev_events)
-    if (e) { cudaEventDestroy(e); e = nullptr; }
   if (st != SNN_OK) return st;
   if (e1 != cudaSuccess || e2 != cudaSuccess)
     return fail(net, SNN_ERR_CUDA, "stream synchronize failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
