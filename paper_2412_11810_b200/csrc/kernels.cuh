@@ -720,9 +720,10 @@ constexpr int RR_PPW = 8;        // pairs per consumer warp (32 accumulator regi
                                  // hide the shared-memory latency of the data-dependent row reads)
 constexpr int RR_MAX_PB = 128;   // at most 16 consumer warps
 constexpr uint32_t RR_TILE_BYTES = RR_ROWS * RR_COLS * sizeof(float);
+constexpr uint32_t RR_STAGE_BYTES = RR_TILE_BYTES + RR_COLS * sizeof(float);   // the tile and one row of zeros after it
 constexpr uint32_t RR_EV_MANY = 7u;   // count field of an event word whose block has more than four firing rows
 __host__ __device__ inline size_t refwd_rows_smem_bytes(int pb) {
-  return (size_t)RR_STAGES * (RR_TILE_BYTES + 2 * (size_t)pb * sizeof(uint32_t)) + 2 * RR_STAGES * sizeof(uint64_t);
+  return (size_t)RR_STAGES * (RR_STAGE_BYTES + 2 * (size_t)pb * sizeof(uint32_t)) + 2 * RR_STAGES * sizeof(uint64_t);
 }
 
 // Event words of the run: thread = (pair, block of 32 rows, layer).
@@ -742,22 +743,24 @@ __global__ void __launch_bounds__(128) rows_events_kernel(const __grid_constant_
       bits = L.words[((size_t)(t - 1) * p.B + b) * L.W + (rb - L.W_pre)];
     }
   }
-  // first word: the number of firing rows (RR_EV_MANY if more than four); second word: up to four row
-  // numbers, ascending, one per byte -- or the raw spike word when there are more
+  // first word: the number of firing rows (RR_EV_MANY if more than four) and, in bytes 1 and 2, the first two of
+  // them; second word: the third and fourth in bytes 0 and 1 -- or the raw spike word when there are more than four.
+  // A row that does not exist is written as RR_ROWS: the consumer's tile has one more row, of zeros, so that it can
+  // add two rows per pair without looking at the count (x + 0 = x exactly, and no accumulator is ever -0)
   const uint32_t cnt = __popc(bits);
-  uint32_t w = RR_EV_MANY, rows = bits;
-  if (cnt <= 4) {
-    w = cnt;
-    rows = 0;
+  uint32_t r[4] = {RR_ROWS, RR_ROWS, RR_ROWS, RR_ROWS};
+  {
     uint32_t rest = bits;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       if (rest) {
-        rows |= (uint32_t)(__ffs(rest) - 1) << (8 * k);
+        r[k] = (uint32_t)(__ffs(rest) - 1);
         rest &= rest - 1;
       }
     }
   }
+  const uint32_t w = (cnt <= 4 ? cnt : RR_EV_MANY) | r[0] << 8 | r[1] << 16;
+  const uint32_t rows = cnt <= 4 ? (r[2] | r[3] << 8) : bits;
   const size_t at = L.ev_off + (size_t)rb * p.ev_stride + pair;
   p.events[at] = w;
   p.events[p.raw_off + at] = rows;
@@ -781,8 +784,8 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_consumers = p.pb / RR_PPW;            // consumer warps 0 .. n_consumers-1, then the producer warp
   extern __shared__ __align__(128) unsigned char s_raw_bytes[];
-  float4* const s_tiles = reinterpret_cast<float4*>(s_raw_bytes);                                 // [RR_STAGES][32][32]
-  uint32_t* const s_ev = reinterpret_cast<uint32_t*>(s_raw_bytes + (size_t)RR_STAGES * RR_TILE_BYTES);   // [RR_STAGES][2][pb]
+  unsigned char* const s_tiles = s_raw_bytes;                                 // [RR_STAGES]: [32][128] fp32, then 128 zeros
+  uint32_t* const s_ev = reinterpret_cast<uint32_t*>(s_raw_bytes + (size_t)RR_STAGES * RR_STAGE_BYTES);   // [RR_STAGES][2][pb]
   uint64_t* const s_full = reinterpret_cast<uint64_t*>(s_ev + (size_t)RR_STAGES * 2 * p.pb);       // [RR_STAGES]
   uint64_t* const s_empty = s_full + RR_STAGES;
   const int n_blocks = L.W_pre + L.W;
@@ -790,6 +793,8 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
     for (int s = 0; s < RR_STAGES; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, n_consumers); }
     mbar_fence_init();
   }
+  for (int q = tid; q < RR_STAGES * RR_COLS; q += blockDim.x)   // the row of zeros behind every tile
+    reinterpret_cast<float*>(s_tiles + (size_t)(q / RR_COLS) * RR_STAGE_BYTES + RR_TILE_BYTES)[q % RR_COLS] = 0.f;
   __syncthreads();
   pdl_wait();
   const uint32_t ev_bytes = (uint32_t)p.pb * sizeof(uint32_t);
@@ -805,7 +810,7 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
         }
         mbar_arrive_expect_tx(s_full + stage, RR_TILE_BYTES + 2 * ev_bytes);
         const bool ff = rb < L.W_pre;
-        tma_load_2d(s_tiles + (size_t)stage * (RR_TILE_BYTES / 16), ff ? &p.map_ff[l] : &p.map_rec[l], col0,
+        tma_load_2d(s_tiles + (size_t)stage * RR_STAGE_BYTES, ff ? &p.map_ff[l] : &p.map_rec[l], col0,
                     (ff ? rb : rb - L.W_pre) * RR_ROWS, s_full + stage);
         uint32_t* const dst = s_ev + (size_t)stage * 2 * p.pb;
         bulk_load(dst, ev_src + (size_t)rb * p.ev_stride, ev_bytes, s_full + stage);
@@ -825,7 +830,7 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
       if (lane == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
       return;
     }
-    const uint32_t tile = lane_off + (uint32_t)stage * RR_TILE_BYTES;
+    const uint32_t tile = lane_off + (uint32_t)stage * RR_STAGE_BYTES;
     const uint32_t* const evs = s_ev + (size_t)stage * 2 * p.pb + warp * RR_PPW;
     uint32_t e[RR_PPW];
 #pragma unroll
@@ -845,25 +850,30 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
       lds_2x64(tile + r * (RR_COLS * 4u), w01, w23);
       add_f32x2(acc01[i], w01); add_f32x2(acc23[i], w23);
     };
+    // Two rows per pair without a look at the count (a missing row is the row of zeros): sixteen independent reads
+    // in flight, no branch; most blocks hold at most two events.  The third and fourth row, or the rows of a block
+    // with more than four (raw spike word, its two lowest bits already done), follow behind a branch on the count,
+    // which is the same for the whole warp.  Per accumulator the rows are added in ascending order.
 #pragma unroll
     for (int i = 0; i < RR_PPW; ++i) {
-      // the count is the same for the whole warp: real branches, the common counts first, straight-line
-      // code for each (independent reads, additions in ascending row order)
-      const uint32_t cnt = e[i], r = rw[i];
-      if (cnt == 0) {
-      } else if (cnt == 1) {
-        add_row(i, r & 0xffu);
-      } else if (cnt == 2) {
-        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu);
-      } else if (cnt == 3) {
-        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu); add_row(i, (r >> 16) & 0xffu);
-      } else if (cnt == 4) {
-        add_row(i, r & 0xffu); add_row(i, (r >> 8) & 0xffu); add_row(i, (r >> 16) & 0xffu); add_row(i, r >> 24);
-      } else {
-        uint32_t bits = r;
-        while (bits) {
-          add_row(i, (uint32_t)__ffs(bits) - 1u);
+      add_row(i, (e[i] >> 8) & 0xffu);
+      add_row(i, (e[i] >> 16) & 0xffu);
+    }
+#pragma unroll
+    for (int i = 0; i < RR_PPW; ++i) {
+      const uint32_t cnt = e[i] & 7u;
+      if (cnt > 2) {
+        if (cnt != RR_EV_MANY) {
+          add_row(i, rw[i] & 0xffu);
+          add_row(i, (rw[i] >> 8) & 0xffu);
+        } else {
+          uint32_t bits = rw[i];
           bits &= bits - 1;
+          bits &= bits - 1;
+          while (bits) {
+            add_row(i, (uint32_t)__ffs(bits) - 1u);
+            bits &= bits - 1;
+          }
         }
       }
     }
