@@ -2137,75 +2137,84 @@ struct BwdStreamParams {
   int surrogate, cell;
 };
 
+constexpr int BWD_STREAM_STAGES = 4;   // chunks in flight per warp
+
 template <int NTN, int NWARP>
 __host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
-  return ((size_t)BWD_STAGES * (BWD_TM + 8 * NTN) * bwd_ld(NWARP) + (size_t)NWARP * BWD_TM * (8 * NTN + 8)) * sizeof(float);
+  // the warps' copy rings (together BWD_STREAM_STAGES x (32 + BP) rows x 128 values) and their partial tiles
+  return ((size_t)BWD_STREAM_STAGES * (BWD_TM + 8 * NTN) * 128 + (size_t)NWARP * BWD_TM * (8 * NTN + 8)) * sizeof(float);
 }
 
 template <int NTN, int NWARP>
 __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
-  constexpr int LD = bwd_ld(NWARP), KS = 16 / NWARP;
-  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, STAGE_F = ROWS * LD, TILE = BWD_TM * BP;
+  // Every warp stages the values of its own k-steps of a chunk (KW adjacent contraction values: 32 rows of W and BP
+  // rows of delta, KW floats each) in a copy ring of its own: no CTA barrier inside the contraction, and the loads,
+  // splits and tensor-core passes of different warps overlap.
+  constexpr int KS = 16 / NWARP, KW = 8 * KS, S = BWD_STREAM_STAGES;
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, WSTAGE_F = ROWS * KW, TILE = BWD_TM * BP;
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
   constexpr int EPI = TILE / NT;
-  constexpr int ITER = ROWS * 32 / NT;      // 16-byte positions of a staged chunk per thread
-  constexpr int JW = BWD_TM * 32 / NT;      // the first JW of them are rows of W, the others rows of delta
-  static_assert(TILE % NT == 0 && ROWS * 32 % NT == 0 && BWD_TM * 32 % NT == 0, "tiles divide evenly among the threads");
+  constexpr int PW = BWD_TM * KW / 4 / 32;   // 16-byte pieces of the W part of a warp's stage per lane
+  constexpr int PD = (BP * KW / 4 + 31) / 32;   // ... of its delta part (the last ones may be past the end)
+  static_assert(TILE % NT == 0 && (BWD_TM * KW / 4) % 32 == 0, "tiles divide evenly among the threads");
   const int tile_row0 = blockIdx.x * BWD_TM;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   __shared__ int s_ok;
   extern __shared__ float4 s_dyn[];
-  float* const s_tiles = reinterpret_cast<float*>(s_dyn);            // [BWD_STAGES][ROWS][LD]
-  float* const s_parts = s_tiles + (size_t)BWD_STAGES * STAGE_F;     // [NWARP][32][TS] partial tiles of the warps
+  float* const ring = reinterpret_cast<float*>(s_dyn) + (size_t)warp * S * WSTAGE_F;   // [S][ROWS][KW] of this warp
+  float* const s_parts = reinterpret_cast<float*>(s_dyn) + (size_t)NWARP * S * WSTAGE_F;   // [NWARP][32][TS] partial tiles
   const int N = p.N, it_all = (N + 127) / 128, n_steps = p.ts_hi - p.ts_lo;
   const int total = n_steps * it_all;                                 // chunks of the whole run
   const int rlast = N - 1, blast = p.B - 1;
-  // fixed copy positions of this thread
-  const float* src_w[JW];
-  int d_row[ITER - JW], dst_off[ITER], kcol[ITER];
+  // fixed copy positions of this lane: piece q = lane + 32 j is row q / (KW / 4), values 4 (q % (KW / 4)) ..
+  const float* src_w[PW];
+  int d_row[PD], w_off[PW], d_off[PD], w_k[PW], d_k[PD];
 #pragma unroll
-  for (int j = 0; j < ITER; ++j) {
-    const int q = tid + j * NT, rr = q >> 5, c4 = q & 31;
-    kcol[j] = 4 * c4;
-    dst_off[j] = rr * LD + 4 * c4;
-    if (j < JW) {   // rows and samples past the end are clamped to the last valid one; never used
-      const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;
-      src_w[j] = p.W_rec + row * N + 4 * c4;
-    } else {
-      d_row[j - JW] = rr - BWD_TM < blast ? rr - BWD_TM : blast;
-    }
+  for (int j = 0; j < PW; ++j) {
+    const int q = lane + 32 * j, rr = q / (KW / 4), part = q % (KW / 4);
+    w_k[j] = warp * KW + 4 * part;
+    w_off[j] = rr * KW + 4 * part;
+    const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;   // rows past the end: a valid one, never used
+    src_w[j] = p.W_rec + row * N + w_k[j];
+  }
+#pragma unroll
+  for (int j = 0; j < PD; ++j) {
+    const int q = lane + 32 * j, rr = q / (KW / 4), part = q % (KW / 4);
+    d_k[j] = rr < BP ? warp * KW + 4 * part : -1;
+    d_off[j] = (BWD_TM + rr) * KW + 4 * part;
+    d_row[j] = rr < blast ? rr : blast;
   }
   // delta_{t+1} of the s-th step of the run (s = 0: the latest)
   auto dn_of = [&](int s) -> const float* {
     return s == 0 ? p.d_first : p.slots + (size_t)(p.buf_slot + p.ts_hi - s) * p.slot_stride + p.state_off;
   };
-  // W part of chunk c (the `it`-th of its step), positions [j0, j1) among the W positions
+  // W part of this warp's share of chunk c (the `it`-th of its step), pieces [j0, j1)
   auto issue_w = [&](int c, int it, int j0, int j1) {
     if (c < total) {
       const int k0 = it * 128;
-      float* st = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
+      float* st = ring + (size_t)(c % S) * WSTAGE_F;
 #pragma unroll
-      for (int j = 0; j < JW; ++j) {
+      for (int j = 0; j < PW; ++j) {
         if (j < j0 || j >= j1) continue;
-        if (k0 + kcol[j] < N) cp_async16(st + dst_off[j], src_w[j] + k0);
-        else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+        cp_async16_or_zero(st + w_off[j], k0 + w_k[j] < N ? src_w[j] + k0 : p.W_rec, k0 + w_k[j] < N);
       }
     }
   };
-  // delta part of chunk c (the `it`-th of its step)
+  // delta part of this warp's share of chunk c (the `it`-th of its step)
   auto issue_d = [&](int c, int it, const float* dn) {
     const int k0 = it * 128;
-    float* st = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
+    float* st = ring + (size_t)(c % S) * WSTAGE_F;
 #pragma unroll
-    for (int j = JW; j < ITER; ++j) {
-      if (k0 + kcol[j] < N) cp_async16(st + dst_off[j], dn + (size_t)d_row[j - JW] * N + kcol[j] + k0);
-      else *reinterpret_cast<float4*>(st + dst_off[j]) = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < PD; ++j) {
+      if (d_k[j] < 0) continue;
+      const bool real = k0 + d_k[j] < N;
+      cp_async16_or_zero(st + d_off[j], real ? dn + (size_t)d_row[j] * N + d_k[j] + k0 : p.W_rec, real);
     }
   };
   // the W parts of the first chunks: they do not depend on anything this launch computes
   int it_pre = 0;   // index within its step of the next chunk whose W part is issued (chunks wrap around the steps)
-  for (int c = 0; c < BWD_STAGES - 1; ++c) {
-    issue_w(c, it_pre, 0, JW);
+  for (int c = 0; c < S - 1; ++c) {
+    issue_w(c, it_pre, 0, PW);
     cp_async_commit();
     if (++it_pre == it_all) it_pre = 0;
   }
@@ -2243,7 +2252,7 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
     }
     // delta parts of the chunks of this step whose W part is already in flight
     const int c0 = s * it_all;
-    for (int cc = 0; cc < BWD_STAGES - 1 && cc < it_all; ++cc) issue_d(c0 + cc, cc, dn);
+    for (int cc = 0; cc < S - 1 && cc < it_all; ++cc) issue_d(c0 + cc, cc, dn);
     cp_async_commit();
     float acc[2][NTN][4];
 #pragma unroll
@@ -2254,19 +2263,18 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
         for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
     for (int it = 0; it < it_all; ++it) {
       const int c = c0 + it;
-      if (it == 0) cp_async_wait<0>();          // the delta parts issued just above are the latest group
-      else cp_async_wait<BWD_STAGES - 2>();     // this thread's copies of chunk c have landed
-      __syncthreads();                               // ... everybody's have, and chunk c-1 has been consumed
-      // refill of the stage chunk c-1 used: chunk c + BWD_STAGES - 1, its delta part only if it is of this step
-      const int c_refill = c + BWD_STAGES - 1;
-      const bool refill_d = it + BWD_STAGES - 1 < it_all;
-      const float* Ws = s_tiles + (size_t)(c % BWD_STAGES) * STAGE_F;
-      const float* Ds = Ws + BWD_TM * LD;
-      const int kl = warp * 8 * KS + 2 * KS * t;   // this lane's values of the chunk
+      if (it == 0) cp_async_wait<0>();   // the delta parts issued just above are the latest group
+      else cp_async_wait<S - 2>();        // this lane's copies of chunk c have landed
+      __syncwarp();                      // ... the whole warp's have, and the warp is done with chunk c-1
+      // refill of the stage chunk c-1 used: chunk c + S - 1, its delta part only if it is of this step
+      const int c_refill = c + S - 1;
+      const bool refill_d = it + S - 1 < it_all;
+      const float* Ws = ring + (size_t)(c % S) * WSTAGE_F;
+      const float* Ds = Ws + BWD_TM * KW;
       // the copies that refill a stage are issued between the tensor-core passes
-      warp_chunk_mma<NTN, KS>(acc, Ws + g * LD + kl, LD, Ds + g * LD + kl, LD, [&](int phase) {
-        if (phase == 0) issue_w(c_refill, it_pre, 0, JW / 2);
-        else if (phase == 1) issue_w(c_refill, it_pre, JW / 2, JW);
+      warp_chunk_mma<NTN, KS>(acc, Ws + g * KW + 2 * KS * t, KW, Ds + g * KW + 2 * KS * t, KW, [&](int phase) {
+        if (phase == 0) issue_w(c_refill, it_pre, 0, PW / 2);
+        else if (phase == 1) issue_w(c_refill, it_pre, PW / 2, PW);
         else if (phase == 2) {
           if (refill_d) issue_d(c_refill, it_pre, dn);
           cp_async_commit();
