@@ -525,6 +525,7 @@ struct SegParams {
   int t0;                     // the operation computes steps t0+1 .. from the state of step t0
   int d0, n;                  // this run: steps t0+d0+1 .. t0+d0+n
   int buf_slot, buf_len;      // step t0+d goes to slot buf_slot + (d-1) % buf_len (as in snn_op)
+  int tiles;                  // refwd_gather_kernel: column tiles of the widest layer
 };
 
 constexpr int RG_ROWS = 4;     // weight rows per copy group
@@ -534,11 +535,13 @@ constexpr size_t REFWD_DYN_SMEM = (size_t)RG_STAGES * RG_ROWS * FWD_THREADS * si
 template <bool GRADED>
 __global__ void __launch_bounds__(FWD_THREADS, 4) refwd_gather_kernel(const __grid_constant__ SegParams p) {
   pdl_launch_dependents();
-  const int l = blockIdx.z / p.n, d = p.d0 + 1 + blockIdx.z % p.n;
+  // grid (sample, step, layer x column tile): the thread blocks that run together work on the same 512 columns
+  // of one layer, so whatever the size of the network the rows they gather stay in L2 between them
+  const int l = blockIdx.z / p.tiles, d = p.d0 + 1 + blockIdx.y;
   const SegLayer& L = p.lay[l];
-  const int col0 = blockIdx.x * FWD_COLS;
+  const int col0 = (blockIdx.z % p.tiles) * FWD_COLS;
   if (col0 >= L.N) return;
-  const int b = blockIdx.y, B = p.B, tid = threadIdx.x, t = p.t0 + d;
+  const int b = blockIdx.x, B = p.B, tid = threadIdx.x, t = p.t0 + d;
   __shared__ const float* s_row[LIST_CHUNK];
   __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
   extern __shared__ float4 s_stage[];   // [RG_STAGES][RG_ROWS][FWD_THREADS]

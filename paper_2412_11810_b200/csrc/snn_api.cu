@@ -510,8 +510,8 @@ struct Exec {
   bool reforward_runs_possible(const snn_op& op) const {
     if (a->flags & SNN_FLAG_REFORWARD_PER_STEP) return false;
     if (reforward_rows()) return true;
-    if (!lo.weights_resident) return false;
-    return (long long)L * std::min(op.buf_len, op.t1 - op.t0) <= 65535;
+    if (!lo.weights_resident && !graded()) return false;
+    return (long long)L * fwd_grid().x <= 65535 && std::min(op.buf_len, op.t1 - op.t0) <= 65535;
   }
   // the currents of a run come from refwd_rows_kernel (weight rows stationary) rather than refwd_gather_kernel
   // (spiking cell beyond L2 by default; the graded cell only on request: with values to fetch per event and 10 %
@@ -623,7 +623,8 @@ struct Exec {
       g.d0 = c.d0 = d0; g.n = c.n = n;
       c.v_start = d0 == 0 ? at<float>(lo.slots) + (size_t)op.in_slot * g.slot_stride : c.carry;
       if (!reforward_rows()) {
-        CUDA_TRY(launch_pdl(kg, dim3(fg.x, fg.y, (unsigned)(L * n)), dim3(FWD_THREADS), REFWD_DYN_SMEM, g));
+        g.tiles = (int)fg.x;
+        CUDA_TRY(launch_pdl(kg, dim3((unsigned)B, (unsigned)n, (unsigned)L * fg.x), dim3(FWD_THREADS), REFWD_DYN_SMEM, g));
         ++launches;
       } else if (const snn_status st = launch_reforward_rows(op, d0, n); st != SNN_OK) {
         return st;
