@@ -294,7 +294,7 @@ struct FwdParams {
 };
 
 constexpr int GATHER_ROWS = 8;     // weight rows per copy group
-constexpr int GATHER_STAGES = 5;   // copy groups in flight per thread (40 rows, 80 KB per CTA)
+constexpr int GATHER_STAGES = 3;   // copy groups in flight per thread (24 rows, 48 KB per CTA: four CTAs per SM)
 constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
 template <bool GEN, bool GRADED>
