@@ -492,6 +492,24 @@ __device__ __forceinline__ void cp_async16_or_zero(void* smem_dst, const void* g
                "l"(gmem_src), "r"(real ? 16u : 0u) : "memory");
 }
 
+// L2 eviction priorities for copies that name one: lines fetched with `l2_keep_policy` are the last to be evicted,
+// lines fetched with `l2_stream_policy` the first.
+__device__ __forceinline__ uint64_t l2_keep_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_stream_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// cp_async16_or_zero with an L2 eviction priority
+__device__ __forceinline__ void cp_async16_or_zero_hint(void* smem_dst, const void* gmem_src, bool real, uint64_t policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gmem_src), "r"(real ? 16u : 0u), "l"(policy) : "memory");
+}
+
 // ------------------------------------------------------------------------------------------
 // Re-forward of a run of steps in two launches (the recomputation passes of Sec. 3).
 //
@@ -2114,14 +2132,27 @@ __global__ void __launch_bounds__(32 * BEV_WARPS) bwd_event_kernel(const __grid_
 //
 // With one launch per step the HBM stream of W_rec stops at every step boundary: the next launch cannot start
 // its copies before delta_t is complete.  But the weights do not depend on the step.  Here a CTA (32 rows of
-// W_rec, all samples, the whole contraction range: no cluster) walks through the steps itself and keeps its
-// copy ring busy across the boundary: while the last chunks of step t are multiplied, the W parts of the first
-// chunks of step t-1 are already on their way; only their delta parts wait until every CTA has published
-// its rows of delta_t (one counter of finished (CTA, step) pairs, release add / acquire poll; delta is read
-// past L1).  Tiling, arithmetic and order of additions are those of bwd_step_kernel with a cluster of one:
-// bit-identical results.  Cooperative launch (all CTAs resident); bounded waits.
+// W_rec, all samples, the whole contraction range: no cluster) walks through the steps itself and its copy ring
+// never drains: while the last chunks of step t are multiplied, the W tiles of the first chunks of step t-1 are
+// already on their way; only their delta tiles wait until every CTA has published its rows of delta_t (one counter
+// of finished (CTA, step) pairs, release add / acquire poll).
+//
+// Roles.  One producer thread issues tiled bulk copies (TMA) into a ring of stages: per chunk of 128 contraction
+// values the W tile [32 rows][128] and the delta tile [BP samples][128], each as four boxes of 32 values (128
+// bytes per row, 128-byte swizzle: the fragment loads below are then spread over the banks).  A stage's `full`
+// barrier takes two arrivals, one that announces the bytes of the W tile and one for the delta tile, so the two
+// halves can be issued at different times.  NWARP consumer warps wait for `full`, multiply their own k-steps of the
+// chunk (3-pass TF32 on mma.sync, fragments read straight from the swizzled stage), and arrive on the stage's
+// `empty` barrier.  The consumers execute no copy instruction and no address arithmetic for copies.
+// Tiling, arithmetic and order of additions are those of bwd_step_kernel with a cluster of one: bit-identical
+// results.  Parts of a box outside the matrix arrive as zeros.  Cooperative launch (all CTAs resident); every
+// wait is bounded, and a wait that runs out raises STATUS_SYNC_TIMEOUT: the producer stops issuing, completes the
+// barriers of the stages it had begun and waits for its copies to land; a consumer warp stops waiting and computing
+// but keeps taking part in the CTA's barriers until the launch ends.
 struct BwdStreamParams {
-  const float* W_rec;       // [N][N]
+  CUtensorMap map_w;        // W_rec [N][N], box 32 rows x 32 values, 128-byte swizzle
+  CUtensorMap map_d;        // delta slots of the run [ts_hi][B][N] (slot buf_slot + z at z), box 1 x BP x 32
+  CUtensorMap map_d0;       // delta_{t+1} of the run's latest step [1][B][N], same box
   const float* g_out;       // [B][N] (last layer) or null
   const float* g_ff;        // feed-forward term of the run [n_steps][B][N] (first row: step t0 + ts_lo + 1), or null;
                             // g_ff_parts partial sums over slices of the contraction range, g_ff_stride floats apart
@@ -2136,107 +2167,141 @@ struct BwdStreamParams {
   uint32_t* progress;       // finished (CTA, step) pairs, zero at launch
   int N, B;
   int buf_slot, ts_lo, ts_hi;   // steps ts = ts_hi-1 .. ts_lo; slot buf_slot + ts holds V on entry, delta on exit
+  int keep_chunks;              // the first keep_chunks chunks of 128 contraction values are asked to stay in L2
   float alpha, theta, beta;
   int surrogate, cell;
 };
 
-constexpr int BWD_STREAM_STAGES = 4;   // chunks in flight per warp
+constexpr size_t BWD_STREAM_KEEP_BYTES = (size_t)64 << 20;   // of W_rec kept in L2 across the steps of a run
+
+// stages of the ring: what fits beside the partial tiles with two CTAs per SM (one for the 16-warp instance)
+template <int NTN> __host__ __device__ constexpr int bwd_stream_stages() { return NTN == 2 ? 3 : 4; }
 
 template <int NTN, int NWARP>
 __host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
-  // the warps' copy rings (together BWD_STREAM_STAGES x (32 + BP) rows x 128 values) and their partial tiles
-  return ((size_t)BWD_STREAM_STAGES * (BWD_TM + 8 * NTN) * 128 + (size_t)NWARP * BWD_TM * (8 * NTN + 8)) * sizeof(float);
+  // the ring (stages of a W tile and a delta tile), the warps' partial tiles, and room to align the ring to 1024 bytes
+  return (size_t)bwd_stream_stages<NTN>() * (BWD_TM + 8 * NTN) * 128 * sizeof(float) +
+         (size_t)NWARP * BWD_TM * (8 * NTN + 8) * sizeof(float) + 1024;
 }
 
 template <int NTN, int NWARP>
-__global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
-  // Every warp stages the values of its own k-steps of a chunk (KW adjacent contraction values: 32 rows of W and BP
-  // rows of delta, KW floats each) in a copy ring of its own: no CTA barrier inside the contraction, and the loads,
-  // splits and tensor-core passes of different warps overlap.
-  constexpr int KS = 16 / NWARP, KW = 8 * KS, S = BWD_STREAM_STAGES;
-  constexpr int NT = 32 * NWARP, BP = 8 * NTN, ROWS = BWD_TM + BP, WSTAGE_F = ROWS * KW, TILE = BWD_TM * BP;
+__global__ void __launch_bounds__(32 * (NWARP + 1), NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
+  constexpr int KS = 16 / NWARP, KW = 8 * KS, S = bwd_stream_stages<NTN>();
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, TILE = BWD_TM * BP;
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
   constexpr int EPI = TILE / NT;
-  constexpr int PW = BWD_TM * KW / 4 / 32;   // 16-byte pieces of the W part of a warp's stage per lane
-  constexpr int PD = (BP * KW / 4 + 31) / 32;   // ... of its delta part (the last ones may be past the end)
-  static_assert(TILE % NT == 0 && (BWD_TM * KW / 4) % 32 == 0, "tiles divide evenly among the threads");
+  constexpr uint32_t W_BOX_BYTES = BWD_TM * 128, D_BOX_BYTES = BP * 128;             // one box of 32 values
+  constexpr uint32_t W_TILE_BYTES = 4 * W_BOX_BYTES, STAGE_BYTES = W_TILE_BYTES + 4 * D_BOX_BYTES;
+  static_assert(TILE % NT == 0, "the output tile divides evenly among the consumer threads");
+  static_assert(W_BOX_BYTES % 1024 == 0 && D_BOX_BYTES % 1024 == 0, "every box starts at a multiple of the swizzle period");
   const int tile_row0 = blockIdx.x * BWD_TM;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  __shared__ int s_ok;
-  extern __shared__ float4 s_dyn[];
-  float* const ring = reinterpret_cast<float*>(s_dyn) + (size_t)warp * S * WSTAGE_F;   // [S][ROWS][KW] of this warp
-  float* const s_parts = reinterpret_cast<float*>(s_dyn) + (size_t)NWARP * S * WSTAGE_F;   // [NWARP][32][TS] partial tiles
+  __shared__ uint64_t s_full[S], s_empty[S];
+  __shared__ int s_abort;
+  extern __shared__ unsigned char s_dyn_raw[];
+  unsigned char* const ring = reinterpret_cast<unsigned char*>(((uintptr_t)s_dyn_raw + 1023) & ~(uintptr_t)1023);
+  float* const s_parts = reinterpret_cast<float*>(ring + (size_t)S * STAGE_BYTES);   // [NWARP][32][TS] partial tiles
   const int N = p.N, it_all = (N + 127) / 128, n_steps = p.ts_hi - p.ts_lo;
   const int total = n_steps * it_all;                                 // chunks of the whole run
-  const int rlast = N - 1, blast = p.B - 1;
-  // fixed copy positions of this lane: piece q = lane + 32 j is row q / (KW / 4), values 4 (q % (KW / 4)) ..
-  const float* src_w[PW];
-  int d_row[PD], w_off[PW], d_off[PD], w_k[PW], d_k[PD];
-#pragma unroll
-  for (int j = 0; j < PW; ++j) {
-    const int q = lane + 32 * j, rr = q / (KW / 4), part = q % (KW / 4);
-    w_k[j] = warp * KW + 4 * part;
-    w_off[j] = rr * KW + 4 * part;
-    const size_t row = tile_row0 + rr < rlast ? tile_row0 + rr : rlast;   // rows past the end: a valid one, never used
-    src_w[j] = p.W_rec + row * N + w_k[j];
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(s_full + s, 2); mbar_init(s_empty + s, NWARP); }
+    mbar_fence_init();
+    s_abort = 0;
   }
+  __syncthreads();
+
+  if (warp == NWARP) {
+    // ---- producer: one thread keeps the ring full
+    if (lane != 0) return;
+    const uint64_t pol_keep = l2_keep_policy(), pol_stream = l2_stream_policy();
+    // The matrix is read once per step and is larger than L2, so left to itself every step would fetch all of it
+    // from HBM.  The first keep_chunks chunks are fetched with the lowest eviction priority and the others with the
+    // highest: that part of the matrix is still in L2 when the next step asks for it.
+    int c_d = 0;          // chunks [0, c_d) have their delta tile issued; chunks [c_d, c) only their W tile
+    int s_known = 0;      // delta_{t+1} is known to be complete for the steps 0 .. s_known of the run
+    int st = 0, it = 0, s_of_c = 0;                  // stage, index within its step and step of chunk c
+    int st_d = 0, it_d = 0, s_of_d = 0;              // the same for chunk c_d
+    uint32_t round = 0;                              // c / S: chunk c waits for the `empty` phase round - 1 of its stage
+    bool ok = true;
+    auto issue_delta = [&]() {                       // delta tile of chunk c_d
+      uint64_t* const bar = s_full + st_d;
+      unsigned char* const dst = ring + (size_t)st_d * STAGE_BYTES + W_TILE_BYTES;
+      mbar_arrive_expect_tx(bar, 4 * D_BOX_BYTES);
+      const CUtensorMap* const map = s_of_d == 0 ? &p.map_d0 : &p.map_d;
+      const int z = s_of_d == 0 ? 0 : p.ts_hi - s_of_d;
 #pragma unroll
-  for (int j = 0; j < PD; ++j) {
-    const int q = lane + 32 * j, rr = q / (KW / 4), part = q % (KW / 4);
-    d_k[j] = rr < BP ? warp * KW + 4 * part : -1;
-    d_off[j] = (BWD_TM + rr) * KW + 4 * part;
-    d_row[j] = rr < blast ? rr : blast;
+      for (int q = 0; q < 4; ++q) tma_load_3d(dst + q * D_BOX_BYTES, map, it_d * 128 + 32 * q, 0, z, bar);
+      ++c_d;
+      st_d = st_d + 1 == S ? 0 : st_d + 1;
+      if (++it_d == it_all) { it_d = 0; ++s_of_d; }
+    };
+    // every CTA has written its rows of delta_{t+1} of step s of the run
+    auto step_ready = [&](int s) {
+      if (s <= s_known) return true;
+      if (!wait_progress(p.progress, (uint32_t)gridDim.x * (uint32_t)s)) return false;
+      fence_proxy_async_all();   // the other CTAs' stores, seen through the counter, before the copies that read them
+      s_known = s;
+      return true;
+    };
+    for (int c = 0; c < total && ok; ++c) {
+      if (c >= S) {
+        // the stage is free once chunk c - S is consumed, which needs that chunk's delta tile: if it is still
+        // missing its step has to be ready now, and the other chunks that wait for the same step go with it
+        if (c_d <= c - S) {
+          ok = step_ready(s_of_d);
+          while (ok && c_d < c && s_of_d <= s_known) issue_delta();
+        }
+        if (ok) ok = mbar_wait(s_empty + st, (round - 1u) & 1u);
+        if (!ok) break;
+      }
+      uint64_t* const bar = s_full + st;
+      unsigned char* const dst = ring + (size_t)st * STAGE_BYTES;
+      mbar_arrive_expect_tx(bar, W_TILE_BYTES);
+      const uint64_t pol = it < p.keep_chunks ? pol_keep : pol_stream;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tma_load_2d_hint(dst + q * W_BOX_BYTES, &p.map_w, it * 128 + 32 * q, tile_row0, bar, pol);
+      // delta tiles of the chunks whose step is known to be ready follow at once
+      while (c_d <= c && s_of_d <= s_known) issue_delta();
+      if (++st == S) { st = 0; ++round; }
+      if (++it == it_all) { it = 0; ++s_of_c; }
+    }
+    // the delta tiles of the last chunks (their W tiles are all issued)
+    while (ok && c_d < total) {
+      ok = step_ready(s_of_d);
+      if (ok) issue_delta();
+    }
+    if (!ok) {
+      // give up: complete the barriers of the stages that have a W tile but no delta tile, then wait for the copies
+      atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+      s_abort = 1;
+      const int c_w = s_of_c * it_all + it;          // chunks [0, c_w) have their W tile issued
+      for (int c = c_d; c < c_w; ++c) mbar_arrive(s_full + c % S);
+      for (int c = c_w > S ? c_w - S : 0; c < c_w; ++c) mbar_wait(s_full + c % S, (uint32_t)(c / S) & 1u);
+    }
+    return;
   }
+
+  // ---- consumers
+  // this lane's fragment position inside a box: row g, values k_lane .. of the chunk (k_lane = KW warp + 2 KS t),
+  // i.e. box k_lane / 32, 16-byte piece (k_lane % 32) / 4 exchanged with piece ^ (row % 8) by the swizzle
+  const int k_lane = KW * warp + 2 * KS * t;
+  const int frag = g * 32 + ((((k_lane & 31) >> 2) ^ g) << 2) + (k_lane & 3);   // floats; rows g + 8 r share row % 8
+  const int w_off = (k_lane >> 5) * (W_BOX_BYTES / 4) + frag, d_off = (int)(W_TILE_BYTES / 4) + (k_lane >> 5) * (D_BOX_BYTES / 4) + frag;
+  auto consumer_barrier = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); };
   // delta_{t+1} of the s-th step of the run (s = 0: the latest)
   auto dn_of = [&](int s) -> const float* {
     return s == 0 ? p.d_first : p.slots + (size_t)(p.buf_slot + p.ts_hi - s) * p.slot_stride + p.state_off;
   };
-  // W part of this warp's share of chunk c (the `it`-th of its step), pieces [j0, j1)
-  auto issue_w = [&](int c, int it, int j0, int j1) {
-    if (c < total) {
-      const int k0 = it * 128;
-      float* st = ring + (size_t)(c % S) * WSTAGE_F;
-#pragma unroll
-      for (int j = 0; j < PW; ++j) {
-        if (j < j0 || j >= j1) continue;
-        cp_async16_or_zero(st + w_off[j], k0 + w_k[j] < N ? src_w[j] + k0 : p.W_rec, k0 + w_k[j] < N);
-      }
-    }
-  };
-  // delta part of this warp's share of chunk c (the `it`-th of its step)
-  auto issue_d = [&](int c, int it, const float* dn) {
-    const int k0 = it * 128;
-    float* st = ring + (size_t)(c % S) * WSTAGE_F;
-#pragma unroll
-    for (int j = 0; j < PD; ++j) {
-      if (d_k[j] < 0) continue;
-      const bool real = k0 + d_k[j] < N;
-      cp_async16_or_zero(st + d_off[j], real ? dn + (size_t)d_row[j] * N + d_k[j] + k0 : p.W_rec, real);
-    }
-  };
-  // the W parts of the first chunks: they do not depend on anything this launch computes
-  int it_pre = 0;   // index within its step of the next chunk whose W part is issued (chunks wrap around the steps)
-  for (int c = 0; c < S - 1; ++c) {
-    issue_w(c, it_pre, 0, PW);
-    cp_async_commit();
-    if (++it_pre == it_all) it_pre = 0;
-  }
-
+  bool dead = false;   // a wait of this warp ran out: no more waiting or computing, only the CTA's barriers
+  int st = 0;
+  uint32_t ph_full = 0;
   for (int s = 0; s < n_steps; ++s) {
     const int ts = p.ts_hi - 1 - s;
-    if (s > 0) {   // every CTA has written its rows of delta_{t+1}
-      if (tid == 0) {
-        const bool ok = wait_progress(p.progress, (uint32_t)gridDim.x * (uint32_t)s);
-        if (!ok) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
-        s_ok = ok ? 1 : 0;
-      }
-      __syncthreads();
-      if (!s_ok) { cp_async_wait<0>(); return; }
-    }
     const float* const dn = dn_of(s);
     float* const Vd = p.slots + (size_t)(p.buf_slot + ts) * p.slot_stride + p.state_off;
     const float* const gff = p.g_ff ? p.g_ff + (size_t)(ts - p.ts_lo) * p.B * N : nullptr;
-    // what the epilogue needs, fetched now (delta_{t+1} may come from another CTA of this launch: past L1)
+    // what the epilogue needs, fetched now.  The rows of delta_{t+1} read here are this CTA's own (written before
+    // the barrier that ended the previous step); the first step's come from before the launch.
     float pre_dn[EPI], pre_go[EPI], pre_gf[EPI], pre_v[EPI];
 #pragma unroll
     for (int j = 0; j < EPI; ++j) {
@@ -2253,10 +2318,6 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
         pre_v[j] = Vd[k];
       }
     }
-    // delta parts of the chunks of this step whose W part is already in flight
-    const int c0 = s * it_all;
-    for (int cc = 0; cc < S - 1 && cc < it_all; ++cc) issue_d(c0 + cc, cc, dn);
-    cp_async_commit();
     float acc[2][NTN][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
@@ -2264,26 +2325,19 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
       for (int nt = 0; nt < NTN; ++nt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
-    for (int it = 0; it < it_all; ++it) {
-      const int c = c0 + it;
-      if (it == 0) cp_async_wait<0>();   // the delta parts issued just above are the latest group
-      else cp_async_wait<S - 2>();        // this lane's copies of chunk c have landed
-      __syncwarp();                      // ... the whole warp's have, and the warp is done with chunk c-1
-      // refill of the stage chunk c-1 used: chunk c + S - 1, its delta part only if it is of this step
-      const int c_refill = c + S - 1;
-      const bool refill_d = it + S - 1 < it_all;
-      const float* Ws = ring + (size_t)(c % S) * WSTAGE_F;
-      const float* Ds = Ws + BWD_TM * KW;
-      // the copies that refill a stage are issued between the tensor-core passes
-      warp_chunk_mma<NTN, KS>(acc, Ws + g * KW + 2 * KS * t, KW, Ds + g * KW + 2 * KS * t, KW, [&](int phase) {
-        if (phase == 0) issue_w(c_refill, it_pre, 0, PW / 2);
-        else if (phase == 1) issue_w(c_refill, it_pre, PW / 2, PW);
-        else if (phase == 2) {
-          if (refill_d) issue_d(c_refill, it_pre, dn);
-          cp_async_commit();
+    if (!dead) {
+      for (int it = 0; it < it_all; ++it) {
+        if (!mbar_wait(s_full + st, ph_full)) {
+          if (lane == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+          dead = true;
+          break;
         }
-      });
-      if (++it_pre == it_all) it_pre = 0;
+        const float* const stage = reinterpret_cast<const float*>(ring + (size_t)st * STAGE_BYTES);
+        warp_chunk_mma<NTN, KS>(acc, stage + w_off, 32, stage + d_off, 32, [](int) {});
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_empty + st);
+        if (++st == S) { st = 0; ph_full ^= 1u; }
+      }
     }
     // the warps' partial tiles, summed in warp order
     {
@@ -2297,14 +2351,15 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
           *reinterpret_cast<float2*>(mine + (r + 8) * TS + cc) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
         }
     }
-    __syncthreads();
+    consumer_barrier();
+    if (s_abort) dead = true;
 #pragma unroll
     for (int j = 0; j < EPI; ++j) {
       const int e = tid + j * NT, i = tile_row0 + e / BP, b = e % BP;
       float sum = 0.f;
 #pragma unroll
       for (int w = 0; w < NWARP; ++w) sum += s_parts[(size_t)w * TILEP + (e / BP) * TS + e % BP];
-      if (i < N && b < p.B) {
+      if (i < N && b < p.B && !dead) {
         const size_t k = (size_t)b * N + i;
         float gs = sum + pre_go[j];
         if (gff) gs += pre_gf[j];
@@ -2315,10 +2370,10 @@ __global__ void __launch_bounds__(32 * NWARP, NWARP == 8 ? 2 : 1) bwd_stream_ker
         if (ts == 0 && p.carry_out) p.carry_out[k] = dl;
       }
     }
-    __syncthreads();   // delta_t of this CTA is written, and the partial tiles are free again
+    fence_proxy_async_all();   // these stores before the other CTAs' bulk copies that the counter lets go
+    consumer_barrier();        // delta_t of this CTA is written, and the partial tiles are free again
     if (tid == 0) publish_progress(p.progress);
   }
-  cp_async_wait<0>();
 }
 
 // ------------------------------------------------------------------------------------------

@@ -932,17 +932,31 @@ struct Exec {
 
   // Steps ts_hi-1 .. ts_lo of one layer in one cooperative launch (bwd_stream_kernel), if the device holds all
   // its CTAs at once; otherwise `done` stays false and the caller launches step by step.
-  template <int NTN, int NWARP> snn_status try_backward_stream(const BwdStreamParams& sp, int tiles, bool& done) {
+  CUtensorMap wrec_map[MAXL];      // W_rec of a layer as boxes of 32 rows x 32 values: 0 not tried yet, 1 ready, -1 not encodable
+  int wrec_map_ready[MAXL] = {0};
+  template <int NTN, int NWARP> snn_status try_backward_stream(BwdStreamParams& sp, int l, int tiles, bool& done) {
     done = false;
     void (*k)(BwdStreamParams) = bwd_stream_kernel<NTN, NWARP>;
     const size_t smem = bwd_stream_smem_bytes<NTN, NWARP>();
+    // tensor maps: the matrix once per step of the executor, the deltas of this run (strides must be multiples of 16 bytes)
+    if (sp.N % 4 != 0 || sp.slot_stride % 4 != 0) return SNN_OK;
+    if (wrec_map_ready[l - 1] == 0)
+      wrec_map_ready[l - 1] = make_tensor_map_2d(&wrec_map[l - 1], a->W_rec[l - 1], (uint64_t)sp.N, (uint64_t)sp.N, (uint64_t)sp.N,
+                                                 BWD_TM, 32, true) ? 1 : -1;
+    if (wrec_map_ready[l - 1] < 0) return SNN_OK;
+    sp.map_w = wrec_map[l - 1];
+    if (!make_tensor_map_3d(&sp.map_d, sp.slots + (size_t)sp.buf_slot * sp.slot_stride + sp.state_off, (uint64_t)sp.N, (uint64_t)sp.B,
+                            (uint64_t)sp.ts_hi, (uint64_t)sp.N, (uint64_t)sp.slot_stride, 32, 8 * NTN, 1) ||
+        !make_tensor_map_3d(&sp.map_d0, sp.d_first, (uint64_t)sp.N, (uint64_t)sp.B, 1, (uint64_t)sp.N, (uint64_t)sp.slot_stride, 32,
+                            8 * NTN, 1))
+      return SNN_OK;
     int& cap = net->bwd_stream_capacity[NTN == 1 ? 0 : NTN == 2 ? 1 : 2];
     if (cap < 0) {
       int dev = 0, sms = 0, per_sm = 0, coop = 0;
       if (cudaGetDevice(&dev) != cudaSuccess ||
           cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
           cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, 32 * NWARP, smem) != cudaSuccess) {
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, 32 * (NWARP + 1), smem) != cudaSuccess) {
         cudaGetLastError();
         cap = 0;
       } else {
@@ -952,7 +966,7 @@ struct Exec {
     if (tiles > cap) return SNN_OK;
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4, main));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)tiles); cfg.blockDim = dim3(32 * NWARP); cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cfg.gridDim = dim3((unsigned)tiles); cfg.blockDim = dim3(32 * (NWARP + 1)); cfg.dynamicSmemBytes = smem; cfg.stream = main;
     cudaLaunchAttribute at1[1];
     at1[0].id = cudaLaunchAttributeCooperative;
     at1[0].val.cooperative = 1;
@@ -1063,7 +1077,6 @@ struct Exec {
           if (CS_l == 1 && B <= 32 && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
             BwdStreamParams sp;
             std::memset(&sp, 0, sizeof sp);
-            sp.W_rec = a->W_rec[l - 1];
             sp.g_out = l == L ? at<float>(lo.g_out) : nullptr;
             sp.g_ff = l < L ? at<float>(lo.gff) : nullptr;
             sp.g_ff_parts = gff_parts; sp.g_ff_stride = lo.gff_stride;
@@ -1072,13 +1085,15 @@ struct Exec {
             sp.slots = at<float>(lo.slots); sp.slot_stride = lo.state_bytes / 4; sp.state_off = lo.layer_off[l];
             sp.status = at<uint32_t>(lo.status); sp.progress = at<uint32_t>(lo.progress);
             sp.N = sz[l]; sp.B = B; sp.buf_slot = op.buf_slot; sp.ts_lo = lo_s; sp.ts_hi = hi;
+            // part of W_rec asked to stay in L2 from one step to the next: whole chunks of 128 columns
+            sp.keep_chunks = (int)std::min<size_t>((size_t)(sz[l] + 127) / 128, BWD_STREAM_KEEP_BYTES / ((size_t)sz[l] * 512));
             sp.alpha = net->alpha; sp.theta = net->theta; sp.beta = net->beta;
             sp.surrogate = net->surrogate; sp.cell = net->cell;
             bool done = false;
             snn_status st = SNN_OK;
-            if (B <= 8) st = try_backward_stream<1, 8>(sp, tiles_l, done);
-            else if (B <= 16) st = try_backward_stream<2, 8>(sp, tiles_l, done);
-            else st = try_backward_stream<4, 16>(sp, tiles_l, done);
+            if (B <= 8) st = try_backward_stream<1, 8>(sp, l, tiles_l, done);
+            else if (B <= 16) st = try_backward_stream<2, 8>(sp, l, tiles_l, done);
+            else st = try_backward_stream<4, 16>(sp, l, tiles_l, done);
             if (st != SNN_OK) return st;
             if (done) continue;
           }
