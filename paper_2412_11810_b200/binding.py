@@ -30,6 +30,8 @@ SNN_FLAG_REFORWARD_ROWS = 512
 SNN_FLAG_FF_PRODUCT_MMA_SYNC = 1024
 SNN_FLAG_SPILL_EVENTS = 2048
 SNN_FLAG_BACKWARD_EVENT_DRIVEN = 4096
+SNN_FLAG_WEIGHT_GRADIENT_GATHER = 8192
+SNN_FLAG_WEIGHT_GRADIENT_SLAB = 16384
 PHASE_NAMES = ["fwd", "refwd1", "refwd2", "bwd", "dw", "readout", "d2h", "h2d", "ffgemm"]
 SNN_OP_FWD, SNN_OP_REFWD1, SNN_OP_REFWD2, SNN_OP_BWD, SNN_OP_D2H, SNN_OP_H2D, SNN_OP_ZERO = range(7)
 STRATEGY_NAMES = {SNN_STANDARD: "standard", SNN_CHUNK: "chunk", SNN_REMOTE: "remote", SNN_DOUBLE: "double",

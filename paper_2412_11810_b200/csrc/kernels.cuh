@@ -2905,6 +2905,133 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------
+// The same weight gradient with the deltas as the stationary operand (spiking cell, large layers).
+//
+// dw_kernel fetches a delta row from L2 once per event: on a network whose layers are thousands wide that is
+// several times the bytes of dW itself and the L2 gather sets the time.  Here a CTA owns a slab of DWS_COLS
+// columns and a group of DWS_ROWS presynaptic rows.  Per window of DWS_PAIRS (t, b) pairs it copies the slab
+// delta[pair][columns] into shared memory once (128 KB) together with the spike words of its rows, and then every
+// warp walks through rows of the group: the row's firing pattern over the window's pairs comes from four ballots
+// over the spike words, the row's values of dW are read (the next rows of the warp already on their way), the slab
+// rows of the pairs in which it fired are added in pair order (two 16-byte shared-memory reads and four packed
+// additions per lane and event), and the row is written back.  Rows that did not fire in the window are not written.
+// Per element the additions are those of dw_kernel in the same order (t descending, b ascending, starting from
+// the stored value; a store and a reload between two windows do not change an fp32 value): the same bits.
+// One CTA of 32 warps per SM: the event loop is bound by instruction issue, and a lane that owns eight columns
+// halves the instructions per byte of a lane that owns four (measured on the largest benchmark network, per train
+// step: 101 ms gathering, 91 ms with 128-column slabs, 58 ms with 256-column slabs and 32 warps).
+constexpr int DWS_V = 2;          // 16-byte pieces of a row per lane
+constexpr int DWS_COLS = 128 * DWS_V;   // columns per CTA
+constexpr int DWS_PAIRS = 128;    // (t, b) pairs per window
+constexpr int DWS_ROWS = 1024;    // presynaptic rows per CTA
+constexpr int DWS_WARPS = 32;
+constexpr int DWS_BATCH = 2;      // rows of a warp whose dW values are in flight together (twice that with the prefetch)
+constexpr size_t DWS_SMEM = (size_t)DWS_PAIRS * DWS_COLS * sizeof(float) + (size_t)(DWS_ROWS / 32) * DWS_PAIRS * sizeof(uint32_t);
+
+__global__ void __launch_bounds__(32 * DWS_WARPS) dw_slab_kernel(const __grid_constant__ DwParams p) {
+  pdl_launch_dependents();
+  const DwArgs& a = p.m[blockIdx.z];
+  const int col0 = blockIdx.x * DWS_COLS, row0 = blockIdx.y * DWS_ROWS;
+  if (row0 >= a.N_pre || col0 >= a.N) return;
+  pdl_wait();
+  extern __shared__ float4 s_slab[];   // [DWS_PAIRS][DWS_V][32] float4, then the spike words [DWS_ROWS / 32][DWS_PAIRS]
+  uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_slab + (size_t)DWS_PAIRS * DWS_V * 32);
+  __shared__ uint32_t s_pair_row[DWS_PAIRS];   // (step, sample) row index ts * B + b of the window's pairs
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int B = p.B, n_steps = p.n_steps, n_pairs = n_steps * B;
+  const int wc0 = row0 >> 5;
+  const int col = col0 + lane * 4;           // this lane's columns: col + 128 v .. + 3, v < DWS_V
+  const int rows_here = a.N_pre - row0 < DWS_ROWS ? a.N_pre - row0 : DWS_ROWS;
+  const uint32_t slab_lane = smem_u32(s_slab) + (uint32_t)lane * 16u;
+  for (int p0 = 0; p0 < n_pairs; p0 += DWS_PAIRS) {
+    const int lim = n_pairs - p0 < DWS_PAIRS ? n_pairs - p0 : DWS_PAIRS;
+    __syncthreads();   // the previous window's readers are done
+    if (tid < DWS_PAIRS) {
+      const int pair = p0 + (tid < lim ? tid : 0);
+      const int ts = n_steps - 1 - pair / B, b = pair % B;      // ts = t - t0 - 1; pairs run t descending, b ascending
+      s_pair_row[tid] = (uint32_t)(ts * B + b);
+    }
+    __syncthreads();
+    for (int pr = warp; pr < DWS_PAIRS; pr += DWS_WARPS) {   // a warp copies whole slab rows
+      const uint32_t rowi = s_pair_row[pr];
+      const float* const src = a.delta0 + (size_t)(rowi / B) * p.slot_stride + (size_t)(rowi % B) * a.N + col;
+#pragma unroll
+      for (int v = 0; v < DWS_V; ++v) {
+        const bool real = pr < lim && col + 128 * v < a.N;
+        cp_async16_or_zero(s_slab + (pr * DWS_V + v) * 32 + lane, real ? src + 128 * v : a.delta0, real);
+      }
+    }
+    cp_async_commit();
+    for (int i = tid; i < (DWS_ROWS / 32) * DWS_PAIRS; i += 32 * DWS_WARPS) {
+      const int jw = i / DWS_PAIRS, pr = i % DWS_PAIRS;
+      uint32_t wd = 0u;
+      if (pr < lim && wc0 + jw < a.Wm) wd = a.mask_row0[(size_t)s_pair_row[pr] * a.Wm + wc0 + jw];
+      s_words[i] = wd;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    // warp w takes rows w, w + DWS_WARPS, ... of the group, DWS_BATCH of them at a time; the dW values of the next
+    // batch are on their way while the current one is added to (rows that turn out not to have fired are read for
+    // nothing, never written)
+    float4 nxt[DWS_BATCH][DWS_V];
+    auto fetch = [&](int r0) {
+#pragma unroll
+      for (int u = 0; u < DWS_BATCH; ++u) {
+        const int r = r0 + u * DWS_WARPS;
+#pragma unroll
+        for (int v = 0; v < DWS_V; ++v) {
+          nxt[u][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (r < rows_here && col + 128 * v < a.N)
+            nxt[u][v] = *reinterpret_cast<const float4*>(a.dW + (size_t)(row0 + r) * a.N + col + 128 * v);
+        }
+      }
+    };
+    fetch(warp);
+    for (int r0 = warp; r0 < rows_here; r0 += DWS_WARPS * DWS_BATCH) {
+      unsigned long long acc[DWS_BATCH][DWS_V][2];   // two fp32 values per register pair
+#pragma unroll
+      for (int u = 0; u < DWS_BATCH; ++u)
+#pragma unroll
+        for (int v = 0; v < DWS_V; ++v) {
+          acc[u][v][0] = (unsigned long long)__float_as_uint(nxt[u][v].x) | ((unsigned long long)__float_as_uint(nxt[u][v].y) << 32);
+          acc[u][v][1] = (unsigned long long)__float_as_uint(nxt[u][v].z) | ((unsigned long long)__float_as_uint(nxt[u][v].w) << 32);
+        }
+      fetch(r0 + DWS_WARPS * DWS_BATCH);
+#pragma unroll
+      for (int u = 0; u < DWS_BATCH; ++u) {
+        const int r = r0 + u * DWS_WARPS;
+        const uint32_t* const wds = s_words + (size_t)((r & (DWS_ROWS - 1)) >> 5) * DWS_PAIRS;
+        bool any = false;
+#pragma unroll
+        for (int w = 0; w < DWS_PAIRS / 32; ++w) {
+          uint32_t bits = __ballot_sync(0xffffffffu, (wds[w * 32 + lane] >> (r & 31)) & 1u);
+          any |= bits != 0u;
+          const uint32_t base = slab_lane + (uint32_t)w * 32u * (DWS_COLS * 4u);
+          while (bits) {   // one event: this lane's pieces of the pair's slab row, two packed additions each
+            const uint32_t q = (uint32_t)__ffs(bits) - 1u;
+            bits &= bits - 1u;
+#pragma unroll
+            for (int v = 0; v < DWS_V; ++v) {
+              unsigned long long d01, d23;
+              lds_2x64(base + q * (DWS_COLS * 4u) + v * 512u, d01, d23);
+              add_f32x2(acc[u][v][0], d01); add_f32x2(acc[u][v][1], d23);
+            }
+          }
+        }
+        if (any && r < rows_here) {
+#pragma unroll
+          for (int v = 0; v < DWS_V; ++v)
+            if (col + 128 * v < a.N)
+              *reinterpret_cast<float4*>(a.dW + (size_t)(row0 + r) * a.N + col + 128 * v) =
+                  make_float4(__uint_as_float((uint32_t)acc[u][v][0]), __uint_as_float((uint32_t)(acc[u][v][0] >> 32)),
+                              __uint_as_float((uint32_t)acc[u][v][1]), __uint_as_float((uint32_t)(acc[u][v][1] >> 32)));
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Readout: logits = scale * c W_out, mean soft-max cross-entropy, and the gradients that
 // leave it.  One small dense product per training step; plain fp32.
 __global__ void __launch_bounds__(256)

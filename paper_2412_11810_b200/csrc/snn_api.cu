@@ -1175,8 +1175,16 @@ struct Exec {
         r.mask_row0 = mask(l, ta);
         if (graded()) { r.off_row0 = off(l, ta); r.pref_row0 = pref(l, ta); r.vals = vals(l); r.cap = lo.cap[l]; }
       }
+      const bool slab = !graded() && !(a->flags & SNN_FLAG_WEIGHT_GRADIENT_GATHER) &&
+                        (!lo.weights_resident || (a->flags & SNN_FLAG_WEIGHT_GRADIENT_SLAB));
+      if (slab) {
+        // the deltas stationary in shared memory, the rows of dW streamed past them (dw_slab_kernel)
+        launch_pdl(dw_slab_kernel, dim3((unsigned)((maxN + DWS_COLS - 1) / DWS_COLS), (unsigned)((maxNpre + DWS_ROWS - 1) / DWS_ROWS), 2u * L),
+                   dim3(32 * DWS_WARPS), DWS_SMEM, d);
+        ++launches;
+      }
       // wider column tiles for wider layers: the per-CTA compaction of the pair lists is amortised over more columns
-      if (maxN >= 1024) launch_dw<8>(d, maxN, maxNpre);
+      else if (maxN >= 1024) launch_dw<8>(d, maxN, maxNpre);
       else if (maxN >= 512) launch_dw<4>(d, maxN, maxNpre);
       else if (maxN >= 256) launch_dw<2>(d, maxN, maxNpre);
       else launch_dw<1>(d, maxN, maxNpre);
@@ -1256,6 +1264,7 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8>, dyn, (int)bwd_stream_smem_bytes<1, 8>()));
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8>, dyn, (int)bwd_stream_smem_bytes<2, 8>()));
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16>, dyn, (int)bwd_stream_smem_bytes<4, 16>()));
+  CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel, dyn, (int)DWS_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, dyn, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, dyn, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, dyn, (int)dw_smem_bytes<4, false>(DW_WINDOW)));

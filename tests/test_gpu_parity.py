@@ -596,6 +596,31 @@ def test_layer_by_layer_backward_as_one_launch_per_run(orc32, B):
     s.close()
 
 
+@pytest.mark.parametrize("B", [5, 32])
+def test_weight_gradient_with_the_deltas_stationary(orc32, B):
+    """Large spiking networks accumulate dW with a slab of the deltas held in shared memory and the rows of dW streamed
+    past it (no gather from L2).  Forced here on a medium network: the bits of the gathering kernel, for segments
+    shorter and longer than a window of 128 pairs (ragged last window), widths that are no multiple of the 128-column
+    slab or the 256-row group, and within tolerance of the oracle; rows no event touched stay exactly zero."""
+    b = sb()
+    w = wl.small(sizes=(70, 644, 300, 9), T=61, B=B, p_in=0.06, g_ff=(2.5, 1.5), g_rec=(1.0, 1.0), seed=47)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    assert all(0.005 < float(x[1:].mean()) < 0.5 for x in ref["S"])
+    s, bits, targets = make_session(w, d)
+    s.train_step(bits, targets, strategy=0, extra_flags=b.SNN_FLAG_WEIGHT_GRADIENT_GATHER)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    f = b.SNN_FLAG_WEIGHT_GRADIENT_SLAB
+    for strat, K, R in [(0, 0, 0), (1, 7, 0), (1, 50, 0), (3, 3, 12)]:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, extra_flags=f)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R)
+    assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
 def test_reforward_as_one_launch_per_segment(orc32):
     """The recomputation passes walk through a whole segment inside one launch (small networks: the
     default), with the input currents gathered per (step, sample) or accumulated with the weight rows
