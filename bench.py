@@ -47,9 +47,10 @@ def read_peaks():
 # the kernel still has that text.  The backward pass of c2 now runs in bwd_segment_kernel, a cooperative launch
 # of thread-block clusters that the profiler cannot launch: no counters, hence no entry.
 NCU_TRAFFIC = {
-    # one launch = 16 steps of one layer: 4,310,053,000 B read + 7,173,888 B written; per layer and step:
-    ("c4", "bwd"): ("bwd_stream_kernel", "ca41333f7fa52ed6e31123c392313300114c5e0e1e0ddab24112db8d45f6252c",
-                    (4310053000 + 7173888) // 16),
+    # one launch = 16 steps of one layer: 3,337,009,000 B read + 6,210,304 B written; per layer and step (less than the
+    # algorithmic bytes: the first 64 MB of the matrix stay in L2 from one step to the next):
+    ("c4", "bwd"): ("bwd_stream_kernel", "19e44b638d5ee27f628c837573444f91372cf28a6a7aa0f01a1a1cbe0da7e4c5",
+                    (3337009000 + 6210304) // 16),
     ("c3", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
                     51018240 + 43264),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
@@ -368,7 +369,7 @@ def run_ours(args, rank, world):
         roof = None
         if per_launch_bytes and ph[dominant][1] > 0:
             kernel = {"fwd": "fwd_step_kernel<true>", "refwd1": "fwd_step_kernel<false>",
-                      "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel", "dw": "dw_kernel"}[dominant]
+                      "refwd2": "fwd_step_kernel<false>", "bwd": "bwd_step_kernel", "dw": "dw_slab_kernel / dw_kernel"}[dominant]
             units = ph[dominant][1]
             if dominant == "fwd" and ph["fwd"][1] < w.T:
                 # small spiking networks: one cooperative launch per forward operation, T steps in all;

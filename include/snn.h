@@ -192,8 +192,8 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
 /* The weight gradient of a segment (the sparse outer product of Methods, "BPTT based SNN training") has two kernels.
  * One gathers, per presynaptic row, the delta rows of the (step, sample) pairs in which it fired; the other keeps a slab
  * of the deltas in shared memory and streams the rows of dW past it, so that dW is read and written once per 128 pairs
- * and nothing is gathered from L2 (the default for the spiking cell when the weights exceed 96 MB).  These flags force
- * one or the other (the graded cell always gathers).  Results are bit-identical either way. */
+ * and nothing is gathered from L2 (the default when the weights exceed 96 MB).  These flags force one or the other.
+ * Results are bit-identical either way. */
 #define SNN_FLAG_WEIGHT_GRADIENT_GATHER 8192u
 #define SNN_FLAG_WEIGHT_GRADIENT_SLAB 16384u
 

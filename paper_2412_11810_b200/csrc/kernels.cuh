@@ -504,11 +504,6 @@ __device__ __forceinline__ uint64_t l2_stream_policy() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
-// cp_async16_or_zero with an L2 eviction priority
-__device__ __forceinline__ void cp_async16_or_zero_hint(void* smem_dst, const void* gmem_src, bool real, uint64_t policy) {
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-               "l"(gmem_src), "r"(real ? 16u : 0u), "l"(policy) : "memory");
-}
 
 // ------------------------------------------------------------------------------------------
 // Re-forward of a run of steps in two launches (the recomputation passes of Sec. 3).
@@ -2773,6 +2768,7 @@ struct DwParams {
   size_t slot_stride;        // floats between consecutive steps (multiple of 4)
   int B, n_steps;
   int window;                // (t, b) pairs compacted at a time: min(n_steps * B rounded up to 32, DW_WINDOW)
+  int slab_rows;             // dw_slab_kernel: presynaptic rows per CTA
 };
 
 constexpr int DW_ROWS = 8;        // rows (warps) per CTA
@@ -2905,7 +2901,7 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------
-// The same weight gradient with the deltas as the stationary operand (spiking cell, large layers).
+// The same weight gradient with the deltas as the stationary operand (large layers).
 //
 // dw_kernel fetches a delta row from L2 once per event: on a network whose layers are thousands wide that is
 // several times the bytes of dW itself and the L2 gather sets the time.  Here a CTA owns a slab of DWS_COLS
@@ -2923,25 +2919,35 @@ __global__ void __launch_bounds__(32 * DW_ROWS) dw_kernel(const __grid_constant_
 constexpr int DWS_V = 2;          // 16-byte pieces of a row per lane
 constexpr int DWS_COLS = 128 * DWS_V;   // columns per CTA
 constexpr int DWS_PAIRS = 128;    // (t, b) pairs per window
-constexpr int DWS_ROWS = 1024;    // presynaptic rows per CTA
+constexpr int DWS_ROWS = 1024;    // presynaptic rows per CTA at most (DwParams::slab_rows: 1024, 512 or 256)
 constexpr int DWS_WARPS = 32;
 constexpr int DWS_BATCH = 2;      // rows of a warp whose dW values are in flight together (twice that with the prefetch)
-constexpr size_t DWS_SMEM = (size_t)DWS_PAIRS * DWS_COLS * sizeof(float) + (size_t)(DWS_ROWS / 32) * DWS_PAIRS * sizeof(uint32_t);
+// shared memory: the slab, the spike words of the row group, and for the graded cell the number of events before each
+// of those words in its (step, sample) list
+template <bool GRADED> constexpr size_t dws_smem_bytes() {
+  return (size_t)DWS_PAIRS * DWS_COLS * sizeof(float) + (size_t)(DWS_ROWS / 32) * DWS_PAIRS * (sizeof(uint32_t) + (GRADED ? sizeof(uint16_t) : 0));
+}
 
+// Graded cell: an event multiplies the delta row by the event's value.  The value of (pair, row) sits in the value pool
+// at the start of the pair's list + the events before the row's spike word + the events before the row inside the word;
+// lane q looks up the value of pair 32 w + q while the ballots are taken, and the event loop hands it round by shuffle.
+template <bool GRADED>
 __global__ void __launch_bounds__(32 * DWS_WARPS) dw_slab_kernel(const __grid_constant__ DwParams p) {
   pdl_launch_dependents();
   const DwArgs& a = p.m[blockIdx.z];
-  const int col0 = blockIdx.x * DWS_COLS, row0 = blockIdx.y * DWS_ROWS;
+  const int col0 = blockIdx.x * DWS_COLS, row0 = blockIdx.y * p.slab_rows;
   if (row0 >= a.N_pre || col0 >= a.N) return;
   pdl_wait();
   extern __shared__ float4 s_slab[];   // [DWS_PAIRS][DWS_V][32] float4, then the spike words [DWS_ROWS / 32][DWS_PAIRS]
   uint32_t* const s_words = reinterpret_cast<uint32_t*>(s_slab + (size_t)DWS_PAIRS * DWS_V * 32);
+  uint16_t* const s_pref = reinterpret_cast<uint16_t*>(s_words + (size_t)(DWS_ROWS / 32) * DWS_PAIRS);   // graded only
   __shared__ uint32_t s_pair_row[DWS_PAIRS];   // (step, sample) row index ts * B + b of the window's pairs
+  __shared__ uint32_t s_pair_off[GRADED ? DWS_PAIRS : 1];   // graded: start of the pair's list in its sample's pool
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, n_steps = p.n_steps, n_pairs = n_steps * B;
   const int wc0 = row0 >> 5;
   const int col = col0 + lane * 4;           // this lane's columns: col + 128 v .. + 3, v < DWS_V
-  const int rows_here = a.N_pre - row0 < DWS_ROWS ? a.N_pre - row0 : DWS_ROWS;
+  const int rows_here = a.N_pre - row0 < p.slab_rows ? a.N_pre - row0 : p.slab_rows;
   const uint32_t slab_lane = smem_u32(s_slab) + (uint32_t)lane * 16u;
   for (int p0 = 0; p0 < n_pairs; p0 += DWS_PAIRS) {
     const int lim = n_pairs - p0 < DWS_PAIRS ? n_pairs - p0 : DWS_PAIRS;
@@ -2950,6 +2956,7 @@ __global__ void __launch_bounds__(32 * DWS_WARPS) dw_slab_kernel(const __grid_co
       const int pair = p0 + (tid < lim ? tid : 0);
       const int ts = n_steps - 1 - pair / B, b = pair % B;      // ts = t - t0 - 1; pairs run t descending, b ascending
       s_pair_row[tid] = (uint32_t)(ts * B + b);
+      if (GRADED) s_pair_off[tid] = a.off_row0[ts * B + b];
     }
     __syncthreads();
     for (int pr = warp; pr < DWS_PAIRS; pr += DWS_WARPS) {   // a warp copies whole slab rows
@@ -2962,11 +2969,16 @@ __global__ void __launch_bounds__(32 * DWS_WARPS) dw_slab_kernel(const __grid_co
       }
     }
     cp_async_commit();
-    for (int i = tid; i < (DWS_ROWS / 32) * DWS_PAIRS; i += 32 * DWS_WARPS) {
+    for (int i = tid; i < (p.slab_rows / 32) * DWS_PAIRS; i += 32 * DWS_WARPS) {
       const int jw = i / DWS_PAIRS, pr = i % DWS_PAIRS;
       uint32_t wd = 0u;
-      if (pr < lim && wc0 + jw < a.Wm) wd = a.mask_row0[(size_t)s_pair_row[pr] * a.Wm + wc0 + jw];
+      uint16_t pf = 0;
+      if (pr < lim && wc0 + jw < a.Wm) {
+        wd = a.mask_row0[(size_t)s_pair_row[pr] * a.Wm + wc0 + jw];
+        if (GRADED) pf = a.pref_row0[(size_t)s_pair_row[pr] * a.Wm + wc0 + jw];
+      }
       s_words[i] = wd;
+      if (GRADED) s_pref[i] = pf;
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -3000,21 +3012,42 @@ __global__ void __launch_bounds__(32 * DWS_WARPS) dw_slab_kernel(const __grid_co
 #pragma unroll
       for (int u = 0; u < DWS_BATCH; ++u) {
         const int r = r0 + u * DWS_WARPS;
-        const uint32_t* const wds = s_words + (size_t)((r & (DWS_ROWS - 1)) >> 5) * DWS_PAIRS;
+        const int jw = (r & (DWS_ROWS - 1)) >> 5;
+        const uint32_t* const wds = s_words + (size_t)jw * DWS_PAIRS;
         bool any = false;
+        uint32_t bits_w[DWS_PAIRS / 32];
+        float val_w[DWS_PAIRS / 32];
 #pragma unroll
         for (int w = 0; w < DWS_PAIRS / 32; ++w) {
-          uint32_t bits = __ballot_sync(0xffffffffu, (wds[w * 32 + lane] >> (r & 31)) & 1u);
-          any |= bits != 0u;
+          const uint32_t wd = wds[w * 32 + lane];
+          const bool on = (wd >> (r & 31)) & 1u;
+          bits_w[w] = __ballot_sync(0xffffffffu, on);
+          any |= bits_w[w] != 0u;
+          val_w[w] = 0.f;
+          if (GRADED && on) {   // the value of this lane's pair for row r
+            const int pr = w * 32 + lane;
+            const uint32_t pos = s_pair_off[pr] + s_pref[jw * DWS_PAIRS + pr] + __popc(wd & ((1u << (r & 31)) - 1u));
+            if (pos < a.cap) val_w[w] = a.vals[(size_t)(s_pair_row[pr] % B) * a.cap + pos];
+          }
+        }
+#pragma unroll
+        for (int w = 0; w < DWS_PAIRS / 32; ++w) {
+          uint32_t bits = bits_w[w];
           const uint32_t base = slab_lane + (uint32_t)w * 32u * (DWS_COLS * 4u);
-          while (bits) {   // one event: this lane's pieces of the pair's slab row, two packed additions each
+          while (bits) {   // one event: this lane's pieces of the pair's slab row, two packed operations each
             const uint32_t q = (uint32_t)__ffs(bits) - 1u;
             bits &= bits - 1u;
+            unsigned long long vv = 0ull;
+            if (GRADED) {
+              const uint32_t sv = __float_as_uint(__shfl_sync(0xffffffffu, val_w[w], (int)q));
+              vv = (unsigned long long)sv | ((unsigned long long)sv << 32);
+            }
 #pragma unroll
             for (int v = 0; v < DWS_V; ++v) {
               unsigned long long d01, d23;
               lds_2x64(base + q * (DWS_COLS * 4u) + v * 512u, d01, d23);
-              add_f32x2(acc[u][v][0], d01); add_f32x2(acc[u][v][1], d23);
+              if (GRADED) { fma_f32x2(acc[u][v][0], d01, vv); fma_f32x2(acc[u][v][1], d23, vv); }
+              else { add_f32x2(acc[u][v][0], d01); add_f32x2(acc[u][v][1], d23); }
             }
           }
         }

@@ -1175,12 +1175,25 @@ struct Exec {
         r.mask_row0 = mask(l, ta);
         if (graded()) { r.off_row0 = off(l, ta); r.pref_row0 = pref(l, ta); r.vals = vals(l); r.cap = lo.cap[l]; }
       }
-      const bool slab = !graded() && !(a->flags & SNN_FLAG_WEIGHT_GRADIENT_GATHER) &&
+      const bool slab = !(a->flags & SNN_FLAG_WEIGHT_GRADIENT_GATHER) &&
                         (!lo.weights_resident || (a->flags & SNN_FLAG_WEIGHT_GRADIENT_SLAB));
       if (slab) {
         // the deltas stationary in shared memory, the rows of dW streamed past them (dw_slab_kernel)
-        launch_pdl(dw_slab_kernel, dim3((unsigned)((maxN + DWS_COLS - 1) / DWS_COLS), (unsigned)((maxNpre + DWS_ROWS - 1) / DWS_ROWS), 2u * L),
-                   dim3(32 * DWS_WARPS), DWS_SMEM, d);
+        // rows per CTA: as many as amortise the copy of the slab, fewer while the grid would not fill the device four
+        // times over (a function of the network alone)
+        const long long slabs = (maxN + DWS_COLS - 1) / DWS_COLS;
+        long long row_units = 0;
+        d.slab_rows = DWS_ROWS;
+        for (;;) {
+          row_units = 0;
+          for (int l = 1; l <= L; ++l)
+            row_units += (sz[l - 1] + d.slab_rows - 1) / d.slab_rows + (sz[l] + d.slab_rows - 1) / d.slab_rows;
+          if (d.slab_rows <= 256 || slabs * row_units >= 4 * 148) break;
+          d.slab_rows /= 2;
+        }
+        const dim3 grid((unsigned)slabs, (unsigned)((maxNpre + d.slab_rows - 1) / d.slab_rows), 2u * L);
+        if (graded()) launch_pdl(dw_slab_kernel<true>, grid, dim3(32 * DWS_WARPS), dws_smem_bytes<true>(), d);
+        else launch_pdl(dw_slab_kernel<false>, grid, dim3(32 * DWS_WARPS), dws_smem_bytes<false>(), d);
         ++launches;
       }
       // wider column tiles for wider layers: the per-CTA compaction of the pair lists is amortised over more columns
@@ -1264,7 +1277,8 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8>, dyn, (int)bwd_stream_smem_bytes<1, 8>()));
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8>, dyn, (int)bwd_stream_smem_bytes<2, 8>()));
   CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16>, dyn, (int)bwd_stream_smem_bytes<4, 16>()));
-  CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel, dyn, (int)DWS_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel<false>, dyn, (int)dws_smem_bytes<false>()));
+  CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel<true>, dyn, (int)dws_smem_bytes<true>()));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, dyn, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<2, false>, dyn, (int)dw_smem_bytes<2, false>(DW_WINDOW)));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<4, false>, dyn, (int)dw_smem_bytes<4, false>(DW_WINDOW)));

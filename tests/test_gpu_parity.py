@@ -621,6 +621,29 @@ def test_weight_gradient_with_the_deltas_stationary(orc32, B):
     s.close()
 
 
+def test_graded_weight_gradient_with_the_deltas_stationary(orc32):
+    """The graded cell on the same kernel: an event multiplies the delta row by its value, looked up in the value pool
+    per (pair, row).  Bits of the gathering kernel, several windows of 128 pairs, ragged sizes, oracle tolerance."""
+    b = sb()
+    w = _graded(sizes=(70, 644, 300, 9), T=45, B=7, seed=53)
+    d = wl.make(w)
+    ref = run_oracle(orc32, w, d)
+    frac = [float((x[1:] != 0).mean()) for x in ref["S"]]
+    assert all(0.05 < f < 0.8 for f in frac), frac
+    s, bits, targets = make_session(w, d)
+    s.train_step(bits, targets, strategy=0, max_activity=1.0, extra_flags=b.SNN_FLAG_WEIGHT_GRADIENT_GATHER)
+    base = _bits(s.dW_ff + s.dW_rec + [s.dW_out])
+    f = b.SNN_FLAG_WEIGHT_GRADIENT_SLAB
+    for strat, K, R in [(0, 0, 0), (1, 7, 0), (3, 5, 20)]:
+        for g in s.dW_ff + s.dW_rec + [s.dW_out]:
+            g.fill_(float("nan"))
+        s.train_step(bits, targets, strategy=strat, chunk_size=K, remote_chunk_size=R, max_activity=1.0, extra_flags=f)
+        for x, y in zip(_bits(s.dW_ff + s.dW_rec + [s.dW_out]), base):
+            assert np.array_equal(x, y), (strat, K, R)
+    assert_grads_close(s.gradients(), ref)
+    s.close()
+
+
 def test_reforward_as_one_launch_per_segment(orc32):
     """The recomputation passes walk through a whole segment inside one launch (small networks: the
     default), with the input currents gathered per (step, sample) or accumulated with the weight rows
