@@ -2132,18 +2132,19 @@ __global__ void __launch_bounds__(32 * BEV_WARPS) bwd_event_kernel(const __grid_
 // already on their way; only their delta tiles wait until every CTA has published its rows of delta_t (one counter
 // of finished (CTA, step) pairs, release add / acquire poll).
 //
-// Roles.  One producer thread issues tiled bulk copies (TMA) into a ring of stages: per chunk of 128 contraction
-// values the W tile [32 rows][128] and the delta tile [BP samples][128], each as four boxes of 32 values (128
-// bytes per row, 128-byte swizzle: the fragment loads below are then spread over the banks).  A stage's `full`
-// barrier takes two arrivals, one that announces the bytes of the W tile and one for the delta tile, so the two
-// halves can be issued at different times.  NWARP consumer warps wait for `full`, multiply their own k-steps of the
+// Roles.  Two producer threads issue tiled bulk copies (TMA) into a ring of stages: per chunk of 128 contraction
+// values one issues the W tile [32 rows][128] and the other the delta tile [BP samples][128], each as four boxes
+// of 32 values (128 bytes per row, 128-byte swizzle: the fragment loads below are then spread over the banks).  A
+// stage's `full` barrier takes two arrivals, one that announces the bytes of the W tile and one for the delta tile,
+// so the two halves are issued at different times: the W side runs ahead across a step boundary, the delta side
+// waits there for the other CTAs.  NWARP consumer warps wait for `full`, multiply their own k-steps of the
 // chunk (3-pass TF32 on mma.sync, fragments read straight from the swizzled stage), and arrive on the stage's
 // `empty` barrier.  The consumers execute no copy instruction and no address arithmetic for copies.
 // Tiling, arithmetic and order of additions are those of bwd_step_kernel with a cluster of one: bit-identical
 // results.  Parts of a box outside the matrix arrive as zeros.  Cooperative launch (all CTAs resident); every
-// wait is bounded, and a wait that runs out raises STATUS_SYNC_TIMEOUT: the producer stops issuing, completes the
-// barriers of the stages it had begun and waits for its copies to land; a consumer warp stops waiting and computing
-// but keeps taking part in the CTA's barriers until the launch ends.
+// wait is bounded, and a wait that runs out raises STATUS_SYNC_TIMEOUT: a producer stops issuing, tells the
+// consumers and waits for its copies to land (the other producer's next wait then runs out too); a consumer warp stops waiting and computing but keeps taking part in the
+// CTA's barriers until the launch ends.
 struct BwdStreamParams {
   CUtensorMap map_w;        // W_rec [N][N], box 32 rows x 32 values, 128-byte swizzle
   CUtensorMap map_d;        // delta slots of the run [ts_hi][B][N] (slot buf_slot + z at z), box 1 x BP x 32
@@ -2180,7 +2181,7 @@ __host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
 }
 
 template <int NTN, int NWARP>
-__global__ void __launch_bounds__(32 * (NWARP + 1), NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
+__global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
   constexpr int KS = 16 / NWARP, KW = 8 * KS, S = bwd_stream_stages<NTN>();
   constexpr int NT = 32 * NWARP, BP = 8 * NTN, TILE = BWD_TM * BP;
   constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
@@ -2205,73 +2206,57 @@ __global__ void __launch_bounds__(32 * (NWARP + 1), NWARP == 8 ? 2 : 1) bwd_stre
   }
   __syncthreads();
 
-  if (warp == NWARP) {
-    // ---- producer: one thread keeps the ring full
+  if (warp >= NWARP) {
+    // ---- producers: one thread for the W tiles, one for the delta tiles.  What bounds the launch is how fast such a
+    // thread gets round its loop, so the loops hold nothing they can do without (one thread issuing both tiles: 46.7 us
+    // per step; two threads: 42.5 us; a look at the abort flag per chunk or both roles in one loop cost 2 to 4 % each).
+    // A producer learns that the launch is failing when one of its own waits runs out.
     if (lane != 0) return;
-    const uint64_t pol_keep = l2_keep_policy(), pol_stream = l2_stream_policy();
-    // The matrix is read once per step and is larger than L2, so left to itself every step would fetch all of it
-    // from HBM.  The first keep_chunks chunks are fetched with the lowest eviction priority and the others with the
-    // highest: that part of the matrix is still in L2 when the next step asks for it.
-    int c_d = 0;          // chunks [0, c_d) have their delta tile issued; chunks [c_d, c) only their W tile
-    int s_known = 0;      // delta_{t+1} is known to be complete for the steps 0 .. s_known of the run
-    int st = 0, it = 0, s_of_c = 0;                  // stage, index within its step and step of chunk c
-    int st_d = 0, it_d = 0, s_of_d = 0;              // the same for chunk c_d
-    uint32_t round = 0;                              // c / S: chunk c waits for the `empty` phase round - 1 of its stage
+    int st = 0, it = 0;          // stage and index within its step of chunk c
+    uint32_t round = 0;          // c / S: chunk c waits for the `empty` phase round - 1 of its stage
+    int c = 0;
     bool ok = true;
-    auto issue_delta = [&]() {                       // delta tile of chunk c_d
-      uint64_t* const bar = s_full + st_d;
-      unsigned char* const dst = ring + (size_t)st_d * STAGE_BYTES + W_TILE_BYTES;
-      mbar_arrive_expect_tx(bar, 4 * D_BOX_BYTES);
-      const CUtensorMap* const map = s_of_d == 0 ? &p.map_d0 : &p.map_d;
-      const int z = s_of_d == 0 ? 0 : p.ts_hi - s_of_d;
+    if (warp == NWARP) {
+      // The matrix is read once per step and is larger than L2, so left to itself every step would fetch all of it
+      // from HBM.  The first keep_chunks chunks are fetched with the lowest eviction priority and the others with the
+      // highest: that part of the matrix is still in L2 when the next step asks for it.
+      const uint64_t pol_keep = l2_keep_policy(), pol_stream = l2_stream_policy();
+      for (; c < total; ++c) {
+        if (c >= S && !mbar_wait(s_empty + st, (round - 1u) & 1u)) { ok = false; break; }   // chunk c - S is consumed
+        uint64_t* const bar = s_full + st;
+        unsigned char* const dst = ring + (size_t)st * STAGE_BYTES;
+        mbar_arrive_expect_tx(bar, W_TILE_BYTES);
+        const uint64_t pol = it < p.keep_chunks ? pol_keep : pol_stream;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tma_load_3d(dst + q * D_BOX_BYTES, map, it_d * 128 + 32 * q, 0, z, bar);
-      ++c_d;
-      st_d = st_d + 1 == S ? 0 : st_d + 1;
-      if (++it_d == it_all) { it_d = 0; ++s_of_d; }
-    };
-    // every CTA has written its rows of delta_{t+1} of step s of the run
-    auto step_ready = [&](int s) {
-      if (s <= s_known) return true;
-      if (!wait_progress(p.progress, (uint32_t)gridDim.x * (uint32_t)s)) return false;
-      fence_proxy_async_all();   // the other CTAs' stores, seen through the counter, before the copies that read them
-      s_known = s;
-      return true;
-    };
-    for (int c = 0; c < total && ok; ++c) {
-      if (c >= S) {
-        // the stage is free once chunk c - S is consumed, which needs that chunk's delta tile: if it is still
-        // missing its step has to be ready now, and the other chunks that wait for the same step go with it
-        if (c_d <= c - S) {
-          ok = step_ready(s_of_d);
-          while (ok && c_d < c && s_of_d <= s_known) issue_delta();
-        }
-        if (ok) ok = mbar_wait(s_empty + st, (round - 1u) & 1u);
-        if (!ok) break;
+        for (int q = 0; q < 4; ++q) tma_load_2d_hint(dst + q * W_BOX_BYTES, &p.map_w, it * 128 + 32 * q, tile_row0, bar, pol);
+        if (++st == S) { st = 0; ++round; }
+        if (++it == it_all) it = 0;
       }
-      uint64_t* const bar = s_full + st;
-      unsigned char* const dst = ring + (size_t)st * STAGE_BYTES;
-      mbar_arrive_expect_tx(bar, W_TILE_BYTES);
-      const uint64_t pol = it < p.keep_chunks ? pol_keep : pol_stream;
+    } else {
+      int s = 0;                 // step of chunk c
+      for (; c < total; ++c) {
+        if (c >= S && !mbar_wait(s_empty + st, (round - 1u) & 1u)) { ok = false; break; }
+        if (it == 0 && s > 0) {  // first chunk of a step: every CTA has written its rows of delta_{t+1}
+          if (!wait_progress(p.progress, (uint32_t)gridDim.x * (uint32_t)s)) { ok = false; break; }
+          fence_proxy_async_all();   // the other CTAs' stores, seen through the counter, before the copies that read them
+        }
+        uint64_t* const bar = s_full + st;
+        unsigned char* const dst = ring + (size_t)st * STAGE_BYTES + W_TILE_BYTES;
+        mbar_arrive_expect_tx(bar, 4 * D_BOX_BYTES);
+        const CUtensorMap* const map = s == 0 ? &p.map_d0 : &p.map_d;
+        const int z = s == 0 ? 0 : p.ts_hi - s;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tma_load_2d_hint(dst + q * W_BOX_BYTES, &p.map_w, it * 128 + 32 * q, tile_row0, bar, pol);
-      // delta tiles of the chunks whose step is known to be ready follow at once
-      while (c_d <= c && s_of_d <= s_known) issue_delta();
-      if (++st == S) { st = 0; ++round; }
-      if (++it == it_all) { it = 0; ++s_of_c; }
-    }
-    // the delta tiles of the last chunks (their W tiles are all issued)
-    while (ok && c_d < total) {
-      ok = step_ready(s_of_d);
-      if (ok) issue_delta();
+        for (int q = 0; q < 4; ++q) tma_load_3d(dst + q * D_BOX_BYTES, map, it * 128 + 32 * q, 0, z, bar);
+        if (++st == S) { st = 0; ++round; }
+        if (++it == it_all) { it = 0; ++s; }
+      }
     }
     if (!ok) {
-      // give up: complete the barriers of the stages that have a W tile but no delta tile, then wait for the copies
+      // give up: raise the status, tell the consumers, and wait (briefly: the copies were issued long ago, and a
+      // barrier whose other half was never issued cannot complete) for the stages this thread has copies in
       atomicOr(p.status, STATUS_SYNC_TIMEOUT);
-      s_abort = 1;
-      const int c_w = s_of_c * it_all + it;          // chunks [0, c_w) have their W tile issued
-      for (int c = c_d; c < c_w; ++c) mbar_arrive(s_full + c % S);
-      for (int c = c_w > S ? c_w - S : 0; c < c_w; ++c) mbar_wait(s_full + c % S, (uint32_t)(c / S) & 1u);
+      *reinterpret_cast<volatile int*>(&s_abort) = 1;
+      for (int cc = c > S ? c - S : 0; cc < c; ++cc) mbar_wait(s_full + cc % S, (uint32_t)(cc / S) & 1u, 1u << 14);
     }
     return;
   }

@@ -956,7 +956,7 @@ struct Exec {
       if (cudaGetDevice(&dev) != cudaSuccess ||
           cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
           cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, 32 * (NWARP + 1), smem) != cudaSuccess) {
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, 32 * (NWARP + 2), smem) != cudaSuccess) {
         cudaGetLastError();
         cap = 0;
       } else {
@@ -966,7 +966,7 @@ struct Exec {
     if (tiles > cap) return SNN_OK;
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4, main));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)tiles); cfg.blockDim = dim3(32 * (NWARP + 1)); cfg.dynamicSmemBytes = smem; cfg.stream = main;
+    cfg.gridDim = dim3((unsigned)tiles); cfg.blockDim = dim3(32 * (NWARP + 2)); cfg.dynamicSmemBytes = smem; cfg.stream = main;
     cudaLaunchAttribute at1[1];
     at1[0].id = cudaLaunchAttributeCooperative;
     at1[0].val.cooperative = 1;
