@@ -1802,16 +1802,16 @@ __host__ __device__ constexpr int bwd_ld(int nwarp) { return nwarp == 8 ? 144 : 
 // load and splits each once; within k-step j the hardware's k slots t and t + 4 take values 2 j and 2 j + 1 of
 // that group, for W and delta alike (the contraction does not care which k sits in which slot as long as both
 // operands agree).  Wl / Dl: this lane's first value in row g of the W tile / the delta tile; further rows of W
-// at multiples of 8 ldw, further sample tiles at multiples of 8 ldd.  Per k-step three passes, small terms
+// at multiples of 8 ldw (2 MT of them: MT tiles of 16 rows), further sample tiles at multiples of 8 ldd.  Per k-step three passes, small terms
 // first; `between(phase)` runs after each pass (phases 0, 1, 2 of the first k-step are where callers issue the
 // copies that refill a stage).
-template <int NTN, int KS, class Between>
-__device__ __forceinline__ void warp_chunk_mma(float (&acc)[2][NTN][4], const float* Wl, int ldw, const float* Dl,
+template <int NTN, int KS, int MT = 2, class Between>
+__device__ __forceinline__ void warp_chunk_mma(float (&acc)[MT][NTN][4], const float* Wl, int ldw, const float* Dl,
                                                int ldd, Between&& between) {
   static_assert(KS == 1 || KS == 2, "one or two k-steps per warp and chunk");
-  uint32_t wh[4][2 * KS], wlo[4][2 * KS], dh[NTN][2 * KS], dlo[NTN][2 * KS];
+  uint32_t wh[2 * MT][2 * KS], wlo[2 * MT][2 * KS], dh[NTN][2 * KS], dlo[NTN][2 * KS];
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
+  for (int r = 0; r < 2 * MT; ++r) {
     float v[2 * KS];
     if (KS == 2) {
       const float4 x = *reinterpret_cast<const float4*>(Wl + (size_t)r * 8 * ldw);
@@ -1838,9 +1838,9 @@ __device__ __forceinline__ void warp_chunk_mma(float (&acc)[2][NTN][4], const fl
   }
 #pragma unroll
   for (int j = 0; j < KS; ++j) {
-    uint32_t a_hi[2][4], a_lo[2][4], b_hi[NTN][2], b_lo[NTN][2];
+    uint32_t a_hi[MT][4], a_lo[MT][4], b_hi[NTN][2], b_lo[NTN][2];
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {   // rows mt 16 + g (loaded row 2 mt) and mt 16 + g + 8 (loaded row 2 mt + 1)
+    for (int mt = 0; mt < MT; ++mt) {   // rows mt 16 + g (loaded row 2 mt) and mt 16 + g + 8 (loaded row 2 mt + 1)
       a_hi[mt][0] = wh[2 * mt][2 * j];     a_hi[mt][1] = wh[2 * mt + 1][2 * j];
       a_hi[mt][2] = wh[2 * mt][2 * j + 1]; a_hi[mt][3] = wh[2 * mt + 1][2 * j + 1];
       a_lo[mt][0] = wlo[2 * mt][2 * j];     a_lo[mt][1] = wlo[2 * mt + 1][2 * j];
@@ -1852,17 +1852,17 @@ __device__ __forceinline__ void warp_chunk_mma(float (&acc)[2][NTN][4], const fl
       b_lo[nt][0] = dlo[nt][2 * j]; b_lo[nt][1] = dlo[nt][2 * j + 1];
     }
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_lo[mt], b_hi[nt]);
     between(3 * j);
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_lo[nt]);
     between(3 * j + 1);
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NTN; ++nt) mma_tf32(acc[mt][nt], a_hi[mt], b_hi[nt]);
     between(3 * j + 2);
@@ -2141,7 +2141,9 @@ __global__ void __launch_bounds__(32 * BEV_WARPS) bwd_event_kernel(const __grid_
 // chunk (3-pass TF32 on mma.sync, fragments read straight from the swizzled stage), and arrive on the stage's
 // `empty` barrier.  The consumers execute no copy instruction and no address arithmetic for copies.
 // Tiling, arithmetic and order of additions are those of bwd_step_kernel with a cluster of one: bit-identical
-// results.  Parts of a box outside the matrix arrive as zeros.  Cooperative launch (all CTAs resident); every
+// results.  Parts of a box outside the matrix arrive as zeros.  When N is a multiple of 32 the tensor maps see the
+// contraction index as [N / 32][32] and a tile is one copy instead of four (the producers' trips round their loops
+// bound the launch, above all with tiles of 16 rows).  Cooperative launch (all CTAs resident); every
 // wait is bounded, and a wait that runs out raises STATUS_SYNC_TIMEOUT: a producer stops issuing, tells the
 // consumers and waits for its copies to land (the other producer's next wait then runs out too); a consumer warp stops waiting and computing but keeps taking part in the
 // CTA's barriers until the launch ends.
@@ -2164,6 +2166,8 @@ struct BwdStreamParams {
   int N, B;
   int buf_slot, ts_lo, ts_hi;   // steps ts = ts_hi-1 .. ts_lo; slot buf_slot + ts holds V on entry, delta on exit
   int keep_chunks;              // the first keep_chunks chunks of 128 contraction values are asked to stay in L2
+  int one_copy;                 // N is a multiple of 32: the maps see the contraction index as [N / 32][32] and a tile is ONE
+                                // copy (map_w [N / 32][N rows][32], box 4 x 16 MT x 32; map_d, map_d0 [slots][N / 32][B][32])
   float alpha, theta, beta;
   int surrogate, cell;
 };
@@ -2171,26 +2175,29 @@ struct BwdStreamParams {
 constexpr size_t BWD_STREAM_KEEP_BYTES = (size_t)64 << 20;   // of W_rec kept in L2 across the steps of a run
 
 // stages of the ring: what fits beside the partial tiles with two CTAs per SM (one for the 16-warp instance)
-template <int NTN> __host__ __device__ constexpr int bwd_stream_stages() { return NTN == 2 ? 3 : 4; }
-
-template <int NTN, int NWARP>
-__host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
-  // the ring (stages of a W tile and a delta tile), the warps' partial tiles, and room to align the ring to 1024 bytes
-  return (size_t)bwd_stream_stages<NTN>() * (BWD_TM + 8 * NTN) * 128 * sizeof(float) +
-         (size_t)NWARP * BWD_TM * (8 * NTN + 8) * sizeof(float) + 1024;
+template <int NTN, int MT> __host__ __device__ constexpr int bwd_stream_stages() {
+  return MT == 2 ? (NTN == 2 ? 3 : 4) : (NTN == 2 ? 5 : 6);
 }
 
-template <int NTN, int NWARP>
+// MT = tiles of 16 rows per CTA: 2 where that still gives every SM a CTA, else 1 (twice the CTAs for layers half as wide)
+template <int NTN, int NWARP, int MT>
+__host__ __device__ constexpr size_t bwd_stream_smem_bytes() {
+  // the ring (stages of a W tile and a delta tile), the warps' partial tiles, and room to align the ring to 1024 bytes
+  return (size_t)bwd_stream_stages<NTN, MT>() * (16 * MT + 8 * NTN) * 128 * sizeof(float) +
+         (size_t)NWARP * 16 * MT * (8 * NTN + 8) * sizeof(float) + 1024;
+}
+
+template <int NTN, int NWARP, int MT>
 __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stream_kernel(const __grid_constant__ BwdStreamParams p) {
-  constexpr int KS = 16 / NWARP, KW = 8 * KS, S = bwd_stream_stages<NTN>();
-  constexpr int NT = 32 * NWARP, BP = 8 * NTN, TILE = BWD_TM * BP;
-  constexpr int TS = BP + 8, TILEP = BWD_TM * TS;
-  constexpr int EPI = TILE / NT;
-  constexpr uint32_t W_BOX_BYTES = BWD_TM * 128, D_BOX_BYTES = BP * 128;             // one box of 32 values
+  constexpr int KS = 16 / NWARP, KW = 8 * KS, S = bwd_stream_stages<NTN, MT>();
+  constexpr int TM = 16 * MT;                                                         // rows per CTA
+  constexpr int NT = 32 * NWARP, BP = 8 * NTN, TILE = TM * BP;
+  constexpr int TS = BP + 8, TILEP = TM * TS;
+  constexpr int EPI = (TILE + NT - 1) / NT;
+  constexpr uint32_t W_BOX_BYTES = TM * 128, D_BOX_BYTES = BP * 128;                  // one box of 32 values
   constexpr uint32_t W_TILE_BYTES = 4 * W_BOX_BYTES, STAGE_BYTES = W_TILE_BYTES + 4 * D_BOX_BYTES;
-  static_assert(TILE % NT == 0, "the output tile divides evenly among the consumer threads");
   static_assert(W_BOX_BYTES % 1024 == 0 && D_BOX_BYTES % 1024 == 0, "every box starts at a multiple of the swizzle period");
-  const int tile_row0 = blockIdx.x * BWD_TM;
+  const int tile_row0 = blockIdx.x * TM;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   __shared__ uint64_t s_full[S], s_empty[S];
   __shared__ int s_abort;
@@ -2227,8 +2234,12 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
         unsigned char* const dst = ring + (size_t)st * STAGE_BYTES;
         mbar_arrive_expect_tx(bar, W_TILE_BYTES);
         const uint64_t pol = it < p.keep_chunks ? pol_keep : pol_stream;
+        if (p.one_copy) {
+          tma_load_3d_hint(dst, &p.map_w, 0, tile_row0, it * 4, bar, pol);
+        } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tma_load_2d_hint(dst + q * W_BOX_BYTES, &p.map_w, it * 128 + 32 * q, tile_row0, bar, pol);
+          for (int q = 0; q < 4; ++q) tma_load_2d_hint(dst + q * W_BOX_BYTES, &p.map_w, it * 128 + 32 * q, tile_row0, bar, pol);
+        }
         if (++st == S) { st = 0; ++round; }
         if (++it == it_all) it = 0;
       }
@@ -2245,8 +2256,12 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
         mbar_arrive_expect_tx(bar, 4 * D_BOX_BYTES);
         const CUtensorMap* const map = s == 0 ? &p.map_d0 : &p.map_d;
         const int z = s == 0 ? 0 : p.ts_hi - s;
+        if (p.one_copy) {
+          tma_load_4d(dst, map, 0, 0, it * 4, z, bar);
+        } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tma_load_3d(dst + q * D_BOX_BYTES, map, it * 128 + 32 * q, 0, z, bar);
+          for (int q = 0; q < 4; ++q) tma_load_3d(dst + q * D_BOX_BYTES, map, it * 128 + 32 * q, 0, z, bar);
+        }
         if (++st == S) { st = 0; ++round; }
         if (++it == it_all) { it = 0; ++s; }
       }
@@ -2287,7 +2302,7 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
     for (int j = 0; j < EPI; ++j) {
       const int e = tid + j * NT, i = tile_row0 + e / BP, b = e % BP;
       pre_dn[j] = pre_go[j] = pre_gf[j] = pre_v[j] = 0.f;
-      if (i < N && b < p.B) {
+      if (e < TILE && i < N && b < p.B) {
         const size_t k = (size_t)b * N + i;
         pre_dn[j] = __ldcg(dn + k);
         pre_go[j] = p.g_out ? p.g_out[k] : 0.f;
@@ -2298,9 +2313,9 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
         pre_v[j] = Vd[k];
       }
     }
-    float acc[2][NTN][4];
+    float acc[MT][NTN][4];
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NTN; ++nt)
 #pragma unroll
@@ -2313,7 +2328,7 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
           break;
         }
         const float* const stage = reinterpret_cast<const float*>(ring + (size_t)st * STAGE_BYTES);
-        warp_chunk_mma<NTN, KS>(acc, stage + w_off, 32, stage + d_off, 32, [](int) {});
+        warp_chunk_mma<NTN, KS, MT>(acc, stage + w_off, 32, stage + d_off, 32, [](int) {});
         __syncwarp();
         if (lane == 0) mbar_arrive(s_empty + st);
         if (++st == S) { st = 0; ph_full ^= 1u; }
@@ -2323,7 +2338,7 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
     {
       float* mine = s_parts + (size_t)warp * TILEP;
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < NTN; ++nt) {
           const int r = mt * 16 + g, cc = nt * 8 + 2 * t;
@@ -2337,9 +2352,11 @@ __global__ void __launch_bounds__(32 * (NWARP + 2), NWARP == 8 ? 2 : 1) bwd_stre
     for (int j = 0; j < EPI; ++j) {
       const int e = tid + j * NT, i = tile_row0 + e / BP, b = e % BP;
       float sum = 0.f;
+      if (e < TILE) {
 #pragma unroll
-      for (int w = 0; w < NWARP; ++w) sum += s_parts[(size_t)w * TILEP + (e / BP) * TS + e % BP];
-      if (i < N && b < p.B && !dead) {
+        for (int w = 0; w < NWARP; ++w) sum += s_parts[(size_t)w * TILEP + (e / BP) * TS + e % BP];
+      }
+      if (e < TILE && i < N && b < p.B && !dead) {
         const size_t k = (size_t)b * N + i;
         float gs = sum + pre_go[j];
         if (gff) gs += pre_gf[j];

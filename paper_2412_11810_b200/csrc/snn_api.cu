@@ -36,7 +36,7 @@ struct snn_net {
   int device = -1;                         // device the two figures below were asked of
   int coop_sms = -1;                       // SMs usable by a cooperative launch (-1: not asked yet)
   int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
-  int bwd_stream_capacity[3] = {-1, -1, -1};   // the same for the three instances of bwd_stream_kernel
+  int bwd_stream_capacity[6] = {-1, -1, -1, -1, -1, -1};   // the same for the six instances of bwd_stream_kernel
 };
 
 namespace {
@@ -932,25 +932,41 @@ struct Exec {
 
   // Steps ts_hi-1 .. ts_lo of one layer in one cooperative launch (bwd_stream_kernel), if the device holds all
   // its CTAs at once; otherwise `done` stays false and the caller launches step by step.
-  CUtensorMap wrec_map[MAXL];      // W_rec of a layer as boxes of 32 rows x 32 values: 0 not tried yet, 1 ready, -1 not encodable
+  CUtensorMap wrec_map[MAXL];      // W_rec of a layer as boxes of 16 MT rows x 32 values: 0 not tried yet, 1 ready, -1 not encodable
   int wrec_map_ready[MAXL] = {0};
-  template <int NTN, int NWARP> snn_status try_backward_stream(BwdStreamParams& sp, int l, int tiles, bool& done) {
+  template <int NTN, int NWARP, int MT> snn_status try_backward_stream(BwdStreamParams& sp, int l, int tiles, bool& done) {
     done = false;
-    void (*k)(BwdStreamParams) = bwd_stream_kernel<NTN, NWARP>;
-    const size_t smem = bwd_stream_smem_bytes<NTN, NWARP>();
+    void (*k)(BwdStreamParams) = bwd_stream_kernel<NTN, NWARP, MT>;
+    const size_t smem = bwd_stream_smem_bytes<NTN, NWARP, MT>();
     // tensor maps: the matrix once per step of the executor, the deltas of this run (strides must be multiples of 16 bytes)
     if (sp.N % 4 != 0 || sp.slot_stride % 4 != 0) return SNN_OK;
-    if (wrec_map_ready[l - 1] == 0)
-      wrec_map_ready[l - 1] = make_tensor_map_2d(&wrec_map[l - 1], a->W_rec[l - 1], (uint64_t)sp.N, (uint64_t)sp.N, (uint64_t)sp.N,
-                                                 BWD_TM, 32, true) ? 1 : -1;
+    sp.one_copy = sp.N % 32 == 0;
+    if (wrec_map_ready[l - 1] == 0) {
+      if (sp.one_copy) {
+        const uint64_t dims[3] = {32, (uint64_t)sp.N, (uint64_t)sp.N / 32}, strides[2] = {(uint64_t)sp.N, 32};
+        const uint32_t box[3] = {32, 16 * MT, 4};
+        wrec_map_ready[l - 1] = make_tensor_map_nd(&wrec_map[l - 1], a->W_rec[l - 1], 3, dims, strides, box) ? 1 : -1;
+      } else {
+        wrec_map_ready[l - 1] = make_tensor_map_2d(&wrec_map[l - 1], a->W_rec[l - 1], (uint64_t)sp.N, (uint64_t)sp.N, (uint64_t)sp.N,
+                                                   16 * MT, 32, true) ? 1 : -1;
+      }
+    }
     if (wrec_map_ready[l - 1] < 0) return SNN_OK;
     sp.map_w = wrec_map[l - 1];
-    if (!make_tensor_map_3d(&sp.map_d, sp.slots + (size_t)sp.buf_slot * sp.slot_stride + sp.state_off, (uint64_t)sp.N, (uint64_t)sp.B,
-                            (uint64_t)sp.ts_hi, (uint64_t)sp.N, (uint64_t)sp.slot_stride, 32, 8 * NTN, 1) ||
-        !make_tensor_map_3d(&sp.map_d0, sp.d_first, (uint64_t)sp.N, (uint64_t)sp.B, 1, (uint64_t)sp.N, (uint64_t)sp.slot_stride, 32,
-                            8 * NTN, 1))
+    const float* const d_slots = sp.slots + (size_t)sp.buf_slot * sp.slot_stride + sp.state_off;
+    if (sp.one_copy) {
+      const uint64_t dims[4] = {32, (uint64_t)sp.B, (uint64_t)sp.N / 32, (uint64_t)sp.ts_hi}, dims0[4] = {32, (uint64_t)sp.B, (uint64_t)sp.N / 32, 1};
+      const uint64_t strides[3] = {(uint64_t)sp.N, 32, (uint64_t)sp.slot_stride};
+      const uint32_t box[4] = {32, 8 * NTN, 4, 1};
+      if (!make_tensor_map_nd(&sp.map_d, d_slots, 4, dims, strides, box) || !make_tensor_map_nd(&sp.map_d0, sp.d_first, 4, dims0, strides, box))
+        return SNN_OK;
+    } else if (!make_tensor_map_3d(&sp.map_d, d_slots, (uint64_t)sp.N, (uint64_t)sp.B, (uint64_t)sp.ts_hi, (uint64_t)sp.N,
+                                   (uint64_t)sp.slot_stride, 32, 8 * NTN, 1) ||
+               !make_tensor_map_3d(&sp.map_d0, sp.d_first, (uint64_t)sp.N, (uint64_t)sp.B, 1, (uint64_t)sp.N, (uint64_t)sp.slot_stride, 32,
+                                   8 * NTN, 1)) {
       return SNN_OK;
-    int& cap = net->bwd_stream_capacity[NTN == 1 ? 0 : NTN == 2 ? 1 : 2];
+    }
+    int& cap = net->bwd_stream_capacity[(NTN == 1 ? 0 : NTN == 2 ? 1 : 2) + 3 * (MT - 1)];
     if (cap < 0) {
       int dev = 0, sms = 0, per_sm = 0, coop = 0;
       if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -1071,9 +1087,11 @@ struct Exec {
           }
           const int tiles_l = (sz[l] + BWD_TM - 1) / BWD_TM;
           int CS_l = 1;
-          // layers with a row tile for every SM: no cluster, so that the run can be one launch that keeps the
-          // weight stream going (bwd_stream_kernel)
-          while (tiles_l < 148 && CS_l < 8 && tiles_l * CS_l * 2 <= wave && sz[l] / (4 * CS_l * 2) >= 32) CS_l *= 2;
+          // layers with a tile of 16 rows for every SM: no cluster, so that the run can be one launch that keeps the
+          // weight stream going (bwd_stream_kernel; tiles of 32 rows where those still cover the SMs)
+          const int tiles16_l = (sz[l] + 15) / 16;
+          const bool wide = tiles_l >= 148 || (tiles16_l >= 148 && B <= 16);   // (two CTAs of 16 rows per SM need B <= 16)
+          while (!wide && CS_l < 8 && tiles_l * CS_l * 2 <= wave && sz[l] / (4 * CS_l * 2) >= 32) CS_l *= 2;
           if (CS_l == 1 && B <= 32 && !(a->flags & SNN_FLAG_BACKWARD_PER_STEP)) {
             BwdStreamParams sp;
             std::memset(&sp, 0, sizeof sp);
@@ -1091,9 +1109,15 @@ struct Exec {
             sp.surrogate = net->surrogate; sp.cell = net->cell;
             bool done = false;
             snn_status st = SNN_OK;
-            if (B <= 8) st = try_backward_stream<1, 8>(sp, l, tiles_l, done);
-            else if (B <= 16) st = try_backward_stream<2, 8>(sp, l, tiles_l, done);
-            else st = try_backward_stream<4, 16>(sp, l, tiles_l, done);
+            if (tiles_l >= 148) {
+              if (B <= 8) st = try_backward_stream<1, 8, 2>(sp, l, tiles_l, done);
+              else if (B <= 16) st = try_backward_stream<2, 8, 2>(sp, l, tiles_l, done);
+              else st = try_backward_stream<4, 16, 2>(sp, l, tiles_l, done);
+            } else {
+              if (B <= 8) st = try_backward_stream<1, 8, 1>(sp, l, tiles16_l, done);
+              else if (B <= 16) st = try_backward_stream<2, 8, 1>(sp, l, tiles16_l, done);
+              else st = try_backward_stream<4, 16, 1>(sp, l, tiles16_l, done);
+            }
             if (st != SNN_OK) return st;
             if (done) continue;
           }
@@ -1274,9 +1298,12 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<1, 8>, dyn, (int)Exec::bwd_smem_bytes(8, bwd_ld(8))));
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<2, 8>, dyn, (int)Exec::bwd_smem_bytes(16, bwd_ld(8))));
   CUDA_TRY(cudaFuncSetAttribute(bwd_step_kernel<4, 16>, dyn, (int)Exec::bwd_smem_bytes(32, bwd_ld(16))));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8>, dyn, (int)bwd_stream_smem_bytes<1, 8>()));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8>, dyn, (int)bwd_stream_smem_bytes<2, 8>()));
-  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16>, dyn, (int)bwd_stream_smem_bytes<4, 16>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8, 2>, dyn, (int)bwd_stream_smem_bytes<1, 8, 2>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8, 2>, dyn, (int)bwd_stream_smem_bytes<2, 8, 2>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16, 2>, dyn, (int)bwd_stream_smem_bytes<4, 16, 2>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<1, 8, 1>, dyn, (int)bwd_stream_smem_bytes<1, 8, 1>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<2, 8, 1>, dyn, (int)bwd_stream_smem_bytes<2, 8, 1>()));
+  CUDA_TRY(cudaFuncSetAttribute(bwd_stream_kernel<4, 16, 1>, dyn, (int)bwd_stream_smem_bytes<4, 16, 1>()));
   CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel<false>, dyn, (int)dws_smem_bytes<false>()));
   CUDA_TRY(cudaFuncSetAttribute(dw_slab_kernel<true>, dyn, (int)dws_smem_bytes<true>()));
   CUDA_TRY(cudaFuncSetAttribute(dw_kernel<1, false>, dyn, (int)dw_smem_bytes<1, false>(DW_WINDOW)));
@@ -1358,7 +1385,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
       net->device = dev;
       net->coop_sms = -1;
       net->fwd_segment_capacity = -1;
-      net->bwd_stream_capacity[0] = net->bwd_stream_capacity[1] = net->bwd_stream_capacity[2] = -1;
+      for (int& c : net->bwd_stream_capacity) c = -1;
     }
   }
   cudaStream_t ms = ex.main;

@@ -68,6 +68,19 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
 }
+// The same with an L2 eviction priority.
+__device__ __forceinline__ void tma_load_3d_hint(void* smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+// Tiled copy of a box of a 4-D tensor map.
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, int x, int y, int z, int w, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
+}
 // Orders this thread's accesses through the generic proxy (ordinary loads and stores, global memory included) with
 // its accesses through the asynchronous proxy (bulk copies): a writer runs it after its stores and before it
 // signals, a reader after it has seen the signal and before it issues the copy that reads the data.
@@ -97,6 +110,22 @@ inline tensor_map_encode_fn tensor_map_encoder() {
     encode = reinterpret_cast<tensor_map_encode_fn>(fn);
   }
   return encode;
+}
+
+// A tensor map of `rank` (<= 5) dimensions over fp32 data, innermost dimension first: extents `dims`, distances of the
+// outer dimensions `strides_floats` (rank - 1 of them, multiples of 4 floats; they need not grow with the dimension: a
+// matrix [rows][cols] can be seen as [cols / 32][rows][32]), box `box`, 128-byte swizzle (box[0] * 4 must be 128).
+inline bool make_tensor_map_nd(CUtensorMap* out, const float* base, int rank, const uint64_t* dims, const uint64_t* strides_floats,
+                               const uint32_t* box) {
+  tensor_map_encode_fn encode = tensor_map_encoder();
+  if (!encode || rank < 2 || rank > 5) return false;
+  cuuint64_t d[5], st[4];
+  cuuint32_t bx[5], el[5];
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; el[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) st[i] = strides_floats[i] * sizeof(float);
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float*>(base), d, st, bx, el,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // A 3-D tensor map over fp32 data [d2][d1][d0] (d0 contiguous; rows stride1_floats apart, planes stride2_floats

@@ -565,15 +565,16 @@ def test_layer_by_layer_backward_order(orc32):
     s.close()
 
 
-@pytest.mark.parametrize("B", [3, 8, 11, 19])
-def test_layer_by_layer_backward_as_one_launch_per_run(orc32, B):
+@pytest.mark.parametrize("B,N1", [(3, 4772), (8, 4772), (11, 4772), (19, 4772), (5, 2404), (14, 2404), (8, 4768), (13, 2400)])
+def test_layer_by_layer_backward_as_one_launch_per_run(orc32, B, N1):
     """Wide layers under the layer-by-layer order run the steps of a run of 32 as ONE cooperative launch that
     keeps the recurrent matrix streaming across step boundaries.  It must give the bits of the same order with
     one launch per step, for each batch tiling (8, 16, 32 samples), a width that is no multiple of the row tile
     or of the 128-wide chunk, runs shorter and longer than the copy ring, and agree with the oracle.  (The wide
-    layer takes that launch for up to 8 samples, where two of its thread blocks fit an SM; the narrow one always.)"""
+    layer takes that launch where its thread blocks all fit the device at once; a layer half as wide takes it with
+    thread blocks of 16 rows, for up to 16 samples.)"""
     b = sb()
-    w = wl.small(sizes=(48, 4772, 132, 7), T=37, B=B, p_in=0.1, g_ff=(2.5, 1.5), g_rec=(1.0, 1.0), seed=43)
+    w = wl.small(sizes=(48, N1, 132, 7), T=37, B=B, p_in=0.1, g_ff=(2.5, 1.5), g_rec=(1.0, 1.0), seed=43)
     d = wl.make(w)
     ref = run_oracle(orc32, w, d)
     assert all(0.005 < float(x[1:].mean()) < 0.5 for x in ref["S"])
