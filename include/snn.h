@@ -142,7 +142,8 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
 /* The backward pass has two launch orders.  Wavefront: one launch per step covers all layers and also
  * multiplies by W_ff of the layer above.  Layer by layer: runs of 32 steps, the feed-forward term of a
  * whole run computed as one product so that W_ff is streamed once per run.  By default the second is
- * used when the weights exceed 96 MB (they then do not stay in L2); these flags force one or the other.
+ * used unless the network is small enough for the backward pass of a segment to run as one launch with the
+ * weights in shared memory (see SNN_FLAG_BACKWARD_PER_STEP); these flags force one or the other.
  * Gradients are bit-identical across strategies for a given order, not between the two orders. */
 #define SNN_FLAG_BACKWARD_LAYER_BY_LAYER 8u
 #define SNN_FLAG_BACKWARD_WAVEFRONT 16u

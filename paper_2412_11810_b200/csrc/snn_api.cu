@@ -90,6 +90,39 @@ struct Layout {
   bool tier2_on_device;
 };
 
+// Cluster size of the wavefront backward kernels along the contraction index: enough CTAs to fill the GPU (one wave:
+// two 256-thread CTAs or one 512-thread CTA per SM on 148 SMs), at least one full warp pass (128 values) per rank; a
+// function of the network sizes and the batch only.
+int backward_cluster_size(const std::vector<int>& sz, int L, int B) {
+  int maxN = 0;
+  for (int l = 1; l <= L; ++l) maxN = std::max(maxN, sz[l]);
+  int minN = maxN;
+  for (int l = 1; l <= L; ++l) minN = std::min(minN, sz[l]);
+  const int tiles = (maxN + BWD_TM - 1) / BWD_TM;
+  const int wave = B <= 16 ? 296 : 148;
+  int CS = 1;
+  while (CS < 8 && tiles * L * CS * 2 <= wave && minN / (4 * CS * 2) >= 32) CS *= 2;
+  return CS;
+}
+// Dynamic shared memory bwd_segment_kernel needs: the largest slice of W_ff(l+1) and W_rec a cluster rank keeps
+// resident (32 rows x its share of the contraction index) and the staging region.
+size_t backward_segment_smem(const std::vector<int>& sz, int L, int B, int CS) {
+  const int nwarp = B <= 16 ? 8 : 16;
+  size_t res_floats = 0;
+  for (int l = 1; l <= L; ++l) {
+    const int q_rec = sz[l] / 4, q_ff = (l < L ? sz[l + 1] : 0) / 4;
+    for (int r = 0; r < CS; ++r) {
+      const int k_rec = (int)((long long)q_rec * (r + 1) / CS) * 4 - (int)((long long)q_rec * r / CS) * 4;
+      const int k_ff = (int)((long long)q_ff * (r + 1) / CS) * 4 - (int)((long long)q_ff * r / CS) * 4;
+      res_floats = std::max(res_floats, (size_t)BWD_TM * bwd_resident_ld(k_ff, k_rec, nwarp));
+    }
+  }
+  const size_t region = B <= 8 ? bwd_segment_region_floats<1, 8>() : B <= 16 ? bwd_segment_region_floats<2, 8>()
+                                                                           : bwd_segment_region_floats<4, 16>();
+  return 4 * (res_floats + region);
+}
+constexpr size_t BWD_SEGMENT_SMEM_MAX = (size_t)218 << 10;
+
 bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float max_activity, uint32_t flags,
                     Layout& lo, std::string& why) {
   const int L = net->L;
@@ -149,13 +182,15 @@ bool compute_layout(const snn_net* net, int T, int B, const snn_ckpt* ck, float 
   lo.event_bytes = cur - ev0;
   for (int l = 0; l <= L; ++l) lo.act[l] = (graded && l > 0) ? take(4 * (size_t)2 * B * sz[l]) : 0;
   {
-    // Networks whose weights do not stay in L2: streaming W_ff once per run of steps instead of once per
-    // step pays for giving up the layer wavefront in the backward pass.  A function of the sizes only.
+    // Networks whose weight slices do not fit the shared memory of the segment kernel: multiplying by W_ff once per
+    // run of steps (one product on the tensor cores, W_ff streamed once) instead of once per step pays for giving
+    // up the layer wavefront in the backward pass.  A function of the sizes and the batch only.
     size_t wbytes = 0;
     int maxN = 0;
     for (int l = 1; l <= L; ++l) { wbytes += 4 * ((size_t)sz[l - 1] * sz[l] + (size_t)sz[l] * sz[l]); maxN = std::max(maxN, sz[l]); }
     lo.weights_resident = wbytes <= ((size_t)96 << 20);
-    lo.layer_major = L > 1 && !lo.weights_resident;
+    lo.layer_major = L > 1 && (!lo.weights_resident ||
+                               backward_segment_smem(sz, L, B, backward_cluster_size(sz, L, B)) > BWD_SEGMENT_SMEM_MAX);
     lo.gff_stride = (size_t)BWD_RUN * B * maxN;
     lo.gff = L > 1 ? take(4 * lo.gff_stride * TCG_MAX_KSPLIT) : 0;
   }
@@ -897,7 +932,7 @@ struct Exec {
       }
     }
     const size_t smem = 4 * (res_floats + bwd_segment_region_floats<NTN, NWARP>());
-    if (smem > ((size_t)218 << 10)) return SNN_OK;
+    if (smem > BWD_SEGMENT_SMEM_MAX) return SNN_OK;
     void (*k)(BwdSegParams) = bwd_segment_kernel<NTN, NWARP>;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas); cfg.blockDim = dim3(32 * NWARP); cfg.dynamicSmemBytes = smem; cfg.stream = main;
@@ -1012,8 +1047,7 @@ struct Exec {
     for (int l = 1; l <= L; ++l) minN = std::min(minN, sz[l]);
     // (one wave: two 256-thread CTAs or one 512-thread CTA per SM on 148 SMs)
     const int wave = B <= 16 ? 296 : 148;
-    int CS = 1;
-    while (CS < 8 && tiles * L * CS * 2 <= wave && minN / (4 * CS * 2) >= 32) CS *= 2;
+    const int CS = backward_cluster_size(sz, L, B);
     int span = begin_span(SNN_PHASE_BWD);
     // event-driven steps (compact-support surrogate): a layer wavefront, one launch per step
     const bool event_driven = (a->flags & SNN_FLAG_BACKWARD_EVENT_DRIVEN) != 0;
