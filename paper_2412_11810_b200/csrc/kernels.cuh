@@ -297,8 +297,17 @@ constexpr int GATHER_ROWS = 8;     // weight rows per copy group
 constexpr int GATHER_STAGES = 3;   // copy groups in flight per thread (24 rows, 48 KB per CTA: four CTAs per SM)
 constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
+// fwd_step_kernel: four consumer warps (a thread owns four neurons) and one producer warp.  The listed weight rows
+// reach shared memory as plain bulk copies (`cp.async.bulk`, one row segment of this CTA's columns per copy, up to
+// 2 KB), eight rows per group, issued by eight lanes of the producer warp at once; groups cycle through a ring of
+// GATHER_STAGES stages guarded by full / empty mbarriers.  The consumers issue no copies: per row and thread one
+// 16-byte shared-memory read and four additions, in list order.
+constexpr int FWDS_THREADS = FWD_THREADS + 32;
+constexpr uint32_t FWDS_ROW_BYTES = FWD_COLS * sizeof(float);                  // a row segment in the ring
+constexpr uint32_t FWDS_GROUP_BYTES = GATHER_ROWS * FWDS_ROW_BYTES;
+
 template <bool GEN, bool GRADED>
-__global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_constant__ FwdParams p) {
+__global__ void __launch_bounds__(FWDS_THREADS) fwd_step_kernel(const __grid_constant__ FwdParams p) {
   pdl_launch_dependents();
   const FwdLayer& L = p.lay[blockIdx.z];
   if (L.mode == 0) return;
@@ -308,13 +317,20 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   const bool tile0 = blockIdx.x == 0;
   __shared__ const float* s_row[LIST_CHUNK];   // addresses of the listed weight rows at this CTA's first column
   __shared__ uint32_t s_pref[GEN ? 2 * MAX_WORDS + 1 : 1];
-  __shared__ uint32_t s_warp[FWD_THREADS / 32];
+  __shared__ uint32_t s_warp[FWDS_THREADS / 32];
   __shared__ float s_val[GRADED ? LIST_CHUNK : 1];
+  __shared__ uint64_t s_full[GATHER_STAGES], s_empty[GATHER_STAGES];
   extern __shared__ float4 s_stage[];   // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
+  const bool producer = threadIdx.x >= FWD_THREADS;        // the fifth warp
   const int col = col0 + threadIdx.x * 4;
-  const bool active = col < L.N;
+  const bool active = !producer && col < L.N;
   const bool step = L.mode == 1;
   if (!step && !(GEN && tile0)) return;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < GATHER_STAGES; ++i) { mbar_init(s_full + i, 1); mbar_init(s_empty + i, FWD_THREADS / 32); }
+    mbar_fence_init();
+  }
+  __syncthreads();
 
   pdl_wait();
   // issue the loads the epilogue needs before anything else
@@ -333,7 +349,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
   if (GEN) {
     wp = WordPair{step ? L.ff_mask + (size_t)b * L.W_pre : nullptr, step ? L.W_pre : 0,
                   L.rec_mask + (size_t)b * L.W, L.W, last_word_mask(L.N_pre)};
-    total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
+    total = prefix_popcounts<FWDS_THREADS>(wp, s_pref, s_warp);
     n_ff = s_pref[wp.n_a];
     if (tile0) {  // this CTA appends the lists to the event pools
       const bool wr_ff = step && L.write_ff_list;
@@ -341,13 +357,13 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
       if (wr_ff) s_ff = L.ff_off[b];
       const uint32_t room_ff = wr_ff ? L.ff_cap - s_ff : 0, room_rec = L.rec_cap - s_rec;
       if (GRADED)
-        write_lists_from_words<FWD_THREADS, true>(
+        write_lists_from_words<FWDS_THREADS, true>(
             wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff, rec_pool + s_rec, room_rec,
             wr_ff ? L.ff_val_src + (size_t)b * L.N_pre : nullptr, L.ff_vals + (size_t)b * L.ff_cap + s_ff,
             L.ff_pref + (size_t)b * L.W_pre, L.rec_val_src + (size_t)b * L.N,
             L.rec_vals + (size_t)b * L.rec_cap + s_rec, L.rec_pref + (size_t)b * L.W);
       else
-        write_lists_from_words<FWD_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff,
+        write_lists_from_words<FWDS_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + s_ff : nullptr, room_ff,
                                                    rec_pool + s_rec, room_rec);
       if (threadIdx.x == 0) {
         const uint32_t n_rec = total - n_ff;
@@ -364,17 +380,22 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
 
   // ---- gather-accumulate in list order
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  // ring position of the next group (both roles count the groups of all chunks alike); bytes of a row segment
+  int gc = 0, slot = 0;
+  uint32_t round = 0;          // gc / GATHER_STAGES
+  bool dead = false;           // a wait of this warp ran out: no more waiting, copying or adding
+  const uint32_t row_bytes = (uint32_t)(L.N - col0 < FWD_COLS ? L.N - col0 : FWD_COLS) * sizeof(float);
   const float* const Wff_tile = L.W_ff + col0;
   const float* const Wrec_tile = L.W_rec + col0;
   for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
     const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
     if (GEN) {
-      fill_rows_from_words<FWD_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
+      fill_rows_from_words<FWDS_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
       if (GRADED)
-        fill_values_from_words<FWD_THREADS>(wp, s_pref, c0, L.ff_val_src + (size_t)b * L.N_pre,
+        fill_values_from_words<FWDS_THREADS>(wp, s_pref, c0, L.ff_val_src + (size_t)b * L.N_pre,
                                             L.rec_val_src + (size_t)b * L.N, s_val);
     } else {
-      for (int i = threadIdx.x; i < n; i += FWD_THREADS) {
+      for (int i = threadIdx.x; i < n; i += FWDS_THREADS) {
         const uint32_t q = c0 + i;
         s_row[i] = q < n_ff
             ? Wff_tile + (size_t)checked_index(ff_pool[checked_index(s_ff + q, L.ff_cap, p.status)], L.N_pre, p.status) * L.N
@@ -385,27 +406,27 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
       }
     }
     __syncthreads();
-    if (active) {
-      // weight rows stream through a per-thread ring of GATHER_STAGES groups of GATHER_ROWS rows:
-      // the copies of the next groups are in flight while the oldest group is added, in list order
-      float4* const ring = s_stage + threadIdx.x;
-      const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
-      const int lane_col = threadIdx.x * 4;
-      auto issue = [&](int g) {
-        if (g < n_groups) {
-          float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
-          const float* const* rows = s_row + g * GATHER_ROWS;
-          if ((g + 1) * GATHER_ROWS <= n) {
-#pragma unroll
-            for (int u = 0; u < GATHER_ROWS; ++u) cp_async16(dst + u * FWD_THREADS, rows[u] + lane_col);
-          } else {
-#pragma unroll
-            for (int u = 0; u < GATHER_ROWS; ++u)
-              if (g * GATHER_ROWS + u < n) cp_async16(dst + u * FWD_THREADS, rows[u] + lane_col);
-          }
+    const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
+    if (producer) {
+      // ---- producer warp: eight lanes copy the eight rows of a group
+      const int lane = threadIdx.x & 31;
+      for (int g = 0; g < n_groups && !dead; ++g) {
+        if (gc >= GATHER_STAGES && !mbar_wait(s_empty + slot, (round - 1u) & 1u)) {   // group gc - GATHER_STAGES is added
+          if (lane == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+          dead = true;
+          break;
         }
-        cp_async_commit();
-      };
+        const int rows_here = n - g * GATHER_ROWS < GATHER_ROWS ? n - g * GATHER_ROWS : GATHER_ROWS;
+        if (lane == 0) mbar_arrive_expect_tx(s_full + slot, (uint32_t)rows_here * row_bytes);
+        __syncwarp();
+        if (lane < rows_here)
+          bulk_load(reinterpret_cast<unsigned char*>(s_stage) + (size_t)slot * FWDS_GROUP_BYTES + (size_t)lane * FWDS_ROW_BYTES,
+                    s_row[g * GATHER_ROWS + lane], row_bytes, s_full + slot);
+        ++gc;
+        if (++slot == GATHER_STAGES) { slot = 0; ++round; }
+      }
+    } else {
+      // ---- consumers: the rows of a group in list order
       auto add_row = [&](const float4 w, int i) {
         if (GRADED) {   // one fused multiply-add per event and neuron
           const float sv = s_val[i];
@@ -416,23 +437,36 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_step_kernel(const __grid_cons
           acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
         }
       };
-      for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
-      for (int g = 0; g < n_groups; ++g) {
-        issue(g + GATHER_STAGES - 1);
-        cp_async_wait<GATHER_STAGES - 1>();
-        const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
-        if ((g + 1) * GATHER_ROWS <= n) {
-#pragma unroll
-          for (int u = 0; u < GATHER_ROWS; ++u) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
-        } else {
-#pragma unroll
-          for (int u = 0; u < GATHER_ROWS; ++u)
-            if (g * GATHER_ROWS + u < n) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
+      for (int g = 0; g < n_groups && !dead; ++g) {
+        if (!mbar_wait(s_full + slot, round & 1u)) {
+          if ((threadIdx.x & 31) == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+          dead = true;
+          break;
         }
+        if (active) {
+          const float4* src = s_stage + (size_t)slot * GATHER_ROWS * FWD_THREADS + threadIdx.x;
+          if ((g + 1) * GATHER_ROWS <= n) {
+#pragma unroll
+            for (int u = 0; u < GATHER_ROWS; ++u) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
+          } else {
+#pragma unroll
+            for (int u = 0; u < GATHER_ROWS; ++u)
+              if (g * GATHER_ROWS + u < n) add_row(src[u * FWD_THREADS], g * GATHER_ROWS + u);
+          }
+        }
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(s_empty + slot);
+        ++gc;
+        if (++slot == GATHER_STAGES) { slot = 0; ++round; }
       }
-      cp_async_wait<0>();
     }
     __syncthreads();
+  }
+  if (producer) {
+    if (dead)   // the copies of the last groups issued may still be on their way: wait for them, briefly
+      for (int cc = gc > GATHER_STAGES ? gc - GATHER_STAGES : 0; cc < gc; ++cc)
+        mbar_wait(s_full + cc % GATHER_STAGES, (uint32_t)(cc / GATHER_STAGES) & 1u, 1u << 14);
+    return;
   }
 
   // ---- leak, reset by subtraction of the previous step's own spike, threshold

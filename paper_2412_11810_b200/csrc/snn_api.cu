@@ -531,7 +531,7 @@ struct Exec {
   snn_status launch_fwd(const FwdParams& p, bool gen) {
     void (*k)(FwdParams) = graded() ? (gen ? fwd_step_kernel<true, true> : fwd_step_kernel<false, true>)
                                     : (gen ? fwd_step_kernel<true, false> : fwd_step_kernel<false, false>);
-    CUDA_TRY(launch_pdl(k, fwd_grid(), dim3(FWD_THREADS), FWD_DYN_SMEM, p));
+    CUDA_TRY(launch_pdl(k, fwd_grid(), dim3(FWDS_THREADS), FWD_DYN_SMEM, p));
     ++launches;
     CUDA_TRY(cudaGetLastError());
     return SNN_OK;
