@@ -297,6 +297,36 @@ constexpr int GATHER_ROWS = 8;     // weight rows per copy group
 constexpr int GATHER_STAGES = 3;   // copy groups in flight per thread (24 rows, 48 KB per CTA: four CTAs per SM)
 constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
+// The producer warp's share of a gather: the n listed rows (addresses in s_row) go into the ring as bulk copies, eight
+// rows per group, up to four groups per trip round the loop (eight lanes each; one when the ring has few stages).
+// `gc` counts the groups of the whole launch (the consumers count alike): group gc uses stage gc % G and the
+// (gc / G)-th phase of its barriers.  A wait that runs out raises the status bit and sets `dead`.
+__device__ __forceinline__ void gather_producer(const float* const* s_row, int n, unsigned char* ring, int G,
+                                                uint64_t* s_full, uint64_t* s_empty, uint32_t row_bytes, int& gc, bool& dead,
+                                                uint32_t* status, uint32_t group_bytes, uint32_t slot_row_bytes) {
+  const int lane = threadIdx.x & 31, sub = lane >> 3, r = lane & 7;
+  const int n_groups = (n + 7) / 8, NB = G >= 8 ? 4 : G >= 6 ? 2 : 1;   // a trip waits for all its stages: a fraction of the ring
+  for (int g0 = 0; g0 < n_groups && !dead; g0 += NB) {
+    const int g = g0 + sub;
+    const bool valid = sub < NB && g < n_groups;
+    const int my_gc = gc + sub, my_slot = my_gc % G;
+    const uint32_t my_round = (uint32_t)(my_gc / G);
+    bool ok = true;
+    if (valid && my_gc >= G) ok = mbar_wait(s_empty + my_slot, (my_round - 1u) & 1u);   // group my_gc - G is added
+    if (__any_sync(0xffffffffu, !ok)) {
+      if (lane == 0) atomicOr(status, STATUS_SYNC_TIMEOUT);
+      dead = true;
+      break;
+    }
+    const int rows_here = valid ? (n - g * 8 < 8 ? n - g * 8 : 8) : 0;
+    if (valid && r == 0) mbar_arrive_expect_tx(s_full + my_slot, (uint32_t)rows_here * row_bytes);
+    __syncwarp();
+    if (r < rows_here)
+      bulk_load(ring + (size_t)my_slot * group_bytes + (size_t)r * slot_row_bytes, s_row[g * 8 + r], row_bytes, s_full + my_slot);
+    gc += n_groups - g0 < NB ? n_groups - g0 : NB;
+  }
+}
+
 // fwd_step_kernel: four consumer warps (a thread owns four neurons) and one producer warp.  The listed weight rows
 // reach shared memory as plain bulk copies (`cp.async.bulk`, one row segment of this CTA's columns per copy, up to
 // 2 KB), eight rows per group, issued by eight lanes of the producer warp at once; groups cycle through a ring of
@@ -408,7 +438,8 @@ __global__ void __launch_bounds__(FWDS_THREADS) fwd_step_kernel(const __grid_con
     __syncthreads();
     const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
     if (producer) {
-      // ---- producer warp: eight lanes copy the eight rows of a group
+      // ---- producer warp: eight lanes copy the eight rows of a group (the loop holds nothing else: with three stages
+      // its trips bound the gather, and the general routine above, four groups per trip, is slower here)
       const int lane = threadIdx.x & 31;
       for (int g = 0; g < n_groups && !dead; ++g) {
         if (gc >= GATHER_STAGES && !mbar_wait(s_empty + slot, (round - 1u) & 1u)) {   // group gc - GATHER_STAGES is added
@@ -1185,6 +1216,7 @@ struct FwdSegParams {
   uint32_t* progress;         // [L][B] finished (tile, step) pairs, zero at launch
   int B, t0, t1;
   int in_slot, buf_slot, buf_len, keep_every, keep_slot;
+  int ring_groups;            // groups of eight rows in the copy ring (dynamic shared memory: 16 KB each)
   float alpha, theta;
 };
 
@@ -1223,7 +1255,13 @@ __global__ void wait_selftest_kernel(uint32_t* status, const uint32_t* counter, 
   status[1] = 1u;   // not reached unless somebody published
 }
 
-__global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_constant__ FwdSegParams p) {
+// The gather is that of fwd_step_kernel: a fifth warp copies the listed rows as bulk copies through a ring of groups
+// of eight rows, the four consumer warps add them in list order.  The ring is as deep as the launch allows
+// (FwdSegParams::ring_groups; one CTA per SM when the grid fits that way: a deep ring is what lets one SM gather from L2
+// at more than the 45 GB/s that four warps of 16-byte copies reach).
+constexpr int SEG_RING_MAX = 10;   // groups of eight rows in the ring at most (160 KB)
+
+__global__ void __launch_bounds__(FWDS_THREADS) fwd_segment_kernel(const __grid_constant__ FwdSegParams p) {
   const int l = blockIdx.z;
   const FwdSegLayer& L = p.lay[l];
   const int col0 = blockIdx.x * FWD_COLS;
@@ -1233,11 +1271,24 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
   __shared__ const float* s_row[LIST_CHUNK];
   __shared__ uint32_t s_words[SEG_WORDS];
   __shared__ uint32_t s_pref[SEG_WORDS + 1];
-  __shared__ uint32_t s_warp[FWD_THREADS / 32];
+  __shared__ uint32_t s_warp[FWDS_THREADS / 32];
   __shared__ int s_ok;
-  extern __shared__ float4 s_stage[];   // [GATHER_STAGES][GATHER_ROWS][FWD_THREADS]
+  __shared__ uint64_t s_full[SEG_RING_MAX], s_empty[SEG_RING_MAX];
+  extern __shared__ float4 s_stage[];   // [ring_groups][GATHER_ROWS][FWD_THREADS]
+  const bool producer = tid >= FWD_THREADS;        // the fifth warp
   const int col = col0 + tid * 4;
-  const bool active = col < L.N;
+  const bool active = !producer && col < L.N;
+  const int G = p.ring_groups;
+  if (tid == 0) {
+    for (int i = 0; i < G; ++i) { mbar_init(s_full + i, 1); mbar_init(s_empty + i, FWD_THREADS / 32); }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  // ring position of the next group (both roles count the groups of all steps alike); bytes of a row segment
+  int gc = 0, slot = 0;
+  uint32_t round = 0;          // gc / G
+  bool dead = false;           // a wait of this warp ran out: no more waiting, copying or adding
+  const uint32_t row_bytes = (uint32_t)(L.N - col0 < FWD_COLS ? L.N - col0 : FWD_COLS) * sizeof(float);
   const float* const Wff_tile = L.W_ff + col0;
   const float* const Wrec_tile = L.W_rec + col0;
   uint32_t* const ff_pool = L.ff_pool + (size_t)b * L.ff_cap;
@@ -1269,20 +1320,20 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
     {
       const uint32_t* ffw = L.ff_words + ((size_t)(t - L.ff_row0) * B + b) * L.W_pre;
       const uint32_t* recw = L.words + ((size_t)(t - 1) * B + b) * L.W;
-      for (int w = tid; w < L.W_pre + L.W; w += FWD_THREADS) {
+      for (int w = tid; w < L.W_pre + L.W; w += FWDS_THREADS) {
         const uint32_t x = __ldcg(w < L.W_pre ? ffw + w : recw + (w - L.W_pre));
         s_words[w] = w == L.W_pre - 1 ? x & last_word_mask(L.N_pre) : x;
       }
     }
     __syncthreads();
     const WordPair wp{s_words, L.W_pre, s_words + L.W_pre, L.W};
-    const uint32_t total = prefix_popcounts<FWD_THREADS>(wp, s_pref, s_warp);
+    const uint32_t total = prefix_popcounts<FWDS_THREADS>(wp, s_pref, s_warp);
     const uint32_t n_ff = s_pref[L.W_pre];
     const uint32_t pw = active ? s_words[L.W_pre + (col >> 5)] >> (col & 31) : 0u;
     if (tile0) {   // append the two lists to the event pools
       const bool wr_ff = L.write_ff_list != 0;
       const uint32_t room_ff = wr_ff ? L.ff_cap - ff_end : 0u, room_rec = L.rec_cap - rec_end;
-      write_lists_from_words<FWD_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + ff_end : nullptr, room_ff,
+      write_lists_from_words<FWDS_THREADS, false>(wp, s_pref, n_ff, wr_ff ? ff_pool + ff_end : nullptr, room_ff,
                                                  rec_pool + rec_end, room_rec);
       const uint32_t n_rec = total - n_ff;
       rec_end += n_rec < room_rec ? n_rec : room_rec;
@@ -1298,37 +1349,37 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (uint32_t c0 = 0; c0 < total; c0 += LIST_CHUNK) {
       const int n = (int)(total - c0 < (uint32_t)LIST_CHUNK ? total - c0 : (uint32_t)LIST_CHUNK);
-      fill_rows_from_words<FWD_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
+      fill_rows_from_words<FWDS_THREADS>(wp, s_pref, c0, Wff_tile, Wrec_tile, L.N, s_row);
       __syncthreads();
-      if (active) {
-        float4* const ring = s_stage + tid;
-        const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
-        const int lane_col = tid * 4;
-        auto issue = [&](int g) {
-          if (g < n_groups) {
-            float4* dst = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
-            const float* const* rows = s_row + g * GATHER_ROWS;
+      const int n_groups = (n + GATHER_ROWS - 1) / GATHER_ROWS;
+      if (producer) {
+        // ---- producer warp
+        gather_producer(s_row, n, reinterpret_cast<unsigned char*>(s_stage), G, s_full, s_empty, row_bytes, gc, dead, p.status,
+                        FWDS_GROUP_BYTES, FWDS_ROW_BYTES);
+      } else {
+        // ---- consumers: the rows of a group in list order
+        for (int g = 0; g < n_groups && !dead; ++g) {
+          if (!mbar_wait(s_full + slot, round & 1u)) {
+            if ((tid & 31) == 0) atomicOr(p.status, STATUS_SYNC_TIMEOUT);
+            dead = true;
+            break;
+          }
+          if (active) {
+            const float4* src = s_stage + (size_t)slot * GATHER_ROWS * FWD_THREADS + tid;
 #pragma unroll
             for (int u = 0; u < GATHER_ROWS; ++u) {
-              const bool real = g * GATHER_ROWS + u < n;
-              cp_async16_or_zero(dst + u * FWD_THREADS, real ? rows[u] + lane_col : Wff_tile, real);
+              if (g * GATHER_ROWS + u < n) {
+                const float4 w = src[u * FWD_THREADS];
+                acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
+                acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
+              }
             }
           }
-          cp_async_commit();
-        };
-        for (int g = 0; g < GATHER_STAGES - 1; ++g) issue(g);
-        for (int g = 0; g < n_groups; ++g) {
-          issue(g + GATHER_STAGES - 1);
-          cp_async_wait<GATHER_STAGES - 1>();
-          const float4* src = ring + (size_t)(g % GATHER_STAGES) * GATHER_ROWS * FWD_THREADS;
-#pragma unroll
-          for (int u = 0; u < GATHER_ROWS; ++u) {   // rows past the list's end were zero-filled: +0 changes nothing
-            const float4 w = src[u * FWD_THREADS];
-            acc.x = __fadd_rn(acc.x, w.x); acc.y = __fadd_rn(acc.y, w.y);
-            acc.z = __fadd_rn(acc.z, w.z); acc.w = __fadd_rn(acc.w, w.w);
-          }
+          __syncwarp();
+          if ((tid & 31) == 0) mbar_arrive(s_empty + slot);
+          ++gc;
+          if (++slot == G) { slot = 0; ++round; }
         }
-        cp_async_wait<0>();
       }
       __syncthreads();
     }
@@ -1353,7 +1404,7 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
         *c = cv;
       }
     }
-    {   // eight neighbouring lanes hold the 32 bits of one spike word
+    if (!producer) {   // eight neighbouring lanes hold the 32 bits of one spike word
       const int lane = tid & 31;
       uint32_t word = nib << (4 * (lane & 7));
       word |= __shfl_xor_sync(0xffffffffu, word, 1);
@@ -1367,6 +1418,8 @@ __global__ void __launch_bounds__(FWD_THREADS) fwd_segment_kernel(const __grid_c
       publish_progress(my_progress);
     }
   }
+  if (producer && dead)   // the copies of the last groups issued may still be on their way: wait for them, briefly
+    for (int cc = gc > G ? gc - G : 0; cc < gc; ++cc) mbar_wait(s_full + cc % G, (uint32_t)(cc / G) & 1u, 1u << 14);
 }
 
 // ------------------------------------------------------------------------------------------

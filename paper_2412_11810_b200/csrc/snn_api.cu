@@ -35,7 +35,7 @@ struct snn_net {
   snn_phase_times phases{};
   int device = -1;                         // device the two figures below were asked of
   int coop_sms = -1;                       // SMs usable by a cooperative launch (-1: not asked yet)
-  int fwd_segment_capacity = -1;           // CTAs of fwd_segment_kernel the device holds at once (-1: not asked yet)
+  int fwd_segment_capacity[2] = {-1, -1};   // CTAs of fwd_segment_kernel the device holds at once with a deep / shallow copy ring (-1: not asked yet)
   int bwd_stream_capacity[6] = {-1, -1, -1, -1, -1, -1};   // the same for the six instances of bwd_stream_kernel
 };
 
@@ -677,20 +677,27 @@ struct Exec {
     if (graded() || !lo.weights_resident || (a->flags & SNN_FLAG_FORWARD_PER_STEP)) return false;
     for (int l = 1; l <= L; ++l)
       if (lo.words[l - 1] + lo.words[l] > SEG_WORDS) return false;
-    if (net->fwd_segment_capacity < 0) {
-      int dev = 0, sms = 0, per_sm = 0, coop = 0;
+    // CTAs the device holds at once with a deep copy ring ([0]: SEG_RING_MAX groups) and with a shallow one ([1])
+    if (net->fwd_segment_capacity[0] < 0) {
+      int dev = 0, sms = 0, coop = 0;
       if (cudaGetDevice(&dev) != cudaSuccess ||
           cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-          cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fwd_segment_kernel, FWD_THREADS, FWD_DYN_SMEM) != cudaSuccess) {
+          cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
         cudaGetLastError();
-        net->fwd_segment_capacity = 0;
-      } else {
-        net->fwd_segment_capacity = coop ? sms * per_sm : 0;
+        coop = 0;
+      }
+      for (int i = 0; i < 2; ++i) {
+        int per_sm = 0;
+        if (!coop || cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fwd_segment_kernel, FWDS_THREADS,
+                                                                   (size_t)(i == 0 ? SEG_RING_MAX : GATHER_STAGES) * FWDS_GROUP_BYTES) != cudaSuccess) {
+          cudaGetLastError();
+          per_sm = 0;
+        }
+        net->fwd_segment_capacity[i] = sms * per_sm;
       }
     }
     const dim3 g = fwd_grid();
-    return (long long)g.x * g.y * g.z <= net->fwd_segment_capacity;
+    return (long long)g.x * g.y * g.z <= std::max(net->fwd_segment_capacity[0], net->fwd_segment_capacity[1]);
   }
 
   // FWD with the weights held in shared memory for the whole launch (fwd_resident_kernel): small LIF networks.
@@ -797,7 +804,10 @@ struct Exec {
     }
     CUDA_TRY(cudaMemsetAsync(ws + lo.progress, 0, 4 * (size_t)L * B, main));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = fwd_grid(); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = FWD_DYN_SMEM; cfg.stream = main;
+    cfg.gridDim = fwd_grid(); cfg.blockDim = dim3(FWDS_THREADS); cfg.stream = main;
+    // the deep ring when the device holds the grid that way (one CTA per SM), else the shallow one
+    p.ring_groups = (long long)cfg.gridDim.x * cfg.gridDim.y * cfg.gridDim.z <= net->fwd_segment_capacity[0] ? SEG_RING_MAX : GATHER_STAGES;
+    cfg.dynamicSmemBytes = (size_t)p.ring_groups * FWDS_GROUP_BYTES;
     cudaLaunchAttribute at1[1];
     at1[0].id = cudaLaunchAttributeCooperative;
     at1[0].val.cooperative = 1;
@@ -1321,7 +1331,7 @@ snn_status opt_in_shared_memory(snn_net* net, int dev) {
   CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, false>, dyn, (int)FWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<true, true>, dyn, (int)FWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(fwd_step_kernel<false, true>, dyn, (int)FWD_DYN_SMEM));
-  CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, dyn, (int)FWD_DYN_SMEM));
+  CUDA_TRY(cudaFuncSetAttribute(fwd_segment_kernel, dyn, (int)(SEG_RING_MAX * FWDS_GROUP_BYTES)));
   CUDA_TRY(cudaFuncSetAttribute(fwd_resident_kernel, dyn, (int)RESIDENT_SMEM_MAX));
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<false>, dyn, (int)REFWD_DYN_SMEM));
   CUDA_TRY(cudaFuncSetAttribute(refwd_gather_kernel<true>, dyn, (int)REFWD_DYN_SMEM));
@@ -1418,7 +1428,7 @@ extern "C" snn_status snn_train_step(snn_net* net, const snn_step_args* a, float
     if (net->device != dev) {   // figures cached per net belong to the device they were asked of
       net->device = dev;
       net->coop_sms = -1;
-      net->fwd_segment_capacity = -1;
+      net->fwd_segment_capacity[0] = net->fwd_segment_capacity[1] = -1;
       for (int& c : net->bwd_stream_capacity) c = -1;
     }
   }
