@@ -47,10 +47,10 @@ def read_peaks():
 # the kernel still has that text.  The backward pass of c2 now runs in bwd_segment_kernel, a cooperative launch
 # of thread-block clusters that the profiler cannot launch: no counters, hence no entry.
 NCU_TRAFFIC = {
-    # one launch = 16 steps of one layer: 3,343,270,000 B read + 5,011,712 B written; per layer and step (less than the
+    # one launch = 16 steps of one layer: 3,337,776,000 B read + 5,214,720 B written; per layer and step (less than the
     # algorithmic bytes: the first 64 MB of the matrix stay in L2 from one step to the next):
-    ("c4", "bwd"): ("bwd_stream_kernel", "276ff864da2e282cffd3aa30545b3c7dbfc504f2427a9d9eeebcb99de198cf2c",
-                    (3343270000 + 5011712) // 16),
+    ("c4", "bwd"): ("bwd_stream_kernel", "5a49fc56be35fd5f7a11f4fa48db838043c34b52375e31c8f755c92e20664b84",
+                    (3337776000 + 5214720) // 16),
     ("c3", "bwd"): ("bwd_step_kernel", "2f4bbd76ae837e3ce2614c31b106f74f4b5e27af23b3429895c113105211be02",
                     51018240 + 43264),
     ("c4", "fwd"): ("fwd_step_kernel", "f984311eddc0b278aeb605935b3e36af28944f04d5c03dee15033512817ce1fb",
