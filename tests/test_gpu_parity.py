@@ -117,6 +117,17 @@ def test_forward_one_launch_per_step_bit_exact(orc32):
     _check_forward(orc32, w, wl.make(w), extra_flags=g)
 
 
+def test_forward_segment_launch_with_the_shallow_ring(orc32):
+    """The cooperative forward launch of L2-resident networks copies weight rows through a ring that is as deep as one
+    thread block per SM allows; a grid of more blocks than SMs (here 4 x 16 x 3 = 192) takes the shallow ring with two
+    blocks per SM.  Same bits as the oracle, event lists included; the stream-weights flag keeps the weights out of
+    shared memory so that this launch is the one that runs."""
+    g = sb().SNN_FLAG_FORWARD_STREAM_WEIGHTS
+    w = wl.small(sizes=(64, 1540, 1540, 1028, 10), T=12, B=16, p_in=0.1, g_ff=(2.5, 1.5, 1.5), g_rec=(1.0, 1.0, 1.0), seed=59)
+    ref = _check_forward(orc32, w, wl.make(w), extra_flags=g)
+    assert all(float(x[1:].mean()) > 0.005 for x in ref["S"])
+
+
 def test_forward_c1_bit_exact(orc32):
     w = wl.WORKLOADS["c1"]
     ref = _check_forward(orc32, w, wl.make(w))
