@@ -147,9 +147,9 @@ snn_status snn_workspace_query_flags(const snn_net* net, int32_t T, int32_t B, c
  * Gradients are bit-identical across strategies for a given order, not between the two orders. */
 #define SNN_FLAG_BACKWARD_LAYER_BY_LAYER 8u
 #define SNN_FLAG_BACKWARD_WAVEFRONT 16u
-/* While the weights fit in L2 the recomputation passes take two launches per run of steps (the input
- * currents of all its steps from the stored events at once, then the leak/reset recurrence); this flag
- * forces one launch per step, the order used for larger networks.  Results are bit-identical either way. */
+/* The recomputation passes take two launches per run of steps (the input currents of all its steps from the
+ * stored events at once, thread blocks ordered so that those that run together gather from the same columns;
+ * then the leak/reset recurrence); this flag forces one launch per step.  Results are bit-identical either way. */
 #define SNN_FLAG_REFORWARD_PER_STEP 32u
 /* Networks whose weights exceed L2 compute those input currents with the weight rows as the stationary
  * operand instead: a thread block reads each row of its column slab once per run and adds it to every
