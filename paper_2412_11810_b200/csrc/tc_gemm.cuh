@@ -7,6 +7,9 @@
 // and not HBM sets the pace).  fp32 accuracy comes from three tf32 products per k-block, small terms first:
 // x = hi + lo with hi = x cut to 10 mantissa bits and lo = (x - hi) cut likewise (hi + lo differs from x by
 // less than 2^-20 |x|), D += W_lo d_hi + W_hi d_lo + W_hi d_hi with fp32 accumulators in tensor memory.
+// The cutting is the tensor cores' own: a kind::tf32 operand is read as its 19 high bits (checked on the device:
+// results are bit for bit the same with the operands cut beforehand), so the staged fp32 tile itself serves as hi and
+// only lo = x - cut(x) is computed and written, to a second tile.
 // The tensor cores do not round an accumulation to nearest, and the error of a long chain of accumulations into
 // one accumulator grows with its length; so the work is spread over three accumulators, summed in fp32 at the
 // end: one for the two small terms of every k-step (they are 2^-11 of the large one: their own rounding no longer
@@ -17,7 +20,7 @@
 //               [128 rows][32 k] and the delta tile [pairs][32 k] (a 3-D box: k, sample, step)
 //   warp 1      allocates tensor memory; one thread issues the tcgen05.mma instructions (12 per k-block) and
 //               commits them to the mbarrier that frees the stage
-//   warps 2-9   split every staged value into hi (in place) and lo (a second tile); warps 2-5 later read the
+//   warps 2-9   write lo = x - cut(x) of every staged value to a second tile; warps 2-5 later read the
 //               accumulator back (tcgen05.ld: a warp reads the 32 lanes 32 (warp % 4) ..) and store it
 // Per stage three mbarriers: bytes landed -> split done -> products done.  All waits are bounded; a wait that
 // runs out raises STATUS_SYNC_TIMEOUT, every role leaves its loop, and tensor memory is still released.
@@ -187,8 +190,8 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
       umma_commit(bar_acc);                   // ... and the accumulator read once all of them are
     }
   } else {
-    // ---- split: every 16-byte piece of the landed tiles -> hi in place, lo in the second tile (same position:
-    // the swizzle is a permutation of positions, the split is elementwise)
+    // ---- split: every 16-byte piece of the landed tiles -> its lo piece in the second tile (same position: the
+    // swizzle is a permutation of positions, the split is elementwise); the landed tile itself is read as hi
     const int ctid = tid - 64;   // 0 .. 255
     const int b_pieces = p.n_cols * (TCG_KB / 4);
     bool ok = true;
@@ -200,25 +203,17 @@ __global__ void __launch_bounds__(TCG_THREADS, 1) ff_gemm_tc_kernel(const __grid
       float4* const al = reinterpret_cast<float4*>(stage_a_lo(s));
       float4* const bh = reinterpret_cast<float4*>(stage_b_hi(s));
       float4* const bl = reinterpret_cast<float4*>(stage_b_lo(s));
-      // both pieces are cut to tf32 here, so that what the tensor cores read needs no rounding of theirs
       auto cut = [](float v) { return __uint_as_float(__float_as_uint(v) & 0xffffe000u); };
-      auto split4 = [&](float4 x, float4& hi, float4& lo) {
-        hi.x = cut(x.x); lo.x = cut(x.x - hi.x);
-        hi.y = cut(x.y); lo.y = cut(x.y - hi.y);
-        hi.z = cut(x.z); lo.z = cut(x.z - hi.z);
-        hi.w = cut(x.w); lo.w = cut(x.w - hi.w);
+      auto lo4 = [&](float4 x) {
+        return make_float4(x.x - cut(x.x), x.y - cut(x.y), x.z - cut(x.z), x.w - cut(x.w));
       };
 #pragma unroll
       for (int q = 0; q < (int)(TCG_A_BYTES / 16) / (32 * TCG_CONV_WARPS); ++q) {
         const int i = ctid + q * 32 * TCG_CONV_WARPS;
-        float4 hi, lo;
-        split4(ah[i], hi, lo);
-        ah[i] = hi; al[i] = lo;
+        al[i] = lo4(ah[i]);
       }
       for (int i = ctid; i < b_pieces; i += 32 * TCG_CONV_WARPS) {
-        float4 hi, lo;
-        split4(bh[i], hi, lo);
-        bh[i] = hi; bl[i] = lo;
+        bl[i] = lo4(bh[i]);
       }
       fence_proxy_async_smem();   // these writes are read by the tensor cores (asynchronous proxy)
       __syncwarp();
