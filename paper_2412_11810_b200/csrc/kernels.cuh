@@ -919,12 +919,6 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
       const uint4 x = reinterpret_cast<const uint4*>(evs)[i];
       e[4 * i] = x.x; e[4 * i + 1] = x.y; e[4 * i + 2] = x.z; e[4 * i + 3] = x.w;
     }
-    uint32_t rw[RR_PPW];
-#pragma unroll
-    for (int i = 0; i < RR_PPW / 4; ++i) {
-      const uint4 x = reinterpret_cast<const uint4*>(evs + p.pb)[i];
-      rw[4 * i] = x.x; rw[4 * i + 1] = x.y; rw[4 * i + 2] = x.z; rw[4 * i + 3] = x.w;
-    }
     // one event: the row's 16 bytes of this lane, two packed additions
     auto add_row = [&](int i, uint32_t r) {
       unsigned long long w01, w23;
@@ -943,12 +937,13 @@ __global__ void __launch_bounds__(32 * (RR_MAX_PB / RR_PPW + 1)) refwd_rows_kern
     for (int i = 0; i < RR_PPW; ++i) {
       const uint32_t cnt = e[i] & 7u;
       if (cnt > 1) add_row(i, (e[i] >> 16) & 0xffu);
-      if (cnt > 2) {
+      if (cnt > 2) {   // the second word of the pair is read only here: one block in five has more than two events
+        const uint32_t rw = evs[p.pb + i];
         if (cnt != RR_EV_MANY) {
-          add_row(i, rw[i] & 0xffu);
-          add_row(i, (rw[i] >> 8) & 0xffu);
+          add_row(i, rw & 0xffu);
+          add_row(i, (rw >> 8) & 0xffu);
         } else {
-          uint32_t bits = rw[i];
+          uint32_t bits = rw;
           bits &= bits - 1;
           bits &= bits - 1;
           while (bits) {
