@@ -294,7 +294,7 @@ struct FwdParams {
 };
 
 constexpr int GATHER_ROWS = 8;     // weight rows per copy group
-constexpr int GATHER_STAGES = 3;   // copy groups in flight per thread (24 rows, 48 KB per CTA: four CTAs per SM)
+constexpr int GATHER_STAGES = 3;   // groups of rows in the copy ring of a forward step (24 rows, 48 KB per CTA: three CTAs per SM)
 constexpr size_t FWD_DYN_SMEM = (size_t)GATHER_STAGES * GATHER_ROWS * FWD_THREADS * sizeof(float4);
 
 // The producer warp's share of a gather: the n listed rows (addresses in s_row) go into the ring as bulk copies, eight
