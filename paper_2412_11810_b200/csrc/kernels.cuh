@@ -765,7 +765,7 @@ __global__ void __launch_bounds__(128) refwd_scan_kernel(const __grid_constant__
 // (a block with more keeps its raw spike word instead).  refwd_rows_kernel then streams the rows: one
 // elected thread issues, per block of 32 rows, one tiled bulk copy (TMA) of the [32 rows][128 columns] tile
 // and one bulk copy of the pairs' event words into a ring of RR_STAGES stages guarded by full / empty
-// mbarriers; the other warps consume: a warp owns 8 pairs, a lane four adjacent columns (8 float4
+// mbarriers; the other warps consume: a warp owns 4 pairs, a lane four adjacent columns (4 float4
 // accumulators per thread, named statically), and an event is one 16-byte shared-memory read and two packed
 // fp32 additions.
 struct RowsLayer {
@@ -797,9 +797,10 @@ struct RowsParams {
 constexpr int RR_COLS = 128;     // columns per CTA (32 lanes x 4)
 constexpr int RR_ROWS = 32;      // rows per tile: one spike word
 constexpr int RR_STAGES = 4;     // tiles in flight per CTA
-constexpr int RR_PPW = 8;        // pairs per consumer warp (32 accumulator registers per thread: many warps per SM
-                                 // hide the shared-memory latency of the data-dependent row reads)
-constexpr int RR_MAX_PB = 128;   // at most 16 consumer warps
+constexpr int RR_PPW = 4;        // pairs per consumer warp (16 accumulator registers per thread: many warps per SM
+                                 // hide the shared-memory latency of the data-dependent row reads; eight pairs per
+                                 // warp, half the warps: 69 against 60 ms for a pass over the largest benchmark network)
+constexpr int RR_MAX_PB = 64;    // at most 16 consumer warps
 constexpr uint32_t RR_TILE_BYTES = RR_ROWS * RR_COLS * sizeof(float);
 constexpr uint32_t RR_STAGE_BYTES = RR_TILE_BYTES + RR_COLS * sizeof(float);   // the tile and one row of zeros after it
 constexpr uint32_t RR_EV_MANY = 7u;   // count field of an event word whose block has more than four firing rows

@@ -58,8 +58,8 @@ def test_workspace_query_and_bad_intervals():
     assert p0 == 0 and p1 == 0 and p2 == 10 * ms
     # same event storage, different number of dense states: T+1, K + T/K, K + 2 (256-byte rounding aside);
     # the strategies that recompute also hold two words per (32 presynaptic rows, step of a chunk, sample),
-    # the pairs rounded up to 128: here 2 blocks of rows
-    scratch = 2 * 4 * 128 * 2
+    # the pairs rounded up to 64: here 2 blocks of rows
+    scratch = 2 * 4 * 64 * 2
     assert abs((d0 - (d1 - scratch)) - ms * (101 - 20)) < 512 and abs((d1 - d2) - ms * (20 - 12)) < 512
     d3, p3 = sb.snn_workspace_query(net, 100, 2, sb.snn_ckpt(sb.SNN_DOUBLE, 5, 20), 0.25)
     d4, p4 = sb.snn_workspace_query(net, 100, 2, sb.snn_ckpt(sb.SNN_DOUBLE_LOCAL, 5, 20), 0.25)
